@@ -1,0 +1,253 @@
+/*
+ * mrl.h -- C ABI of libmrl: the token-level policy-loss pass that every learner of
+ * Mutual RL (GRPO base update with PRP / XGRPO / SGT experience sharing) runs on each
+ * optimisation step, as hand-written CUDA for NVIDIA B200 (sm_100a).
+ *
+ * Conventions that hold for every entry point unless its comment says otherwise
+ * ---------------------------------------------------------------------------
+ *  - Plain C.  Every function returns an int status (MRL_OK = 0 or an MRL_ERR_* code) and
+ *    never throws.  mrl_status_string() names a code.
+ *  - Pointers marked [device] are CUDA device pointers, valid on the current device, owned by
+ *    the caller, alive until the work enqueued by the call has finished.  Pointers marked
+ *    [host] are read during the call only.  Nothing is allocated, freed or retained.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  All work
+ *    is enqueued on it; the call does not synchronise and may return before the work runs.
+ *  - Argument errors are detected on the host before anything is enqueued (MRL_ERR_INVALID_ARG,
+ *    MRL_ERR_UNSUPPORTED_DTYPE, MRL_ERR_WORKSPACE_TOO_SMALL).  A failed launch gives MRL_ERR_CUDA.
+ *  - Errors that only the device can see never fault: the kernel ORs a bit into the caller's
+ *    `status` word [device, int32[1], nullable], treats the offending row as masked and goes
+ *    on.  The library never clears `status`; zero it before the first call and read it after
+ *    your own synchronisation.  Bits: MRL_DEV_BAD_TOKEN_ID (an id outside [0, V)),
+ *    MRL_DEV_TIMEOUT (a bounded wait on the kernel's own asynchronous copy ran out; outputs of
+ *    that call are then unspecified).
+ *  - `workspace` [device] is scratch of at least mrl_workspace_bytes(...) bytes, 256-byte
+ *    aligned, contents unspecified before and after.  Calls that share a workspace must not
+ *    overlap on the device.
+ *  - Row-major everywhere.  "Row t" is one response-token position: its logits row predicts
+ *    ids[t] (the caller has already applied the next-token shift and dropped prompt rows).
+ *  - Notation follows the paper: P prompts, M policies, G (the paper's K) rollouts per policy
+ *    and prompt, S sequences, N rows, V vocabulary, H hidden size.
+ */
+#ifndef MRL_H_
+#define MRL_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define MRL_VERSION 100
+
+/* return codes */
+#define MRL_OK 0
+#define MRL_ERR_INVALID_ARG 1
+#define MRL_ERR_BAD_TOKEN_ID 2       /* reserved for host-side id checks; device checks use the status word */
+#define MRL_ERR_UNSUPPORTED_DTYPE 3
+#define MRL_ERR_WORKSPACE_TOO_SMALL 4
+#define MRL_ERR_CUDA 5
+#define MRL_ERR_TIMEOUT 6
+#define MRL_ERR_UNSUPPORTED_SHAPE 7
+
+/* bits of the device status word */
+#define MRL_DEV_BAD_TOKEN_ID 1
+#define MRL_DEV_TIMEOUT 2
+
+/* element types of logits / dlogits */
+#define MRL_F32 0
+#define MRL_BF16 1
+
+/* mrl_adv_params.mode: which normalisation of the group-centred reward (Sec. 3; App. A) */
+#define MRL_ADV_MEAN_ONLY 0     /* A = r - mean                                  (Sec. 3, A-tilde)    */
+#define MRL_ADV_GROUP_ZNORM 1   /* A = (r - mean) / (std_group + eps)            (Sec. 3, A-tilde-zn) */
+#define MRL_ADV_BATCH_ZNORM 2   /* A = (r - mean_group) / (std_batch + eps)      (App. A)             */
+
+/* mrl_adv_params.sgt_pick: how y* is chosen among the peer successes (App. B) */
+#define MRL_PICK_NONE 0
+#define MRL_PICK_FIRST 1        /* lowest flat index m*G+g */
+#define MRL_PICK_SHORTEST 2     /* smallest seq_len, ties to the lowest flat index ("shorter-response heuristic") */
+#define MRL_PICK_ALL 3          /* every peer success */
+#define MRL_PICK_SEEDED 4       /* the (splitmix64(seed*2^32 + p) mod n_success)-th success in flat order ("random choice") */
+
+/* mrl_loss_params.agg_mode */
+#define MRL_AGG_TOKEN_MEAN 0            /* one masked mean over all tokens */
+#define MRL_AGG_SEQ_MEAN_TOKEN_MEAN 1   /* Eq. (1): E_tok within each sequence, then the mean over sequences */
+
+/* mrl_loss_params.flags */
+#define MRL_FLAG_ACCUMULATE_LOSS 1u   /* loss[0..1] and stats += this call (micro-batch accumulation, App. A) */
+#define MRL_FLAG_SKIP_ZERO_ROWS 2u    /* rows whose gradient multiplier is known to be zero before reading the
+                                         logits (A = 0 or weight 0, and no NLL weight) are not read: logp = 0,
+                                         dlogits row = 0, they still count in the denominators */
+#define MRL_FLAG_ACCUMULATE_DW 4u     /* fused LM head: dW is float32 [V, H] and is added to, not overwritten */
+
+/* `which` of mrl_workspace_bytes */
+#define MRL_WS_TOKEN_LOGPROBS 0
+#define MRL_WS_POLICY_LOSS 1
+#define MRL_WS_FUSED_LMHEAD 2
+
+typedef struct mrl_adv_params {
+  int32_t mode;             /* MRL_ADV_* */
+  int32_t ddof;             /* 0: population std (divide by n), 1: sample std (n - 1) */
+  float eps;                /* added to the std (Sec. 3) */
+  float sgt_success_thr;    /* success iff r >  this (App. A: 0.8) */
+  float sgt_negative_thr;   /* negative iff r < this (App. A: 0.2) */
+  int32_t sgt_pick;         /* MRL_PICK_* */
+  uint64_t seed;            /* MRL_PICK_SEEDED only (low 32 bits used) */
+} mrl_adv_params;
+
+typedef struct mrl_loss_params {
+  float eps_lo;             /* clip band is [1 - eps_lo, 1 + eps_hi]; the paper uses 0.2 for both */
+  float eps_hi;
+  int32_t agg_mode;         /* MRL_AGG_* */
+  uint32_t flags;           /* MRL_FLAG_* */
+  double pg_denominator;    /* TOKEN_MEAN: number of valid tokens of the whole step when the step is fed in
+                               several calls; <= 0: the valid tokens of this call */
+  double seq_denominator;   /* SEQ_MEAN_TOKEN_MEAN: number of sequences of the whole step; <= 0: S */
+  float nll_coeff;          /* lambda_SGT / n_gated (Eq. (2), App. B); 0 disables the NLL term */
+  int32_t reserved;
+} mrl_loss_params;
+
+/*
+ * mrl_group_advantages -- group-relative advantages and the SGT rescue gate.
+ *
+ * Defined by: Sec. 3 (r-bar, A-tilde, A-tilde-zn); App. A (group mean then batch whitening);
+ * Sec. 5.1 (PRP: advantages normalised over the unified pool of own and peer rollouts);
+ * App. H, value-level coupling (XGRPO: mu_pool, sigma_pool over all M*K rewards of the prompt);
+ * Sec. 5.3, App. A, App. B (SGT: gate = the learner has no success among its G rollouts and a
+ * peer has one; success r > 0.8, negative r < 0.2; one peer success per learner and prompt).
+ *
+ *   rewards        [device] float32 [P, M, G]
+ *   seq_len        [device] int32   [P, M, G] response lengths; nullable unless sgt_pick = SHORTEST
+ *   learner        index in [0, M) of the policy the gate is evaluated for
+ *   ap             [host]
+ *   adv_own        [device] float32 [P, M, G]  each policy normalised within its own group; nullable
+ *   adv_pool       [device] float32 [P, M, G]  normalised over the M*G rewards of the prompt; nullable
+ *   rescue         [device] uint8   [P]        1 where the gate fires for `learner`; nullable
+ *   pick           [device] int32   [P]        flat index m*G+g of the selected peer success, -1 if
+ *                                              none (lowest selected index for PICK_ALL); nullable
+ *   nll_seq_weight [device] float32 [P, M, G]  1.0 on selected rollouts, else 0; nullable
+ *   n_gated        [device] int32   [1]        number of selected rollouts; nullable
+ *
+ * BATCH_ZNORM divides adv_own by the std of the group-centred values of that policy's whole
+ * batch (its P*G values) and adv_pool by the std over all P*M*G pool-centred values.
+ * All outputs are overwritten.  Integer outputs are exact; thresholds are compared in float32.
+ * Limits: 1 <= M*G <= 1024.  Returns MRL_ERR_INVALID_ARG for sizes outside the limits, a
+ * learner outside [0, M), an unknown mode, or SHORTEST without seq_len.  P = 0 is a no-op.
+ */
+int mrl_group_advantages(const float* rewards, const int32_t* seq_len, int32_t P, int32_t M, int32_t G,
+                         int32_t learner, const mrl_adv_params* ap, float* adv_own, float* adv_pool,
+                         uint8_t* rescue, int32_t* pick, float* nll_seq_weight, int32_t* n_gated,
+                         void* stream);
+
+/*
+ * mrl_token_logprobs -- the token log-prob trace l_theta(x, y) of Sec. 3:
+ *   lse_t = log sum_v exp(z[t, v]),  logp_t = z[t, ids_t] - lse_t.
+ *
+ *   logits [device] dtype [N, ld], ld >= V elements between rows (read once)
+ *   dtype  MRL_BF16 or MRL_F32
+ *   ids    [device] int32 [N]
+ *   mask   [device] uint8 [N], nullable = all ones; rows with mask 0 are not read
+ *   logp   [device] float32 [N]; 0 on masked rows and rows with a bad id
+ *   lse    [device] float32 [N], nullable; 0 on those rows
+ *   workspace: mrl_workspace_bytes(MRL_WS_TOKEN_LOGPROBS, ...) (currently 0; may be NULL then)
+ *
+ * float32 accumulation; results are bitwise reproducible from run to run.
+ * N = 0 is a no-op.  V < 1, ld < V, N < 0, a null required pointer -> MRL_ERR_INVALID_ARG.
+ */
+int mrl_token_logprobs(const void* logits, int32_t dtype, int64_t N, int32_t V, int64_t ld,
+                       const int32_t* ids, const uint8_t* mask, float* logp, float* lse,
+                       int32_t* status, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * mrl_policy_loss_fwd_bwd -- the logits-in pass: log-probs, importance ratio, clipped
+ * surrogate, masked aggregation and the gradient with respect to the logits, with each logits
+ * row read from HBM once and each dlogits row written once.
+ *
+ * Defined by: Sec. 3 (w = exp(l_theta - l_old); Eq. (1)); Sec. 5.1 (PRP: the same update on
+ * peer text, with the learner-snapshot or the THL-aligned trace as `logp_old`); Sec. 5.3 Eq. (2)
+ * and App. B (SGT: lambda * NLL of the selected peer success, averaged per token and over the
+ * gated examples); App. H, proof of Prop. 1 (softmax score e_i - pi).
+ *
+ * With m_t the validity of row t (mask and id in range), len_s the valid tokens of sequence s:
+ *   c_t  = m_t / D                (TOKEN_MEAN,  D = pg_denominator)
+ *        = m_t / (S_d * len_s)    (SEQ_MEAN_TOKEN_MEAN, S_d = seq_denominator)
+ *   cn_t = nll_coeff * m_t * nll_weight_t / len_s
+ *   rho_t = exp(logp_t - logp_old_t),  A_t = adv_seq[sequence of t],  u_t = tok_weight_t
+ *   loss[0] = - sum_t c_t u_t min(rho_t A_t, clip(rho_t, 1-eps_lo, 1+eps_hi) A_t)
+ *   loss[1] = - sum_t cn_t logp_t
+ *   g_t = c_t u_t A_t rho_t [t unclipped] + cn_t
+ *   dlogits[t, v] = g_t (softmax(z_t)[v] - [v == ids_t])
+ * t is clipped iff (A_t > 0 and rho_t > 1+eps_hi) or (A_t < 0 and rho_t < 1-eps_lo); equality is
+ * unclipped.  Rows with c_t u_t A_t = 0 add exactly 0 to loss[0].
+ *
+ *   logits     [device] dtype [N, ld]
+ *   ids, mask  as in mrl_token_logprobs
+ *   cu_seqlens [device] int32 [S+1], non-decreasing, cu[0] = 0, cu[S] = N: sequence s owns rows
+ *              [cu[s], cu[s+1])
+ *   adv_seq    [device] float32 [S]
+ *   logp_old   [device] float32 [N] behaviour-policy trace; nullable = equal to logp (rho = 1)
+ *   tok_weight [device] float32 [N] stop-gradient weight u_t (PRP density weight); nullable = 1
+ *   nll_weight [device] float32 [N] SGT weight (1 on rows of a selected y*); nullable = 0
+ *   lp         [host]
+ *   dlogits    [device] dtype [N, ld_out]; may equal `logits` with ld_out = ld (in place);
+ *              nullable = forward only.  Every row is written (zeros where g_t = 0).
+ *   logp       [device] float32 [N], nullable
+ *   loss       [device] float32 [2]: policy-gradient term, NLL term
+ *   stats      [device] int64 [4], nullable: valid rows, clipped rows (valid, A != 0), rows
+ *              read from HBM, rows with a bad id
+ *   workspace: mrl_workspace_bytes(MRL_WS_POLICY_LOSS, N, V, 0, dtype, S)
+ *
+ * float32 row arithmetic on the input dtype, float64 for the final N-term sums (fixed order:
+ * bitwise reproducible).  dlogits is rounded to nearest even.  The fast path (one thread-block
+ * cluster per row, row resident in shared memory) needs bf16, V % 8 == 0, ld % 8 == 0,
+ * ld_out % 8 == 0 and 16-byte aligned logits/dlogits; anything else takes a general kernel
+ * with the same results.  N = 0: loss (and stats) are zeroed unless ACCUMULATE_LOSS.
+ */
+int mrl_policy_loss_fwd_bwd(const void* logits, int32_t dtype, int64_t N, int32_t V, int64_t ld,
+                            const int32_t* ids, const uint8_t* mask, const int32_t* cu_seqlens,
+                            int32_t S, const float* adv_seq, const float* logp_old,
+                            const float* tok_weight, const float* nll_weight,
+                            const mrl_loss_params* lp, void* dlogits, int64_t ld_out, float* logp,
+                            float* loss, int64_t* stats, int32_t* status, void* workspace,
+                            size_t workspace_bytes, void* stream);
+
+/*
+ * mrl_fused_lmhead_loss_fwd_bwd -- the hidden-in pass: the same loss with z = hidden W^T formed
+ * tile by tile on the tensor cores and reduced on the fly, so the [N, V] logits are never
+ * stored; backward gives dHidden = dZ W and dW = dZ^T hidden.
+ *
+ * Defined by: the same passages as mrl_policy_loss_fwd_bwd (the paper's l_theta is the log-softmax
+ * of the learner's output layer; it says nothing about the LM head itself).
+ *
+ *   hidden  [device] bf16 [N, H]   (contiguous, 16-byte aligned, H % 64 == 0)
+ *   W       [device] bf16 [V, H]   (contiguous, 16-byte aligned)
+ *   ids .. lp  as in mrl_policy_loss_fwd_bwd
+ *   dHidden [device] bf16 [N, H], overwritten
+ *   dW      [device] bf16 [V, H], overwritten; with MRL_FLAG_ACCUMULATE_DW float32 [V, H], added to
+ *   logp, loss, stats, status  as above
+ *   workspace: mrl_workspace_bytes(MRL_WS_FUSED_LMHEAD, N, V, H, MRL_BF16, S)
+ *
+ * bf16 operands, float32 accumulation; dZ is rounded to bf16 before the two backward products.
+ */
+int mrl_fused_lmhead_loss_fwd_bwd(const void* hidden, const void* W, int64_t N, int32_t H, int32_t V,
+                                  const int32_t* ids, const uint8_t* mask, const int32_t* cu_seqlens,
+                                  int32_t S, const float* adv_seq, const float* logp_old,
+                                  const float* tok_weight, const float* nll_weight,
+                                  const mrl_loss_params* lp, void* dHidden, void* dW, float* logp,
+                                  float* loss, int64_t* stats, int32_t* status, void* workspace,
+                                  size_t workspace_bytes, void* stream);
+
+/* Scratch bytes an entry point needs for the given sizes (0 if none).  Pure host arithmetic. */
+size_t mrl_workspace_bytes(int32_t which, int64_t N, int32_t V, int32_t H, int32_t dtype, int32_t S);
+
+/* Static, NUL-terminated name of a return code. */
+const char* mrl_status_string(int code);
+
+/* MRL_VERSION of the loaded library. */
+int mrl_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MRL_H_ */

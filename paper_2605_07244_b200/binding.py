@@ -1,0 +1,158 @@
+"""ctypes binding of libmrl.so: same names as the C ABI, argument marshalling only.
+
+Tensors are torch tensors used as device (or pinned host) memory; every step of the path runs
+inside the library's CUDA kernels.  There is no fallback: a missing library raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+from .build import LIB_PATH
+
+OK = 0
+F32, BF16 = 0, 1
+ADV_MEAN_ONLY, ADV_GROUP_ZNORM, ADV_BATCH_ZNORM = 0, 1, 2
+PICK_NONE, PICK_FIRST, PICK_SHORTEST, PICK_ALL, PICK_SEEDED = 0, 1, 2, 3, 4
+AGG_TOKEN_MEAN, AGG_SEQ_MEAN_TOKEN_MEAN = 0, 1
+FLAG_ACCUMULATE_LOSS, FLAG_SKIP_ZERO_ROWS, FLAG_ACCUMULATE_DW = 1, 2, 4
+WS_TOKEN_LOGPROBS, WS_POLICY_LOSS, WS_FUSED_LMHEAD = 0, 1, 2
+DEV_BAD_TOKEN_ID, DEV_TIMEOUT = 1, 2
+
+EXPORTS = ("mrl_group_advantages", "mrl_token_logprobs", "mrl_policy_loss_fwd_bwd",
+           "mrl_fused_lmhead_loss_fwd_bwd", "mrl_workspace_bytes", "mrl_status_string", "mrl_version")
+
+
+class AdvParams(C.Structure):
+    _fields_ = [("mode", C.c_int32), ("ddof", C.c_int32), ("eps", C.c_float),
+                ("sgt_success_thr", C.c_float), ("sgt_negative_thr", C.c_float),
+                ("sgt_pick", C.c_int32), ("seed", C.c_uint64)]
+
+
+class LossParams(C.Structure):
+    _fields_ = [("eps_lo", C.c_float), ("eps_hi", C.c_float), ("agg_mode", C.c_int32),
+                ("flags", C.c_uint32), ("pg_denominator", C.c_double), ("seq_denominator", C.c_double),
+                ("nll_coeff", C.c_float), ("reserved", C.c_int32)]
+
+
+class MrlError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} ({code})")
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """The loaded library; raises if it has not been built (there is no other code path)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2605_07244_b200.build` "
+                               "(or __graft_entry__.build()) first; there is no CPU fallback")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, i64, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_size_t
+        L.mrl_group_advantages.argtypes = [vp, vp, i32, i32, i32, i32, C.POINTER(AdvParams), vp, vp, vp, vp, vp, vp, vp]
+        L.mrl_group_advantages.restype = C.c_int
+        L.mrl_token_logprobs.argtypes = [vp, i32, i64, i32, i64, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.mrl_token_logprobs.restype = C.c_int
+        L.mrl_policy_loss_fwd_bwd.argtypes = [vp, i32, i64, i32, i64, vp, vp, vp, i32, vp, vp, vp, vp,
+                                              C.POINTER(LossParams), vp, i64, vp, vp, vp, vp, vp, sz, vp]
+        L.mrl_policy_loss_fwd_bwd.restype = C.c_int
+        L.mrl_fused_lmhead_loss_fwd_bwd.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, vp, vp, vp,
+                                                    C.POINTER(LossParams), vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.mrl_fused_lmhead_loss_fwd_bwd.restype = C.c_int
+        L.mrl_workspace_bytes.argtypes = [i32, i64, i32, i32, i32, i32]
+        L.mrl_workspace_bytes.restype = sz
+        L.mrl_status_string.argtypes = [C.c_int]
+        L.mrl_status_string.restype = C.c_char_p
+        L.mrl_version.argtypes = []
+        L.mrl_version.restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def _p(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return BF16
+    if t.dtype == torch.float32:
+        return F32
+    raise MrlError(3, "dtype")
+
+
+def _check(code: int, where: str):
+    if code != OK:
+        raise MrlError(code, where)
+
+
+def status_string(code: int) -> str:
+    return lib().mrl_status_string(code).decode()
+
+
+def version() -> int:
+    return lib().mrl_version()
+
+
+def workspace_bytes(which: int, N: int, V: int, H: int = 0, dtype: int = BF16, S: int = 0) -> int:
+    return int(lib().mrl_workspace_bytes(which, N, V, H, dtype, S))
+
+
+def mrl_group_advantages(rewards, seq_len, learner: int, ap: AdvParams, adv_own=None, adv_pool=None,
+                         rescue=None, pick=None, nll_seq_weight=None, n_gated=None, stream=None):
+    P, M, G = rewards.shape
+    _check(lib().mrl_group_advantages(_p(rewards), _p(seq_len), P, M, G, learner, C.byref(ap), _p(adv_own),
+                                      _p(adv_pool), _p(rescue), _p(pick), _p(nll_seq_weight), _p(n_gated),
+                                      _stream(stream)), "mrl_group_advantages")
+
+
+def mrl_token_logprobs(logits, ids, mask, logp, lse=None, status=None, workspace=None, V=None, stream=None):
+    N = logits.shape[0]
+    V = logits.shape[1] if V is None else V
+    ld = logits.stride(0) if N > 1 else max(logits.shape[1], V)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib().mrl_token_logprobs(_p(logits), _dtype_code(logits), N, V, ld, _p(ids), _p(mask), _p(logp),
+                                    _p(lse), _p(status), _p(workspace), ws_bytes, _stream(stream)),
+           "mrl_token_logprobs")
+
+
+def mrl_policy_loss_fwd_bwd(logits, ids, mask, cu_seqlens, adv_seq, logp_old, tok_weight, nll_weight,
+                            lp: LossParams, dlogits, logp, loss, stats=None, status=None, workspace=None,
+                            V=None, stream=None):
+    N = logits.shape[0]
+    V = logits.shape[1] if V is None else V
+    S = cu_seqlens.numel() - 1
+    ld = logits.stride(0) if N > 1 else max(logits.shape[1], V)
+    ld_out = ld if dlogits is None else (dlogits.stride(0) if N > 1 else max(dlogits.shape[1], V))
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib().mrl_policy_loss_fwd_bwd(_p(logits), _dtype_code(logits), N, V, ld, _p(ids), _p(mask),
+                                         _p(cu_seqlens), S, _p(adv_seq), _p(logp_old), _p(tok_weight),
+                                         _p(nll_weight), C.byref(lp), _p(dlogits), ld_out, _p(logp), _p(loss),
+                                         _p(stats), _p(status), _p(workspace), ws_bytes, _stream(stream)),
+           "mrl_policy_loss_fwd_bwd")
+
+
+def mrl_fused_lmhead_loss_fwd_bwd(hidden, W, ids, mask, cu_seqlens, adv_seq, logp_old, tok_weight, nll_weight,
+                                  lp: LossParams, dHidden, dW, logp, loss, stats=None, status=None,
+                                  workspace=None, stream=None):
+    N, H = hidden.shape
+    V = W.shape[0]
+    S = cu_seqlens.numel() - 1
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib().mrl_fused_lmhead_loss_fwd_bwd(_p(hidden), _p(W), N, H, V, _p(ids), _p(mask), _p(cu_seqlens), S,
+                                               _p(adv_seq), _p(logp_old), _p(tok_weight), _p(nll_weight),
+                                               C.byref(lp), _p(dHidden), _p(dW), _p(logp), _p(loss), _p(stats),
+                                               _p(status), _p(workspace), ws_bytes, _stream(stream)),
+           "mrl_fused_lmhead_loss_fwd_bwd")

@@ -1,0 +1,127 @@
+// Shared device/host helpers of libmrl (sm_100a only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "mrl.h"
+
+#define MRL_LOG2E 1.4426950408889634f
+#define MRL_LN2 0.6931471805599453f
+
+#define MRL_CUDA_OK(expr)                       \
+  do {                                          \
+    cudaError_t e__ = (expr);                   \
+    if (e__ != cudaSuccess) return MRL_ERR_CUDA; \
+  } while (0)
+
+static inline size_t mrl_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Carves sub-buffers out of the caller's workspace; every piece is 256-byte aligned.
+struct MrlCarver {
+  char* base;
+  size_t off;
+  explicit MrlCarver(void* p) : base(static_cast<char*>(p)), off(0) {}
+  template <typename T>
+  T* take(size_t n) {
+    T* p = reinterpret_cast<T*>(base + off);
+    off += mrl_align_up(n * sizeof(T), 256);
+    return p;
+  }
+};
+
+namespace mrl {
+
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__device__ __forceinline__ float bf16lo_to_f32(uint32_t packed) { return __uint_as_float(packed << 16); }
+__device__ __forceinline__ float bf16hi_to_f32(uint32_t packed) { return __uint_as_float(packed & 0xffff0000u); }
+
+// round-to-nearest-even pack of two floats: low half = a, high half = b
+__device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(b), "f"(a));
+  return r;
+}
+
+// Running log-sum-exp state in the base-2 domain: sum_i 2^(x_i - m), x = z * log2(e).
+struct Lse2 {
+  float m;  // running maximum of the scaled values (-inf when empty)
+  float s;  // sum of 2^(x - m)
+};
+
+__device__ __forceinline__ Lse2 lse2_empty() { return Lse2{-INFINITY, 0.f}; }
+
+__device__ __forceinline__ Lse2 lse2_merge(Lse2 a, Lse2 b) {
+  float m = fmaxf(a.m, b.m);
+  if (m == -INFINITY) return Lse2{m, 0.f};
+  return Lse2{m, a.s * ex2_approx(a.m - m) + b.s * ex2_approx(b.m - m)};
+}
+
+__device__ __forceinline__ Lse2 lse2_warp_reduce(Lse2 v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    Lse2 w;
+    w.m = __shfl_xor_sync(0xffffffffu, v.m, o);
+    w.s = __shfl_xor_sync(0xffffffffu, v.s, o);
+    v = lse2_merge(v, w);
+  }
+  return v;
+}
+
+// Block-wide merge in a fixed order; every thread gets the result.  `scratch` holds 2*32 floats.
+template <int kThreads>
+__device__ __forceinline__ Lse2 lse2_block_reduce(Lse2 v, float* scratch) {
+  constexpr int kWarps = kThreads / 32;
+  v = lse2_warp_reduce(v);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (lane == 0) {
+    scratch[warp] = v.m;
+    scratch[32 + warp] = v.s;
+  }
+  __syncthreads();
+  Lse2 r = lse2_empty();
+  if (lane < kWarps) r = Lse2{scratch[lane], scratch[32 + lane]};
+  r = lse2_warp_reduce(r);
+  __syncthreads();
+  return r;
+}
+
+// Per-row scalar inputs of the loss and what the row contributes.
+struct RowIn {
+  float A;         // advantage of the row's sequence
+  float cu;        // c_t * u_t
+  float cn;        // NLL coefficient
+  float logp_old;  // behaviour trace (ignored when has_old is false)
+  bool has_old;
+};
+
+struct RowOut {
+  float logp;
+  float pg_term;   // -cu * min(rho A, clip(rho) A)
+  float nll_term;  // -cn * logp
+  float g;         // dlogits = g * (p - onehot)
+  bool clipped;
+};
+
+// Ratio, clipped surrogate and gradient multiplier of one valid row (Eq. (1), Eq. (2)).
+__device__ __forceinline__ RowOut mrl_row_loss(float logp, const RowIn& in, float eps_lo, float eps_hi) {
+  RowOut o;
+  o.logp = logp;
+  const float rho = in.has_old ? expf(logp - in.logp_old) : 1.0f;
+  const float lo = 1.0f - eps_lo, hi = 1.0f + eps_hi;
+  const bool live = (in.cu != 0.f) && (in.A != 0.f);
+  o.clipped = (in.A > 0.f && rho > hi) || (in.A < 0.f && rho < lo);
+  const float s = fminf(rho * in.A, fminf(fmaxf(rho, lo), hi) * in.A);
+  o.pg_term = live ? -in.cu * s : 0.f;
+  o.nll_term = (in.cn != 0.f) ? -in.cn * logp : 0.f;
+  o.g = ((live && !o.clipped) ? in.cu * in.A * rho : 0.f) + in.cn;
+  return o;
+}
+
+}  // namespace mrl

@@ -1,0 +1,104 @@
+"""Shared plumbing of the GPU parity tests: run the C ABI on one set of inputs, run the oracle on the
+same inputs, compare.  Tolerances are the ones the task states: ids / masks / gate outputs bit-exact,
+log-probs 1e-4 absolute, loss 1e-5 relative, bf16 gradients 1e-2 relative L2 (fp32 gradients 1e-5)."""
+from __future__ import annotations
+
+import torch
+
+from oracle import mrl_oracle as O
+from paper_2605_07244_b200 import binding as B
+
+LOGP_ATOL = 1e-4
+LOSS_RTOL = 1e-5
+GRAD_REL_L2_BF16 = 1e-2
+GRAD_REL_L2_F32 = 1e-5
+TIE_MARGIN = 2e-5     # |rho - clip bound| below this: fp32 and fp64 may legitimately disagree on "clipped"
+
+
+def dev(t, dtype=None):
+    if t is None:
+        return None
+    t = torch.as_tensor(t)
+    if dtype is not None:
+        t = t.to(dtype)
+    return t.cuda().contiguous()
+
+
+def make_lp(eps_lo=0.2, eps_hi=0.2, agg=0, flags=0, pg_den=0.0, seq_den=0.0, nll_coeff=0.0):
+    return B.LossParams(eps_lo, eps_hi, agg, flags, pg_den, seq_den, nll_coeff, 0)
+
+
+def oracle_lp(lp: B.LossParams) -> O.LossParams:
+    # float32 parameters are upcast exactly, as the kernel sees them
+    return O.LossParams(eps_lo=float(lp.eps_lo), eps_hi=float(lp.eps_hi), agg_mode=lp.agg_mode,
+                        pg_denominator=lp.pg_denominator, seq_denominator=lp.seq_denominator,
+                        nll_coeff=float(lp.nll_coeff))
+
+
+def run_gpu_policy_loss(logits, ids, mask, cu, adv, logp_old, tok_weight, nll_weight, lp, V=None,
+                        inplace=False, want_dlogits=True, loss_init=None, stats_init=None):
+    """All arguments are CPU tensors (or None); returns CPU results of the CUDA path."""
+    zl = dev(logits)
+    N = zl.shape[0]
+    Vv = zl.shape[1] if V is None else V
+    S = cu.numel() - 1
+    ws = torch.empty(max(B.workspace_bytes(B.WS_POLICY_LOSS, N, Vv, 0, B.BF16, S), 256), dtype=torch.uint8,
+                     device="cuda")
+    dl = None
+    if want_dlogits:
+        dl = zl if inplace else torch.full_like(zl, float("nan"))
+    logp = torch.full((N,), float("nan"), device="cuda")
+    loss = torch.full((2,), float("nan"), device="cuda") if loss_init is None else dev(loss_init)
+    stats = torch.full((4,), -1, dtype=torch.int64, device="cuda") if stats_init is None else dev(stats_init)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    B.mrl_policy_loss_fwd_bwd(zl, dev(ids, torch.int32), dev(mask, torch.uint8), dev(cu, torch.int32),
+                              dev(adv, torch.float32), dev(logp_old, torch.float32),
+                              dev(tok_weight, torch.float32), dev(nll_weight, torch.float32), lp, dl, logp, loss,
+                              stats, status, ws, V=Vv)
+    torch.cuda.synchronize()
+    return dict(logp=logp.cpu(), loss=loss.cpu(), stats=stats.cpu(), status=int(status.cpu()),
+                dlogits=None if dl is None else dl.cpu())
+
+
+def rel_l2(a, b):
+    a, b = a.double(), b.double()
+    den = float(b.norm())
+    return float((a - b).norm()) / den if den > 0 else float(a.norm())
+
+
+def compare_policy_loss(got, ref, V, dtype, check_stats=True, loss_floor=0.0):
+    """got: run_gpu_policy_loss output; ref: oracle.policy_loss output (float64, same inputs)."""
+    assert torch.isfinite(got["logp"]).all()
+    err = (got["logp"].double() - ref["logp"]).abs().max()
+    assert err <= LOGP_ATOL, f"logp abs err {err}"
+    for k, name in ((0, "loss_pg"), (1, "loss_nll")):
+        L = ref[name]
+        d = abs(float(got["loss"][k]) - L)
+        assert d <= LOSS_RTOL * max(abs(L), loss_floor) + 1e-12, f"{name}: got {float(got['loss'][k])} want {L}"
+    tie = ref["valid"] & (ref["margin"] < TIE_MARGIN)
+    if check_stats:
+        assert int(got["stats"][0]) == ref["stats"][0]
+        assert abs(int(got["stats"][1]) - ref["stats"][1]) <= int(tie.sum())
+    if got["dlogits"] is not None:
+        dz = got["dlogits"][:, :V].double()
+        want = ref["dlogits"]
+        assert torch.isfinite(dz).all()
+        keep = ~tie
+        tol = GRAD_REL_L2_BF16 if dtype == torch.bfloat16 else GRAD_REL_L2_F32
+        e = rel_l2(dz[keep], want[keep])
+        assert e <= tol, f"dlogits rel L2 {e}"
+        # rows that must be exactly zero are exactly zero
+        zero_rows = keep & (ref["g"] == 0)
+        assert dz[zero_rows].abs().max() == 0 if zero_rows.any() else True
+        # per-row check on rows with a gradient: no single row hides behind the global norm
+        live = keep & (ref["g"] != 0)
+        if live.any():
+            # (g = c u A rho + cn may cancel: the error scales with |c u A rho| + |cn|, not with |g|)
+            num = (dz[live] - want[live]).norm(dim=1)
+            cancel = ((ref["g"] - ref["cn"]).abs() + ref["cn"].abs())[live] / ref["g"][live].abs()
+            # and a row whose softmax is (nearly) one-hot has dz ~ 0: measure against |g|, the scale of g (p - onehot)
+            den = torch.maximum(want[live].norm(dim=1), ref["g"][live].abs()) * cancel
+            assert (num / den).max() <= 2 * tol, f"worst row rel L2 {(num / den).max()}"
+        for r in tie.nonzero()[:, 0].tolist():      # near-tie rows: either side of the clip is valid
+            alt = rel_l2(dz[r], want[r])
+            assert alt <= tol or dz[r].abs().max() == 0 or want[r].abs().max() == 0
