@@ -1,0 +1,412 @@
+#!/usr/bin/env python
+"""Benchmark of the policy-loss hot path on B200 (one process per GPU).
+
+    python bench.py --gpus N --steps K --warmup W [--impl reference] [--workload C2|C5]
+
+A step is one pass of the whole hot path over one batch of synthetic input: group advantages and
+SGT gate (mrl_group_advantages), then log-probs, ratio, clipped surrogate, aggregation and dlogits
+(mrl_policy_loss_fwd_bwd).  The workload at N = 1 is config 2 of the baseline (Qwen-size vocabulary,
+logits in, bf16, packed ragged sequences); each rank of an N-GPU run processes its own batch of the
+same shape (independent replicas, no data-path collective), so scaling is weak.
+
+Rank 0 prints ONE JSON line.  `--impl reference` times the CPU float64 oracle on a bounded sample
+of the same workload instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2605_07244_b200 import synth  # noqa: E402
+
+METRIC = "policy_loss_fwd_bwd_tokens_per_s"
+UNIT = "tokens/s"
+ORACLE_ROWS = 2048          # rows of the workload the CPU baseline is timed on
+REFERENCE_ROWS = 1024       # rows per step of the --impl reference arm
+
+
+# ------------------------------------------------------------------------------------------ helpers
+
+def measured_peaks():
+    """Measured roofline denominators; the stated fallback when the file is absent."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d["bf16_tflops"]),
+                    bf16_tflops_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+def profile_traffic(key: str):
+    """DRAM bytes per unit of the dominant kernel from the committed ncu summary (None if absent)."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    if not os.path.exists(path):
+        return None
+    with open(path) as f:
+        return json.load(f).get(key)
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, device_index: int, period_s: float = 0.005):
+        self.period = period_s
+        self.samples = []
+        self.reasons = set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        self._h = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            try:
+                uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+                self._h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + uuid) if not uuid.startswith("GPU-") else uuid)
+            except Exception:
+                self._h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._h = None
+
+    def _loop(self):
+        nv = self._nv
+        names = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+                 0x4: "sw_power_cap", 0x80: "hw_power_brake_slowdown"}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self._h is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2], "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(s)}
+
+
+def aggregate_over_ranks(local_ms: float, local_units: float, world: int):
+    """Max time over ranks and total units (the whole-job view); a no-op for one rank."""
+    if world == 1:
+        return local_ms, local_units
+    import torch.distributed as dist
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor([local_ms], dtype=torch.float64, device=dev)
+    u = torch.tensor([local_units], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+def barrier(world: int):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+# ------------------------------------------------------------------------------------------ workloads
+
+class LogitsInWorkload:
+    """Config 2: 8 prompts x G = 8, ragged lengths in [128, 1024] packed, V = 151,936, bf16 logits."""
+
+    def __init__(self, w: synth.Workload, seed: int, device):
+        from paper_2605_07244_b200 import binding as B
+        self.B = B
+        self.w = w
+        self.meta = synth.make_meta(w, seed)
+        self.batch = synth.make_batch(self.meta)
+        b = self.batch
+        self.N, self.V, self.S = b.N, w.V, b.S
+        P, M, G = w.P, w.M, w.G
+        dev = device
+        self.z = torch.empty(self.N, self.V, dtype=w.dtype, device=dev)
+        for a in range(0, self.N, w.rows_per_block):
+            e = min(self.N, a + w.rows_per_block)
+            self.z[a:e] = b.logits_rows(a, e, device=dev)
+        self.dz = torch.empty_like(self.z)
+        self.ids = b.ids.to(dev)
+        self.cu = b.cu_seqlens.to(dev)
+        self.rewards = self.meta.rewards.to(dev)
+        self.seq_len = self.meta.seq_len.to(dev)
+        self.adv_own = torch.empty(P, M, G, device=dev)
+        self.adv_pool = torch.empty(P, M, G, device=dev)
+        self.rescue = torch.empty(P, dtype=torch.uint8, device=dev)
+        self.pick = torch.empty(P, dtype=torch.int32, device=dev)
+        self.nllw_seq = torch.empty(P, M, G, device=dev)
+        self.n_gated = torch.empty(1, dtype=torch.int32, device=dev)
+        self.logp = torch.empty(self.N, device=dev)
+        self.loss = torch.zeros(2, device=dev)
+        self.stats = torch.zeros(4, dtype=torch.int64, device=dev)
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.ws = torch.empty(B.workspace_bytes(B.WS_POLICY_LOSS, self.N, self.V, 0, B.BF16, self.S),
+                              dtype=torch.uint8, device=dev)
+        self.ap = B.AdvParams(B.ADV_GROUP_ZNORM, 0, 1e-6, 0.8, 0.2, B.PICK_SHORTEST, 0)
+        self.lp = B.LossParams(0.2, 0.2, B.AGG_TOKEN_MEAN, 0, 0.0, 0.0, 0.0, 0)
+        # behaviour trace: logp_old = logp + N(0, 0.1); logp from the library's forward (input preparation)
+        B.mrl_token_logprobs(self.z, self.ids, None, self.logp)
+        self.logp_old = self.logp + b.noise.to(dev)
+        torch.cuda.synchronize()
+        self.kernels_per_step = 6    # adv_prompt, seq_count, row_coef, row (cluster), row_terms, finalize
+        self.bytes_per_token = 2 * self.V * self.z.element_size()   # read V + write V elements
+
+    def step(self, z=None, dz=None):
+        B = self.B
+        B.mrl_group_advantages(self.rewards, self.seq_len, 0, self.ap, self.adv_own, self.adv_pool, self.rescue,
+                               self.pick, self.nllw_seq, self.n_gated)
+        # M = 1: adv_own laid out [P, 1, G] is the per-sequence advantage in packed (p, g) order
+        B.mrl_policy_loss_fwd_bwd(self.z if z is None else z, self.ids, None, self.cu, self.adv_own, self.logp_old,
+                                  None, None, self.lp, self.dz if dz is None else dz, self.logp, self.loss,
+                                  self.stats, self.status, self.ws)
+
+    def tokens(self):
+        return self.N
+
+    def describe(self):
+        return {"workload": f"{self.w.name}: Qwen-scale vocab, logits-in: {self.w.P} prompts x G={self.w.G}, packed "
+                            "ragged T in [128,1024], V=151936, bf16 logits N(0,2^2) + one +12 spike per row, "
+                            "GRPO group z-norm, eps 0.2",
+                "rows": self.N, "sequences": self.S, "V": self.V, "logits_dtype": "bf16",
+                "l2": "inputs (%.1f GB logits) exceed the 126 MB L2; no flush needed" % (self.z.numel() * 2 / 1e9)}
+
+    # ---- end to end: host buffers in, host buffers out, copies inside the timed region
+    def e2e_setup(self):
+        self.h_z = torch.empty(self.z.shape, dtype=self.z.dtype, pin_memory=True)
+        self.h_z.copy_(self.z)
+        self.h_dz = torch.empty(self.z.shape, dtype=self.z.dtype, pin_memory=True)
+        self.h_small_in = [t.cpu().pin_memory() for t in (self.ids, self.cu, self.rewards, self.seq_len, self.logp_old)]
+        self.d_small_in = [self.ids, self.cu, self.rewards, self.seq_len, self.logp_old]
+        self.h_logp = torch.empty(self.N, pin_memory=True)
+        self.h_loss = torch.empty(2, pin_memory=True)
+        h2d = self.h_z.numel() * 2 + sum(t.numel() * t.element_size() for t in self.h_small_in)
+        d2h = self.h_dz.numel() * 2 + self.N * 4 + 8
+        return h2d, d2h
+
+    def e2e_step(self):
+        for h, d in zip(self.h_small_in, self.d_small_in):
+            d.copy_(h, non_blocking=True)
+        self.z.copy_(self.h_z, non_blocking=True)
+        self.step()
+        self.h_dz.copy_(self.dz, non_blocking=True)
+        self.h_logp.copy_(self.logp, non_blocking=True)
+        self.h_loss.copy_(self.loss, non_blocking=True)
+
+    # ---- CPU baseline: the oracle on the first ORACLE_ROWS rows of the same batch
+    def oracle_sample(self, rows):
+        from oracle import mrl_oracle as O
+        b = self.batch
+        rows = min(rows, self.N)
+        s_end = int(torch.searchsorted(b.cu_seqlens.long(), torch.tensor(rows), right=True)) - 1
+        s_end = max(s_end, 1)
+        n = int(b.cu_seqlens[s_end])
+        z = self.z[:n].cpu()
+        adv, _ = O.group_advantages(self.meta.rewards)
+        adv_seq = adv[b.seq_p.long(), b.seq_m.long(), b.seq_g.long()][:s_end]
+        args = (z, b.ids[:n], None, b.cu_seqlens[:s_end + 1], adv_seq, self.logp_old[:n].cpu())
+        return O, args, n
+
+
+def time_oracle(O, args, repeats=1):
+    best = None
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        O.policy_loss(*args, None, None, O.LossParams())
+        dt = time.perf_counter() - t0
+        best = dt if best is None else min(best, dt)
+    return best
+
+
+# ------------------------------------------------------------------------------------------ arms
+
+def run_reference(args, rank, world):
+    """The oracle as it stands on the host cores; each step is a bounded sample of the workload."""
+    if rank != 0:
+        return
+    from oracle import mrl_oracle as O
+    w = synth.CONFIGS[args.workload]
+    meta = synth.make_meta(w, args.seed)
+    batch = synth.make_batch(meta)
+    n_seq = 1
+    while int(batch.cu_seqlens[n_seq]) < REFERENCE_ROWS and n_seq < batch.S:
+        n_seq += 1
+    n = int(batch.cu_seqlens[n_seq])
+    z = batch.logits_rows(0, n)
+    adv, _ = O.group_advantages(meta.rewards)
+    adv_seq = adv[batch.seq_p.long(), batch.seq_m.long(), batch.seq_g.long()][:n_seq]
+    logp, _, _ = O.token_logprobs(z, batch.ids[:n])
+    logp_old = (logp + batch.noise[:n].double()).float()
+    call = (z, batch.ids[:n], None, batch.cu_seqlens[:n_seq + 1], adv_seq, logp_old)
+    for _ in range(min(args.warmup, 1)):
+        O.policy_loss(*call, None, None, O.LossParams())
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        O.group_advantages(meta.rewards)
+        O.policy_loss(*call, None, None, O.LossParams())
+    dt = time.perf_counter() - t0
+    value = n * args.steps / dt
+    cores = torch.get_num_threads()
+    sample = f"first {n} rows ({n_seq} sequences) of the workload per step, full V, fwd+bwd"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "rows_per_step": n, "V": w.V},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def run_e2e(args, wl, world):
+    e2e_steps = max(1, min(args.steps, 3))
+    h2d, d2h = wl.e2e_setup()
+    wl.e2e_step()
+    torch.cuda.synchronize()
+    barrier(world)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        wl.e2e_step()
+    e1.record()
+    torch.cuda.synchronize()
+    barrier(world)
+    e2e_ms, e2e_tokens = aggregate_over_ranks(e0.elapsed_time(e1), wl.tokens() * e2e_steps, world)
+    return {"value": e2e_tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+            "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+            "note": "C-ABI calls on device buffers bracketed by pinned-host copies of every input (logits "
+                    "included) and of dlogits, logp and loss"}
+
+
+def run_ours(args, rank, world, local_rank):
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    from paper_2605_07244_b200 import binding as B
+    from paper_2605_07244_b200 import build
+    build.build()
+    B.lib()
+    if args.workload not in ("C2", "C2s"):
+        raise SystemExit("bench.py times config 2 (logits-in); C2s is its small profiling case; "
+                         "other configs are parity-test cases")
+    wl = LogitsInWorkload(synth.CONFIGS[args.workload], args.seed + rank, device)
+    peaks = measured_peaks()
+
+    for _ in range(max(args.warmup, 3)):
+        wl.step()
+    torch.cuda.synchronize()
+
+    timer = B.DominantKernelTimer(args.steps)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier(world)
+    torch.cuda.synchronize()
+    with ClockSampler(local_rank) as clocks, timer:
+        ev0.record()
+        for _ in range(args.steps):
+            wl.step()
+        ev1.record()
+        torch.cuda.synchronize()
+    barrier(world)
+    local_ms = ev0.elapsed_time(ev1)
+    kernel_ms = timer.elapsed_ms(args.steps)
+    status = int(wl.status.cpu())
+    if status != 0:
+        raise SystemExit(f"device status word is {status} after the timed region")
+    total_ms, total_tokens = aggregate_over_ranks(local_ms, wl.tokens() * args.steps, world)
+    value = total_tokens / (total_ms * 1e-3)
+
+    # dominant kernel against the HBM roofline
+    k_avg_ms = sum(kernel_ms) / len(kernel_ms)
+    alg_bytes = wl.bytes_per_token * wl.tokens()
+    achieved = alg_bytes / (k_avg_ms * 1e-3) / 1e9
+    per_token = profile_traffic("row_cluster_kernel_dram_bytes_per_token_V151936")
+    roofline = {"bound": "hbm", "kernel": "row_cluster_kernel", "achieved": achieved, "peak": peaks["hbm_gbs"],
+                "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"] + " (copy, burst)",
+                "algorithmic_bytes_per_launch": alg_bytes, "kernel_ms": k_avg_ms,
+                "traffic": None if per_token is None else per_token * wl.tokens()}
+
+    # end to end: pinned host buffers -> device -> kernels -> pinned host buffers
+    e2e = None
+    if not args.no_e2e:
+        e2e = run_e2e(args, wl, world)
+
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        O, oargs, n = wl.oracle_sample(ORACLE_ROWS)
+        dt = time_oracle(O, oargs)
+        cpu_baseline = {"value": n / dt, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
+                        "sample": f"first {n} rows of the same batch, full V, fwd+bwd, float64, {dt:.1f} s"}
+
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": dict(wl.describe(), parallelism=f"replicas x{world}"),
+            "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": wl.kernels_per_step * args.steps,
+            "roofline": roofline, "cpu_baseline": cpu_baseline,
+        }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="C2")
+    ap.add_argument("--seed", type=int, default=2)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="profiling runs only: skip the host-buffer leg")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    try:
+        run_ours(args, rank, world, local_rank)
+    finally:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

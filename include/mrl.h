@@ -238,6 +238,17 @@ int mrl_fused_lmhead_loss_fwd_bwd(const void* hidden, const void* W, int64_t N, 
                                   float* loss, int64_t* stats, int32_t* status, void* workspace,
                                   size_t workspace_bytes, void* stream);
 
+/*
+ * mrl_profile_dominant_kernel -- instrumentation for benchmarks; the paper has no counterpart.
+ * Registers n pairs of CUDA events (cudaEvent_t passed as void*, created and owned by the caller).
+ * From then on every launch of an entry point's dominant kernel (the per-row kernel of
+ * mrl_token_logprobs / mrl_policy_loss_fwd_bwd; each tensor-core kernel of the fused LM head)
+ * records start_events[i % n] just before and stop_events[i % n] just after it on the call's
+ * stream, i counting such launches since registration.  n = 0 (or null arrays) unregisters.
+ * The arrays [host] must stay alive while registered.  Process-wide and not thread-safe.
+ */
+int mrl_profile_dominant_kernel(void** start_events, void** stop_events, int32_t n);
+
 /* Scratch bytes an entry point needs for the given sizes (0 if none).  Pure host arithmetic. */
 size_t mrl_workspace_bytes(int32_t which, int64_t N, int32_t V, int32_t H, int32_t dtype, int32_t S);
 

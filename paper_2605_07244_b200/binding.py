@@ -22,7 +22,7 @@ WS_TOKEN_LOGPROBS, WS_POLICY_LOSS, WS_FUSED_LMHEAD = 0, 1, 2
 DEV_BAD_TOKEN_ID, DEV_TIMEOUT = 1, 2
 
 EXPORTS = ("mrl_group_advantages", "mrl_token_logprobs", "mrl_policy_loss_fwd_bwd",
-           "mrl_fused_lmhead_loss_fwd_bwd", "mrl_workspace_bytes", "mrl_status_string", "mrl_version")
+           "mrl_fused_lmhead_loss_fwd_bwd", "mrl_workspace_bytes", "mrl_status_string", "mrl_version", "mrl_profile_dominant_kernel")
 
 
 class AdvParams(C.Structure):
@@ -69,6 +69,8 @@ def lib() -> C.CDLL:
         L.mrl_workspace_bytes.restype = sz
         L.mrl_status_string.argtypes = [C.c_int]
         L.mrl_status_string.restype = C.c_char_p
+        L.mrl_profile_dominant_kernel.argtypes = [C.POINTER(vp), C.POINTER(vp), i32]
+        L.mrl_profile_dominant_kernel.restype = C.c_int
         L.mrl_version.argtypes = []
         L.mrl_version.restype = C.c_int
         _lib = L
@@ -156,3 +158,28 @@ def mrl_fused_lmhead_loss_fwd_bwd(hidden, W, ids, mask, cu_seqlens, adv_seq, log
                                                C.byref(lp), _p(dHidden), _p(dW), _p(logp), _p(loss), _p(stats),
                                                _p(status), _p(workspace), ws_bytes, _stream(stream)),
            "mrl_fused_lmhead_loss_fwd_bwd")
+
+
+class DominantKernelTimer:
+    """Registers n CUDA-event pairs around the dominant kernel of the following calls; `elapsed_ms()`
+    returns the duration of every recorded launch (after a synchronise)."""
+
+    def __init__(self, n: int):
+        self.n = n
+        self.start = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
+        self.stop = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
+        for e in self.start + self.stop:      # torch creates the CUDA event lazily: force it
+            e.record()
+        torch.cuda.synchronize()
+        self._a = (C.c_void_p * n)(*[e.cuda_event for e in self.start])
+        self._b = (C.c_void_p * n)(*[e.cuda_event for e in self.stop])
+
+    def __enter__(self):
+        _check(lib().mrl_profile_dominant_kernel(self._a, self._b, self.n), "mrl_profile_dominant_kernel")
+        return self
+
+    def __exit__(self, *exc):
+        lib().mrl_profile_dominant_kernel(None, None, 0)
+
+    def elapsed_ms(self, count: int):
+        return [self.start[i].elapsed_time(self.stop[i]) for i in range(min(count, self.n))]

@@ -34,3 +34,35 @@ extern "C" const char* mrl_status_string(int code) {
 }
 
 extern "C" int mrl_version(void) { return MRL_VERSION; }
+
+namespace {
+void** g_prof_start = nullptr;
+void** g_prof_stop = nullptr;
+int g_prof_n = 0;
+long long g_prof_i = 0;
+}  // namespace
+
+extern "C" int mrl_profile_dominant_kernel(void** start_events, void** stop_events, int32_t n) {
+  if (n < 0) return MRL_ERR_INVALID_ARG;
+  if (n == 0 || start_events == nullptr || stop_events == nullptr) {
+    g_prof_start = g_prof_stop = nullptr;
+    g_prof_n = 0;
+  } else {
+    g_prof_start = start_events;
+    g_prof_stop = stop_events;
+    g_prof_n = n;
+  }
+  g_prof_i = 0;
+  return MRL_OK;
+}
+
+void mrl_profile_before(cudaStream_t st) {
+  if (g_prof_n > 0) cudaEventRecord(static_cast<cudaEvent_t>(g_prof_start[g_prof_i % g_prof_n]), st);
+}
+
+void mrl_profile_after(cudaStream_t st) {
+  if (g_prof_n > 0) {
+    cudaEventRecord(static_cast<cudaEvent_t>(g_prof_stop[g_prof_i % g_prof_n]), st);
+    ++g_prof_i;
+  }
+}

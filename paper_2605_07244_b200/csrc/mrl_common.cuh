@@ -31,6 +31,10 @@ struct MrlCarver {
   }
 };
 
+// Benchmark instrumentation (mrl_profile_dominant_kernel): event pairs recorded around dominant kernels.
+void mrl_profile_before(cudaStream_t st);
+void mrl_profile_after(cudaStream_t st);
+
 namespace mrl {
 
 __device__ __forceinline__ float ex2_approx(float x) {

@@ -599,10 +599,12 @@ int launch_rows(RowParams p, int dtype, cudaStream_t st) {
   if (p.N > 0x7fffffffll / kMaxCluster) return MRL_ERR_UNSUPPORTED_SHAPE;
   const int C = pick_cluster(p, dtype);
   if (C == 0) {
+    mrl_profile_before(st);
     if (dtype == MRL_BF16)
       row_general_kernel<__nv_bfloat16><<<(unsigned)p.N, kThreads, 0, st>>>(p);
     else
       row_general_kernel<float><<<(unsigned)p.N, kThreads, 0, st>>>(p);
+    mrl_profile_after(st);
     return cudaGetLastError() == cudaSuccess ? MRL_OK : MRL_ERR_CUDA;
   }
   const int vecs = (p.V / 8 + C - 1) / C;
@@ -623,7 +625,9 @@ int launch_rows(RowParams p, int dtype, cudaStream_t st) {
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  mrl_profile_before(st);
   MRL_CUDA_OK(cudaLaunchKernelEx(&cfg, row_cluster_kernel, p));
+  mrl_profile_after(st);
   return MRL_OK;
 }
 

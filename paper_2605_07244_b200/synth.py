@@ -48,7 +48,9 @@ C3 = Workload("C3-prp-pool", P=16, M=2, G=8, V=128256, dtype=torch.bfloat16, own
 C4 = Workload("C4-xgrpo-sgt", P=64, M=2, G=16, V=151936, dtype=torch.bfloat16, own_len=(512, 512))
 C5 = Workload("C5-fused-lmhead", P=64, M=1, G=16, V=151936, dtype=torch.bfloat16, own_len=(64, 64),
               reward_beta=False, H=4096)
-CONFIGS = {"C1": C1, "C2": C2, "C3": C3, "C4": C4, "C5": C5}
+# config 2 with a quarter of the prompts: still far larger than L2, small enough for a profiler capture
+C2_SMALL = replace(C2, name="C2-qwen-vocab-2-prompts", P=2)
+CONFIGS = {"C1": C1, "C2": C2, "C3": C3, "C4": C4, "C5": C5, "C2s": C2_SMALL}
 
 
 def scaled(w: Workload, **kw) -> Workload:
