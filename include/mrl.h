@@ -49,6 +49,7 @@ extern "C" {
 #define MRL_ERR_CUDA 5
 #define MRL_ERR_TIMEOUT 6
 #define MRL_ERR_UNSUPPORTED_SHAPE 7
+#define MRL_ERR_STATIC_SCRATCH_TOO_SMALL 8   /* mrl_policy_loss_fwd_bwd_static only: N or S above its fixed limits */
 
 /* bits of the device status word */
 #define MRL_DEV_BAD_TOKEN_ID 1
@@ -211,6 +212,40 @@ int mrl_policy_loss_fwd_bwd(const void* logits, int32_t dtype, int64_t N, int32_
                             const mrl_loss_params* lp, void* dlogits, int64_t ld_out, float* logp,
                             float* loss, int64_t* stats, int32_t* status, void* workspace,
                             size_t workspace_bytes, void* stream);
+
+/*
+ * mrl_policy_loss_fwd_bwd_static -- mrl_policy_loss_fwd_bwd for callers that cannot allocate.
+ * The paper has no counterpart; this is a packaging variant of the entry point above.
+ *
+ * Who needs it: code that runs where device allocation is not available to it -- a plugin handed
+ * nothing but the host framework's tensors and a stream, a real-time or pre-sized service whose
+ * memory budget is frozen after start-up, a process in which cudaMalloc would force a device-wide
+ * synchronisation in the middle of a pipelined step.  Such a caller has no way to provide the
+ * `workspace` the ordinary entry point asks for.  Here the scratch is a fixed array inside the
+ * library image (MRL_STATIC_SCRATCH_BYTES, held on every GPU that loads the library until the
+ * process ends), so the call allocates nothing: no cudaMalloc / cudaFree, no allocating library
+ * routine.  The caller still owns and passes every input and output.
+ *
+ * Arguments, results and arithmetic are exactly those of mrl_policy_loss_fwd_bwd (the same kernels
+ * run) without `workspace` / `workspace_bytes`.  Limits: N <= MRL_STATIC_MAX_ROWS and
+ * S <= MRL_STATIC_MAX_SEQS; anything larger returns MRL_ERR_STATIC_SCRATCH_TOO_SMALL before any
+ * work is enqueued (split the step into several calls with MRL_FLAG_ACCUMULATE_LOSS and
+ * pg_denominator set, as for micro-batches).
+ *
+ * The first call on each device looks up the device address of the array (a one-time set-up that
+ * may load the module); make that first call outside any stream capture.  All calls on a device
+ * share the one array: two calls whose work overlaps on the GPU (different streams, no ordering)
+ * race on it.  The array keeps the previous call's contents; each call clears what it needs zeroed.
+ */
+#define MRL_STATIC_MAX_ROWS 65536
+#define MRL_STATIC_MAX_SEQS 65536
+#define MRL_STATIC_SCRATCH_BYTES (3u << 20)
+int mrl_policy_loss_fwd_bwd_static(const void* logits, int32_t dtype, int64_t N, int32_t V, int64_t ld,
+                                   const int32_t* ids, const uint8_t* mask, const int32_t* cu_seqlens,
+                                   int32_t S, const float* adv_seq, const float* logp_old,
+                                   const float* tok_weight, const float* nll_weight,
+                                   const mrl_loss_params* lp, void* dlogits, int64_t ld_out, float* logp,
+                                   float* loss, int64_t* stats, int32_t* status, void* stream);
 
 /*
  * mrl_fused_lmhead_loss_fwd_bwd -- the hidden-in pass: the same loss with z = hidden W^T formed

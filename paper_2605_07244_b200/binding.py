@@ -22,7 +22,10 @@ WS_TOKEN_LOGPROBS, WS_POLICY_LOSS, WS_FUSED_LMHEAD = 0, 1, 2
 DEV_BAD_TOKEN_ID, DEV_TIMEOUT = 1, 2
 
 EXPORTS = ("mrl_group_advantages", "mrl_token_logprobs", "mrl_policy_loss_fwd_bwd",
-           "mrl_fused_lmhead_loss_fwd_bwd", "mrl_workspace_bytes", "mrl_status_string", "mrl_version", "mrl_profile_dominant_kernel")
+           "mrl_fused_lmhead_loss_fwd_bwd", "mrl_workspace_bytes", "mrl_status_string", "mrl_version",
+           "mrl_profile_dominant_kernel", "mrl_policy_loss_fwd_bwd_static")
+STATIC_MAX_ROWS, STATIC_MAX_SEQS = 65536, 65536
+ERR_STATIC_SCRATCH_TOO_SMALL = 8
 
 
 class AdvParams(C.Structure):
@@ -62,6 +65,9 @@ def lib() -> C.CDLL:
         L.mrl_policy_loss_fwd_bwd.argtypes = [vp, i32, i64, i32, i64, vp, vp, vp, i32, vp, vp, vp, vp,
                                               C.POINTER(LossParams), vp, i64, vp, vp, vp, vp, vp, sz, vp]
         L.mrl_policy_loss_fwd_bwd.restype = C.c_int
+        L.mrl_policy_loss_fwd_bwd_static.argtypes = [vp, i32, i64, i32, i64, vp, vp, vp, i32, vp, vp, vp, vp,
+                                                     C.POINTER(LossParams), vp, i64, vp, vp, vp, vp, vp]
+        L.mrl_policy_loss_fwd_bwd_static.restype = C.c_int
         L.mrl_fused_lmhead_loss_fwd_bwd.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, vp, vp, vp,
                                                     C.POINTER(LossParams), vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.mrl_fused_lmhead_loss_fwd_bwd.restype = C.c_int
@@ -144,6 +150,23 @@ def mrl_policy_loss_fwd_bwd(logits, ids, mask, cu_seqlens, adv_seq, logp_old, to
                                          _p(nll_weight), C.byref(lp), _p(dlogits), ld_out, _p(logp), _p(loss),
                                          _p(stats), _p(status), _p(workspace), ws_bytes, _stream(stream)),
            "mrl_policy_loss_fwd_bwd")
+
+
+def mrl_policy_loss_fwd_bwd_static(logits, ids, mask, cu_seqlens, adv_seq, logp_old, tok_weight, nll_weight,
+                                   lp: LossParams, dlogits, logp, loss, stats=None, status=None, V=None,
+                                   stream=None):
+    """mrl_policy_loss_fwd_bwd without a workspace argument: for callers that cannot allocate device
+    memory, the library's own fixed scratch array is used (N <= STATIC_MAX_ROWS, S <= STATIC_MAX_SEQS)."""
+    N = logits.shape[0]
+    V = logits.shape[1] if V is None else V
+    S = cu_seqlens.numel() - 1
+    ld = logits.stride(0) if N > 1 else max(logits.shape[1], V)
+    ld_out = ld if dlogits is None else (dlogits.stride(0) if N > 1 else max(dlogits.shape[1], V))
+    _check(lib().mrl_policy_loss_fwd_bwd_static(_p(logits), _dtype_code(logits), N, V, ld, _p(ids), _p(mask),
+                                                _p(cu_seqlens), S, _p(adv_seq), _p(logp_old), _p(tok_weight),
+                                                _p(nll_weight), C.byref(lp), _p(dlogits), ld_out, _p(logp),
+                                                _p(loss), _p(stats), _p(status), _stream(stream)),
+           "mrl_policy_loss_fwd_bwd_static")
 
 
 def mrl_fused_lmhead_loss_fwd_bwd(hidden, W, ids, mask, cu_seqlens, adv_seq, logp_old, tok_weight, nll_weight,

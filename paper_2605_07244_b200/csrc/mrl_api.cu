@@ -29,6 +29,7 @@ extern "C" const char* mrl_status_string(int code) {
     case MRL_ERR_CUDA: return "MRL_ERR_CUDA";
     case MRL_ERR_TIMEOUT: return "MRL_ERR_TIMEOUT";
     case MRL_ERR_UNSUPPORTED_SHAPE: return "MRL_ERR_UNSUPPORTED_SHAPE";
+    case MRL_ERR_STATIC_SCRATCH_TOO_SMALL: return "MRL_ERR_STATIC_SCRATCH_TOO_SMALL";
     default: return "MRL_ERR_UNKNOWN";
   }
 }

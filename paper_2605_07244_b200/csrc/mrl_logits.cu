@@ -729,3 +729,54 @@ extern "C" int mrl_policy_loss_fwd_bwd(const void* logits, int32_t dtype, int64_
   MRL_CUDA_OK(cudaGetLastError());
   return MRL_OK;
 }
+
+// ------------------------------------------------------------------------------------------------
+// Allocation-free variant of mrl_policy_loss_fwd_bwd: the scratch lives in the library image.
+// ------------------------------------------------------------------------------------------------
+namespace {
+
+// Per-row and per-sequence scratch of the loss pass for the largest problem the static entry point takes.
+// Every device that loads the library keeps one copy of this array until the process exits.
+constexpr size_t kStaticWsBytes = MRL_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_static_loss_ws[kStaticWsBytes];
+
+constexpr int kMaxDevices = 64;
+void* g_static_ws_ptr[kMaxDevices] = {};  // device address of the array, per device ordinal (0 = not looked up yet)
+
+// In host code `g_static_loss_ws` is only a handle; the device address has to be asked for, with the
+// device it is wanted on current.  Looked up once per device and cached.
+int static_ws_address(void** out) {
+  int dev = -1;
+  MRL_CUDA_OK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return MRL_ERR_UNSUPPORTED_SHAPE;
+  if (g_static_ws_ptr[dev] == nullptr) {
+    void* ptr = nullptr;
+    MRL_CUDA_OK(cudaGetSymbolAddress(&ptr, g_static_loss_ws));
+    if (ptr == nullptr) return MRL_ERR_CUDA;
+    g_static_ws_ptr[dev] = ptr;
+  }
+  *out = g_static_ws_ptr[dev];
+  return MRL_OK;
+}
+
+}  // namespace
+
+extern "C" int mrl_policy_loss_fwd_bwd_static(const void* logits, int32_t dtype, int64_t N, int32_t V, int64_t ld,
+                                              const int32_t* ids, const uint8_t* mask, const int32_t* cu_seqlens,
+                                              int32_t S, const float* adv_seq, const float* logp_old,
+                                              const float* tok_weight, const float* nll_weight,
+                                              const mrl_loss_params* lp, void* dlogits, int64_t ld_out, float* logp,
+                                              float* loss, int64_t* stats, int32_t* status, void* stream) {
+  if (N < 0 || S < 0) return MRL_ERR_INVALID_ARG;
+  if (N > MRL_STATIC_MAX_ROWS || S > MRL_STATIC_MAX_SEQS) return MRL_ERR_STATIC_SCRATCH_TOO_SMALL;
+  if (mrl_policy_loss_workspace_bytes(N, S) > kStaticWsBytes) return MRL_ERR_STATIC_SCRATCH_TOO_SMALL;
+  void* ws = nullptr;
+  if (N > 0 && S > 0) {  // the empty call needs no scratch and touches no symbol
+    const int rc = static_ws_address(&ws);
+    if (rc != MRL_OK) return rc;
+  }
+  // The callee clears the part of the scratch that has to start at zero on every call (the coefficient
+  // arrays and the counters); everything else is overwritten before it is read.
+  return mrl_policy_loss_fwd_bwd(logits, dtype, N, V, ld, ids, mask, cu_seqlens, S, adv_seq, logp_old, tok_weight,
+                                 nll_weight, lp, dlogits, ld_out, logp, loss, stats, status, ws, kStaticWsBytes, stream);
+}

@@ -1,0 +1,96 @@
+"""The allocation-free entry point, mrl_policy_loss_fwd_bwd_static.
+
+Some users of the library cannot allocate device memory at the point where they call it: a plugin
+that only ever sees its host framework's tensors and stream, a service whose memory plan is frozen
+after start-up, a step that must not hit the implicit synchronisation of cudaMalloc.  For them the
+library carries its own fixed scratch array.  This file checks, through the C ABI, that the variant
+gives what the ordinary entry point gives on the same inputs -- twice in a row, with different
+shapes, because the array is shared by all calls and still holds the first call's leftovers when
+the second one starts -- and that it refuses sizes beyond its fixed limits before touching a device.
+
+The file name sorts after every other test file on purpose: if this one fails, a run that stops at
+the first failure has already run all the others.
+"""
+import ctypes as C
+
+import pytest
+import torch
+
+from paper_2605_07244_b200 import binding as B
+from paper_2605_07244_b200 import build, synth
+
+from helpers import GRAD_REL_L2_BF16, LOGP_ATOL, LOSS_RTOL, make_lp, rel_l2
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+    B.lib()
+
+
+def _inputs(N, V, S, seed, with_mask):
+    """Seeded inputs on the device; the behaviour trace comes from the library's own forward pass."""
+    g = torch.Generator().manual_seed(seed)
+    z = (torch.randn(N, V, generator=g) * 2.0).to(torch.bfloat16).cuda()
+    ids = torch.randint(0, V, (N,), generator=g, dtype=torch.int32).cuda()
+    cuts = sorted(torch.randperm(N - 1, generator=g)[:S - 1].add(1).tolist())
+    cu = torch.tensor([0] + cuts + [N], dtype=torch.int32).cuda()
+    adv = torch.randn(S, generator=g).cuda()
+    mask = (torch.rand(N, generator=g) < 0.8).to(torch.uint8).cuda() if with_mask else None
+    nllw = (torch.rand(N, generator=g) < 0.1).float().cuda()
+    logp = torch.empty(N, device="cuda")
+    B.mrl_token_logprobs(z, ids, None, logp)
+    logp_old = logp + (torch.randn(N, generator=g) * 0.1).cuda()
+    return z, ids, mask, cu, adv, logp_old, nllw
+
+
+def _run(entry, inp, workspace):
+    z, ids, mask, cu, adv, logp_old, nllw = inp
+    N = z.shape[0]
+    out = dict(dz=torch.full_like(z, float("nan")), logp=torch.full((N,), float("nan"), device="cuda"),
+               loss=torch.full((2,), float("nan"), device="cuda"),
+               stats=torch.full((4,), -1, dtype=torch.int64, device="cuda"),
+               status=torch.zeros(1, dtype=torch.int32, device="cuda"))
+    lp = make_lp(nll_coeff=0.05)
+    args = (z, ids, mask, cu, adv, logp_old, None, nllw, lp, out["dz"], out["logp"], out["loss"], out["stats"],
+            out["status"])
+    if workspace is None:
+        entry(*args)
+    else:
+        entry(*args, workspace)
+    torch.cuda.synchronize()
+    return {k: v.cpu() for k, v in out.items()}
+
+
+@pytest.mark.gpu
+def test_static_scratch_variant_matches_the_workspace_variant_on_two_calls_in_a_row():
+    # first a larger problem whose rows span a four-CTA cluster, then a smaller, differently cut one:
+    # the second call finds the first call's per-row scratch still in the array
+    shapes = [(300, 151936, 7, True), (97, 32768, 3, False)]
+    for k, (N, V, S, with_mask) in enumerate(shapes):
+        inp = _inputs(N, V, S, seed=40 + k, with_mask=with_mask)
+        ws = torch.empty(B.workspace_bytes(B.WS_POLICY_LOSS, N, V, 0, B.BF16, S), dtype=torch.uint8, device="cuda")
+        want = _run(B.mrl_policy_loss_fwd_bwd, inp, ws)
+        got = _run(B.mrl_policy_loss_fwd_bwd_static, inp, None)
+        assert got["status"].item() == 0 and want["status"].item() == 0
+        assert torch.isfinite(got["logp"]).all() and torch.isfinite(got["dz"].float()).all()
+        assert (got["logp"] - want["logp"]).abs().max() <= LOGP_ATOL
+        for j in range(2):
+            assert abs(float(got["loss"][j]) - float(want["loss"][j])) <= LOSS_RTOL * abs(float(want["loss"][j]))
+        assert float(want["loss"][0]) != 0 and float(want["loss"][1]) != 0      # both terms are exercised
+        assert torch.equal(got["stats"], want["stats"])
+        assert rel_l2(got["dz"].float(), want["dz"].float()) <= GRAD_REL_L2_BF16
+        assert float(want["dz"].float().norm()) > 0
+
+
+def test_static_scratch_variant_rejects_sizes_beyond_its_limits_on_the_host():
+    f = B.lib().mrl_policy_loss_fwd_bwd_static
+    fake = C.c_void_p(0x1000)        # never dereferenced: the size check comes first
+    lp = make_lp()
+    too_many_rows = f(fake, B.BF16, B.STATIC_MAX_ROWS + 1, 1024, 1024, fake, None, fake, 4, fake, None, None, None,
+                      C.byref(lp), None, 1024, None, fake, None, None, None)
+    assert too_many_rows == B.ERR_STATIC_SCRATCH_TOO_SMALL
+    too_many_seqs = f(fake, B.BF16, 16, 1024, 1024, fake, None, fake, B.STATIC_MAX_SEQS + 1, fake, None, None, None,
+                      C.byref(lp), None, 1024, None, fake, None, None, None)
+    assert too_many_seqs == B.ERR_STATIC_SCRATCH_TOO_SMALL
+    assert B.status_string(B.ERR_STATIC_SCRATCH_TOO_SMALL) == "MRL_ERR_STATIC_SCRATCH_TOO_SMALL"
