@@ -31,6 +31,27 @@ struct MrlCarver {
   }
 };
 
+// Per-row scratch of the loss passes (carved from the caller's workspace) and the host steps around the row kernels.
+struct MrlLossWs {
+  float *rowA, *rowcu, *rowcn;        // A_t, c_t u_t, cn_t
+  float *row_m2, *row_s, *row_zt;     // base-2 running max, sum of 2^(x - max), target logit
+  double *pg_term, *nll_term;
+  uint8_t* rowstat;                   // MRL_ROW_* bits
+  int32_t* seq_cnt;
+  unsigned long long* totals;
+  size_t bytes;
+};
+#define MRL_ROW_VALID 1
+#define MRL_ROW_CLIPPED 2
+#define MRL_ROW_READ 4
+size_t mrl_policy_loss_workspace_bytes(long long N, int S);
+int mrl_rows_prepare(void* workspace, long long N, int V, int S, const int32_t* ids, const uint8_t* mask,
+                     const int32_t* cu_seqlens, const float* adv_seq, const float* tok_weight,
+                     const float* nll_weight, const mrl_loss_params* lp, int32_t* status, cudaStream_t st,
+                     MrlLossWs* out);
+int mrl_rows_finish(const MrlLossWs& w, long long N, const float* logp_old, const mrl_loss_params* lp, float* logp,
+                    float* loss, int64_t* stats, cudaStream_t st);
+
 // Benchmark instrumentation (mrl_profile_dominant_kernel): event pairs recorded around dominant kernels.
 void mrl_profile_before(cudaStream_t st);
 void mrl_profile_after(cudaStream_t st);

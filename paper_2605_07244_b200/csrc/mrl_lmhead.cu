@@ -1,14 +1,715 @@
-// Hidden-in path (fused LM head): placeholder until the tcgen05 kernels land.
+// Hidden-in path (fused LM head): mrl_fused_lmhead_loss_fwd_bwd.
+//
+// Every product of the pass is a "TN" GEMM  C[M, N] = A[M, K] * B[N, K]^T  (both operands K-major, bf16, fp32
+// accumulation) on one persistent tcgen05 kernel, specialised by its epilogue:
+//   forward    z = hidden W^T, tile by tile; the epilogue folds each tile into per-row (max, sum 2^x) partials and
+//              picks the target logit; the [N, V] logits are never stored
+//   backward   per vocabulary chunk: recompute the z tile, write D = g (softmax - onehot) in bf16 as D[N, Vc] and
+//              D^T[Vc, N]; dHidden (+)= D (W^T)^T; dW[chunk] = D^T (hidden^T)^T
+// Kernel anatomy (one CTA per SM, 192 threads): warp 0 feeds a shared-memory ring with TMA tile loads
+// (128-byte swizzle, no multicast), one thread of warp 1 issues tcgen05.mma into one of two TMEM accumulators,
+// warps 2..5 drain the other accumulator with tcgen05.ld while the next tile's MMAs run.  Every mbarrier wait is
+// bounded; when one runs out the CTA raises MRL_DEV_TIMEOUT in the status word, lets its copies land and frees
+// its TMEM.
+#include <cuda.h>
+
 #include "mrl_common.cuh"
 
-size_t mrl_fused_lmhead_workspace_bytes(long long N, int V, int H, int S) {
-  (void)N; (void)V; (void)H; (void)S;
-  return 0;
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64;  // CTA tile; BK * 2 bytes = one 128-byte swizzle row
+constexpr int UMMA_K = 16;
+constexpr int kStages = 4;
+constexpr int kAccStages = 2;
+constexpr int kTmemCols = kAccStages * BN;  // 512: all of tensor memory
+constexpr int kGemmThreads = 192;
+constexpr uint32_t kABytes = BM * BK * 2, kBBytes = BN * BK * 2, kStageBytes = kABytes + kBBytes;
+constexpr size_t kGemmSmem = (size_t)kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr uint32_t kWaitLimit = 1u << 24;   // mbarrier polls before a wait gives up (of the order of a second)
+constexpr int kVChunk = 16384;              // vocabulary columns per backward chunk (multiple of BN)
+constexpr int kGroupM = 16;                 // row-tiles per raster group (operand reuse through L2)
+
+enum { EPI_LSE = 0, EPI_DZ = 1, EPI_STORE = 2 };
+enum { C_BF16 = 0, C_F32 = 1, C_F32_ADD = 2, C_BF16_FROM_ACC = 3 };
+
+struct GemmParams {
+  int M, N, K;
+  int m_tiles, n_tiles, k_blocks;
+  int32_t* status;
+  // EPI_LSE
+  float2* partial;        // [n_tiles][part_ld]: (running max, sum) of the tile's columns, base-2 domain
+  long long part_ld;
+  const int32_t* ids;     // [M]
+  float* zt;              // [M] target logit
+  int col0;               // vocabulary index of column 0 of this product
+  // EPI_DZ
+  const float* g;         // [M] gradient multiplier g_t
+  const float* lse2;      // [M] log2 sum_v 2^(z log2 e)
+  __nv_bfloat16* D;       // [M, ldD]
+  long long ldD;
+  __nv_bfloat16* DT;      // [N, ldDT]
+  long long ldDT;
+  // EPI_STORE
+  void* C;                // bf16 or fp32 [M, ldc]
+  float* Cacc;            // fp32 [M, ldacc] running sum (C_BF16_FROM_ACC reads it, C_F32 / C_F32_ADD write C)
+  long long ldc, ldacc;
+  int c_mode;
+};
+
+// ------------------------------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  False when the limit ran out here (the abort flag is raised) or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t i = 0; i < kWaitLimit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 1023u) == 1023u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]^T, one 128 x 256 x 16 step
+__device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accum) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accum)
+      : "memory");
+}
+// 32 lanes x 32 consecutive fp32 columns of tensor memory: thread i gets lane (base + i), columns [col, col + 32)
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, float* v) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
-extern "C" int mrl_fused_lmhead_loss_fwd_bwd(const void*, const void*, int64_t, int32_t, int32_t, const int32_t*,
-                                             const uint8_t*, const int32_t*, int32_t, const float*, const float*,
-                                             const float*, const float*, const mrl_loss_params*, void*, void*,
-                                             float*, float*, int64_t*, int32_t*, void*, size_t, void*) {
-  return MRL_ERR_UNSUPPORTED_SHAPE;
+// Shared-memory matrix descriptor of a K-major tile stored as 128-byte rows with the 128-byte swizzle (what the
+// TMA tile load writes): 8-row groups 1024 bytes apart, descriptor version 1 (sm_100), layout type SWIZZLE_128B.
+__device__ __forceinline__ uint64_t smem_desc_k128(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3ffffu) >> 4);   // start address, 16-byte units
+  d |= (uint64_t)1 << 16;                    // leading byte offset (unused by swizzled K-major layouts)
+  d |= (uint64_t)(1024 >> 4) << 32;          // stride byte offset between 8-row groups
+  d |= (uint64_t)1 << 46;                    // descriptor version
+  d |= (uint64_t)2 << 61;                    // SWIZZLE_128B
+  return d;
+}
+// kind::f16 instruction descriptor: fp32 accumulator, bf16 x bf16, both K-major, N = 256, M = 128
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+// tile t -> (row-tile, column-tile): row-tiles run fastest inside a group of kGroupM, so that the CTAs of one wave
+// share a handful of A and B tiles
+__device__ __forceinline__ void tile_coords(int t, int m_tiles, int n_tiles, int& m, int& n) {
+  const int per_group = kGroupM * n_tiles;
+  const int grp = t / per_group, r = t - grp * per_group;
+  const int m0 = grp * kGroupM;
+  const int gm = min(kGroupM, m_tiles - m0);
+  n = r / gm;
+  m = m0 + (r - n * gm);
+}
+
+// ------------------------------------------------------------------------------------------ epilogues
+// one thread = one row of the tile; v[] = 32 consecutive accumulator columns starting at tile column c
+
+struct LseRow {
+  float m, s, zt;
+  bool has;
+};
+
+__device__ __forceinline__ void epi_lse_batch(const float* v, int c, int ncols_valid, int rel_id, LseRow& st) {
+  float bm = -INFINITY;
+#pragma unroll
+  for (int j = 0; j < 32; ++j)
+    if (c + j < ncols_valid) bm = fmaxf(bm, v[j]);
+  if (bm == -INFINITY) return;  // no valid column in this batch
+  const float m_new = fmaxf(st.m, bm * MRL_LOG2E);
+  st.s *= mrl::ex2_approx(st.m - m_new);  // first batch: 0 * 2^-inf = 0
+  st.m = m_new;
+  float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+  for (int j = 0; j < 32; j += 2) {
+    if (c + j < ncols_valid) s0 += mrl::ex2_approx(fmaf(v[j], MRL_LOG2E, -m_new));
+    if (c + j + 1 < ncols_valid) s1 += mrl::ex2_approx(fmaf(v[j + 1], MRL_LOG2E, -m_new));
+  }
+  st.s += s0 + s1;
+  if (rel_id >= c && rel_id < c + 32) {
+#pragma unroll
+    for (int j = 0; j < 32; ++j)
+      if (rel_id == c + j) st.zt = v[j];
+    st.has = true;
+  }
+}
+
+__device__ __forceinline__ void store_bf16x32(__nv_bfloat16* dst, const float* d, int nvalid) {
+  if (nvalid >= 32 && (reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      uint4 u;
+      u.x = mrl::pack_bf16x2(d[q * 8 + 0], d[q * 8 + 1]);
+      u.y = mrl::pack_bf16x2(d[q * 8 + 2], d[q * 8 + 3]);
+      u.z = mrl::pack_bf16x2(d[q * 8 + 4], d[q * 8 + 5]);
+      u.w = mrl::pack_bf16x2(d[q * 8 + 6], d[q * 8 + 7]);
+      reinterpret_cast<uint4*>(dst)[q] = u;
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < 32; ++j)
+      if (j < nvalid) dst[j] = __float2bfloat16_rn(d[j]);
+  }
+}
+
+// ------------------------------------------------------------------------------------------ the GEMM kernel
+template <int EPI>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
+                   const GemmParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_addr(smem_raw);
+  const uint32_t tiles = (raw + 1023u) & ~1023u;  // swizzled tiles need 1024-byte alignment
+  unsigned char* tiles_ptr = smem_raw + (tiles - raw);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(tiles_ptr + (size_t)kStages * kStageBytes);
+  // bars[0..kStages): full, [kStages..2kStages): empty, then tmem_full[2], tmem_empty[2]
+  const uint32_t bar0 = smem_addr(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
+  auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kStages + a); };
+  auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kStages + kAccStages + a); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 2 * kAccStages);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int total_tiles = p.m_tiles * p.n_tiles;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < kAccStages; ++a) {
+      mbar_init(tfull_bar(a), 1);
+      mbar_init(tempty_bar(a), 4);  // one arrival per epilogue warp
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(tmem_slot)),
+                 "r"((uint32_t)kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------- TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+        int m, n;
+        tile_coords(t, p.m_tiles, p.n_tiles, m, n);
+        for (int kb = 0; kb < p.k_blocks; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t a_dst = tiles + (uint32_t)stage * kStageBytes;
+          mbar_expect_tx(full_bar(stage), kStageBytes);
+          tma_load_2d(a_dst, &tmapA, kb * BK, m * BM, full_bar(stage));
+          tma_load_2d(a_dst + kABytes, &tmapB, kb * BK, n * BN, full_bar(stage));
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer
+    if (lane == 0) {
+      int stage = 0, acc = 0;
+      uint32_t phase = 0, acc_phase = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)acc * BN;
+        for (int kb = 0; kb < p.k_blocks; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_src = tiles + (uint32_t)stage * kStageBytes;
+          const uint64_t adesc = smem_desc_k128(a_src), bdesc = smem_desc_k128(a_src + kABytes);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k)  // 32 bytes along K inside the swizzle row: +2 in 16-byte units
+            tc_mma(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), kIdesc, (kb | k) != 0);
+          tc_commit(empty_bar(stage));  // the stage is free once these MMAs have read it
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        tc_commit(tfull_bar(acc));
+        if (++acc == kAccStages) { acc = 0; acc_phase ^= 1u; }
+      }
+    }
+  } else {
+    // ---------------- epilogue: warps 2..5 own TMEM lanes 32 * (warp % 4) .. + 31
+    const int quad = warp & 3;
+    const int row_in_tile = quad * 32 + lane;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+      int m, n;
+      tile_coords(t, p.m_tiles, p.n_tiles, m, n);
+      const int row = m * BM + row_in_tile;
+      const bool row_ok = row < p.M;
+      const int ncols_valid = min(BN, p.N - n * BN);
+      // per-row inputs before the accumulator is ready
+      LseRow st = {-INFINITY, 0.f, 0.f, false};
+      int rel_id = -1;
+      float g = 0.f, neg_k = 0.f, l2 = 0.f, sgn = 1.f;
+      if (EPI == EPI_LSE) {
+        if (row_ok) rel_id = p.ids[row] - (p.col0 + n * BN);
+      } else if (EPI == EPI_DZ) {
+        if (row_ok) {
+          g = p.g[row];
+          l2 = p.lse2[row];
+          rel_id = p.ids[row] - (p.col0 + n * BN);
+        }
+        neg_k = -(l2 - log2f(fabsf(g)));  // 2^(z log2e - k) = |g| softmax(z); unused when g = 0
+        sgn = g < 0.f ? -1.f : 1.f;
+      }
+      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)acc * BN;
+#pragma unroll 1
+      for (int c = 0; c < BN; c += 32) {
+        if (c >= ncols_valid) break;  // uniform across the CTA
+        float v[32];
+        tc_ld32(t_row + (uint32_t)c, v);
+        if (EPI == EPI_LSE) {
+          epi_lse_batch(v, c, ncols_valid, rel_id, st);
+        } else if (EPI == EPI_DZ) {
+          float d[32];
+          if (g == 0.f) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) d[j] = 0.f;
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) d[j] = sgn * mrl::ex2_approx(fmaf(v[j], MRL_LOG2E, neg_k));
+            if (rel_id >= c && rel_id < c + 32) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (rel_id == c + j) d[j] = g * (mrl::ex2_approx(fmaf(v[j], MRL_LOG2E, -l2)) - 1.0f);
+            }
+          }
+          if (row_ok) {
+            const int nvalid = ncols_valid - c;
+            store_bf16x32(p.D + (long long)row * p.ldD + (long long)n * BN + c, d, nvalid);
+#pragma unroll
+            for (int j = 0; j < 32; ++j)  // a warp writes 32 consecutive rows of one column: 64 contiguous bytes
+              if (j < nvalid) p.DT[(long long)(n * BN + c + j) * p.ldDT + row] = __float2bfloat16_rn(d[j]);
+          }
+        } else {
+          if (row_ok) {
+            const int nvalid = ncols_valid - c;
+            const long long col = (long long)n * BN + c;
+            if (p.c_mode == C_BF16) {
+              store_bf16x32(static_cast<__nv_bfloat16*>(p.C) + (long long)row * p.ldc + col, v, nvalid);
+            } else if (p.c_mode == C_BF16_FROM_ACC) {
+              const float* a = p.Cacc + (long long)row * p.ldacc + col;
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (j < nvalid) v[j] += a[j];
+              store_bf16x32(static_cast<__nv_bfloat16*>(p.C) + (long long)row * p.ldc + col, v, nvalid);
+            } else {
+              float* o = static_cast<float*>(p.C) + (long long)row * p.ldc + col;
+              const bool add = p.c_mode == C_F32_ADD;
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (j < nvalid) o[j] = add ? o[j] + v[j] : v[j];
+            }
+          }
+        }
+      }
+      // the accumulator has been read: hand it back to the MMA warp
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(acc));
+      if (EPI == EPI_LSE && row_ok) {
+        p.partial[(long long)n * p.part_ld + row] = make_float2(st.m, st.s);
+        if (st.has) p.zt[row] = st.zt;
+      }
+      if (++acc == kAccStages) { acc = 0; acc_phase ^= 1u; }
+    }
+  }
+
+  // ---------------- teardown
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    if (threadIdx.x == 0 && p.status != nullptr) atomicOr(p.status, MRL_DEV_TIMEOUT);
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);  // let copies and MMAs still in flight land before the CTA goes
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols)
+                 : "memory");
+  }
+}
+
+// ------------------------------------------------------------------------------------------ small kernels
+// out[c, r] = in[r, c]; in [R, ld_in], out [C, ld_out]
+__global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16* __restrict__ in, long long R,
+                                                              long long C, long long ld_in,
+                                                              __nv_bfloat16* __restrict__ out, long long ld_out) {
+  __shared__ __nv_bfloat16 tile[64][66];
+  const long long r0 = (long long)blockIdx.y * 64, c0 = (long long)blockIdx.x * 64;
+  const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;
+  for (int i = ty; i < 64; i += 4) {
+    const long long r = r0 + i, c = c0 + tx;
+    tile[i][tx] = (r < R && c < C) ? in[r * ld_in + c] : __float2bfloat16(0.f);
+  }
+  __syncthreads();
+  for (int i = ty; i < 64; i += 4) {
+    const long long c = c0 + i, r = r0 + tx;
+    if (c < C && r < R) out[c * ld_out + r] = tile[tx][i];
+  }
+}
+
+// Merges the per-tile partials of every row in tile order, then the row's ratio / clip / gradient multiplier.
+__global__ void __launch_bounds__(256) lmhead_rows_kernel(long long N, int V, int n_tiles, const float2* __restrict__ partial,
+                                                           long long part_ld, const float* __restrict__ zt,
+                                                           const int32_t* __restrict__ ids,
+                                                           const uint8_t* __restrict__ mask,
+                                                           const float* __restrict__ rowA,
+                                                           const float* __restrict__ rowcu,
+                                                           const float* __restrict__ rowcn,
+                                                           const float* __restrict__ logp_old, float eps_lo,
+                                                           float eps_hi, float* __restrict__ row_m2,
+                                                           float* __restrict__ row_s, float* __restrict__ row_zt,
+                                                           uint8_t* __restrict__ rowstat, float* __restrict__ g_out,
+                                                           float* __restrict__ lse2_out) {
+  const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= N) return;
+  const int id = ids[t];
+  const bool valid = (mask == nullptr || mask[t] != 0) && id >= 0 && id < V;
+  mrl::Lse2 acc = mrl::lse2_empty();
+  if (valid)
+    for (int n = 0; n < n_tiles; ++n) {
+      const float2 q = partial[(long long)n * part_ld + t];
+      acc = mrl::lse2_merge(acc, mrl::Lse2{q.x, q.y});
+    }
+  float g = 0.f, l2 = 0.f;
+  uint8_t st = 0;
+  if (valid) {
+    l2 = acc.m + log2f(acc.s);
+    const float logp = zt[t] - l2 * MRL_LN2;
+    mrl::RowIn in;
+    in.A = rowA[t];
+    in.cu = rowcu[t];
+    in.cn = rowcn[t];
+    in.has_old = logp_old != nullptr;
+    in.logp_old = in.has_old ? logp_old[t] : 0.f;
+    const mrl::RowOut ro = mrl::mrl_row_loss(logp, in, eps_lo, eps_hi);
+    g = ro.g;
+    st = MRL_ROW_VALID | MRL_ROW_READ;
+    if (ro.clipped && in.A != 0.f) st |= MRL_ROW_CLIPPED;
+  }
+  row_m2[t] = acc.m;
+  row_s[t] = acc.s;
+  row_zt[t] = valid ? zt[t] : 0.f;
+  rowstat[t] = st;
+  g_out[t] = g;
+  lse2_out[t] = l2;
+}
+
+// ------------------------------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn == nullptr) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// Tensor map of a row-major bf16 matrix [rows, cols] (ld elements between rows) read in [box_rows x 64] tiles.
+int make_tmap(CUtensorMap* map, const void* base, long long rows, long long cols, long long ld, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return MRL_ERR_CUDA;
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? MRL_OK : MRL_ERR_CUDA;
+}
+
+int sm_count() {
+  static int n[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  if (n[dev] == 0) {
+    int v = 0;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) v = 148;
+    n[dev] = v;
+  }
+  return n[dev];
+}
+
+template <int EPI>
+int launch_gemm(const void* A, long long lda, const void* B, long long ldb, GemmParams p, cudaStream_t st) {
+  if (p.M <= 0 || p.N <= 0 || p.K <= 0) return MRL_OK;
+  CUtensorMap ta, tb;
+  int rc = make_tmap(&ta, A, p.M, p.K, lda, BM);
+  if (rc != MRL_OK) return rc;
+  rc = make_tmap(&tb, B, p.N, p.K, ldb, BN);
+  if (rc != MRL_OK) return rc;
+  p.m_tiles = (p.M + BM - 1) / BM;
+  p.n_tiles = (p.N + BN - 1) / BN;
+  p.k_blocks = (p.K + BK - 1) / BK;
+  const long long tiles = (long long)p.m_tiles * p.n_tiles;
+  if (tiles > 0x7fffffffll) return MRL_ERR_UNSUPPORTED_SHAPE;
+  const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
+  MRL_CUDA_OK(cudaFuncSetAttribute(lmhead_gemm_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)kGemmSmem));
+  mrl_profile_before(st);
+  lmhead_gemm_kernel<EPI><<<grid, kGemmThreads, kGemmSmem, st>>>(ta, tb, p);
+  mrl_profile_after(st);
+  MRL_CUDA_OK(cudaGetLastError());
+  return MRL_OK;
+}
+
+int launch_transpose(const __nv_bfloat16* in, long long R, long long C, long long ld_in, __nv_bfloat16* out,
+                     long long ld_out, cudaStream_t st) {
+  if (R == 0 || C == 0) return MRL_OK;
+  dim3 grid((unsigned)((C + 63) / 64), (unsigned)((R + 63) / 64));
+  if (grid.y > 65535u) return MRL_ERR_UNSUPPORTED_SHAPE;
+  transpose_bf16_kernel<<<grid, 256, 0, st>>>(in, R, C, ld_in, out, ld_out);
+  MRL_CUDA_OK(cudaGetLastError());
+  return MRL_OK;
+}
+
+long long pad_to(long long x, long long a) { return (x + a - 1) / a * a; }
+
+struct LmheadWs {
+  void* rows;            // per-row scratch of the loss (MrlLossWs)
+  float *g, *lse2, *zt;
+  float2* partial;
+  __nv_bfloat16 *WT, *HT, *D, *DT;
+  float* dH_acc;
+  long long part_ld, ldWT, ldHT, ldD, ldDT;
+  int n_tiles_fwd, vchunk, n_chunks;
+  size_t bytes;
+};
+
+LmheadWs carve_lmhead_ws(void* ws, long long N, int V, int H, int S) {
+  LmheadWs w;
+  MrlCarver c(ws);
+  w.rows = c.take<unsigned char>(mrl_policy_loss_workspace_bytes(N, S));
+  w.g = c.take<float>((size_t)N);
+  w.lse2 = c.take<float>((size_t)N);
+  w.zt = c.take<float>((size_t)N);
+  w.n_tiles_fwd = (V + BN - 1) / BN;
+  w.part_ld = pad_to(N, BM);
+  w.partial = c.take<float2>((size_t)w.n_tiles_fwd * (size_t)w.part_ld);
+  w.vchunk = V < kVChunk ? (int)pad_to(V, BN) : kVChunk;
+  w.n_chunks = (V + w.vchunk - 1) / w.vchunk;
+  w.ldWT = pad_to(V, 8);
+  w.ldHT = pad_to(N, 8);
+  w.ldD = w.vchunk;
+  w.ldDT = pad_to(N, 8);
+  w.WT = c.take<__nv_bfloat16>((size_t)H * (size_t)w.ldWT);
+  w.HT = c.take<__nv_bfloat16>((size_t)H * (size_t)w.ldHT);
+  w.D = c.take<__nv_bfloat16>((size_t)N * (size_t)w.ldD);
+  w.DT = c.take<__nv_bfloat16>((size_t)w.vchunk * (size_t)w.ldDT);
+  w.dH_acc = w.n_chunks > 1 ? c.take<float>((size_t)N * (size_t)H) : nullptr;
+  w.bytes = c.off;
+  return w;
+}
+
+}  // namespace
+
+size_t mrl_fused_lmhead_workspace_bytes(long long N, int V, int H, int S) {
+  if (N <= 0 || V <= 0 || H <= 0) return 0;
+  return carve_lmhead_ws(nullptr, N, V, H, S).bytes;
+}
+
+// C[M, N] = A[M, K] B[N, K]^T with a plain store (bf16 or fp32, optionally added to): the building block of the
+// two backward products, also reachable on its own for checks of the tensor-core mainloop.
+int mrl_lmhead_gemm_tn(const void* A, long long lda, const void* B, long long ldb, int M, int N, int K, void* C,
+                       long long ldc, int c_mode, float* Cacc, long long ldacc, int32_t* status, cudaStream_t st) {
+  GemmParams p = {};
+  p.M = M;
+  p.N = N;
+  p.K = K;
+  p.C = C;
+  p.ldc = ldc;
+  p.c_mode = c_mode;
+  p.Cacc = Cacc;
+  p.ldacc = ldacc;
+  p.status = status;
+  return launch_gemm<EPI_STORE>(A, lda, B, ldb, p, st);
+}
+
+extern "C" int mrl_fused_lmhead_loss_fwd_bwd(const void* hidden, const void* W, int64_t N, int32_t H, int32_t V,
+                                             const int32_t* ids, const uint8_t* mask, const int32_t* cu_seqlens,
+                                             int32_t S, const float* adv_seq, const float* logp_old,
+                                             const float* tok_weight, const float* nll_weight,
+                                             const mrl_loss_params* lp, void* dHidden, void* dW, float* logp,
+                                             float* loss, int64_t* stats, int32_t* status, void* workspace,
+                                             size_t workspace_bytes, void* stream) {
+  if (lp == nullptr || loss == nullptr || N < 0 || S < 0 || V < 1 || H < 1) return MRL_ERR_INVALID_ARG;
+  if (H % 64 != 0) return MRL_ERR_UNSUPPORTED_SHAPE;
+  if (N > 0x7fffff00ll) return MRL_ERR_UNSUPPORTED_SHAPE;
+  if (lp->agg_mode != MRL_AGG_TOKEN_MEAN && lp->agg_mode != MRL_AGG_SEQ_MEAN_TOKEN_MEAN) return MRL_ERR_INVALID_ARG;
+  if (!(lp->eps_lo >= 0.f) || !(lp->eps_hi >= 0.f)) return MRL_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const bool accum_loss = lp->flags & MRL_FLAG_ACCUMULATE_LOSS;
+  const bool accum_dw = lp->flags & MRL_FLAG_ACCUMULATE_DW;
+  if (N == 0 || S == 0) {
+    if (N != 0) return MRL_ERR_INVALID_ARG;
+    if (!accum_loss) {
+      MRL_CUDA_OK(cudaMemsetAsync(loss, 0, 2 * sizeof(float), st));
+      if (stats != nullptr) MRL_CUDA_OK(cudaMemsetAsync(stats, 0, 4 * sizeof(int64_t), st));
+    }
+    if (dW != nullptr && !accum_dw) MRL_CUDA_OK(cudaMemsetAsync(dW, 0, (size_t)V * H * 2, st));
+    return MRL_OK;
+  }
+  if (hidden == nullptr || W == nullptr || ids == nullptr || cu_seqlens == nullptr || adv_seq == nullptr)
+    return MRL_ERR_INVALID_ARG;
+  if ((dHidden == nullptr) != (dW == nullptr)) return MRL_ERR_INVALID_ARG;  // both gradients or forward only
+  if ((reinterpret_cast<uintptr_t>(hidden) & 15) || (reinterpret_cast<uintptr_t>(W) & 15) ||
+      (reinterpret_cast<uintptr_t>(dHidden) & 15) || (reinterpret_cast<uintptr_t>(dW) & 15))
+    return MRL_ERR_INVALID_ARG;
+  const size_t need = mrl_fused_lmhead_workspace_bytes(N, V, H, S);
+  if (workspace == nullptr || workspace_bytes < need) return MRL_ERR_WORKSPACE_TOO_SMALL;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255) != 0) return MRL_ERR_INVALID_ARG;
+  const LmheadWs w = carve_lmhead_ws(workspace, N, V, H, S);
+  const __nv_bfloat16* hid = static_cast<const __nv_bfloat16*>(hidden);
+  const __nv_bfloat16* Wm = static_cast<const __nv_bfloat16*>(W);
+
+  MrlLossWs rw;
+  int rc = mrl_rows_prepare(w.rows, N, V, S, ids, mask, cu_seqlens, adv_seq, tok_weight, nll_weight, lp, status, st,
+                            &rw);
+  if (rc != MRL_OK) return rc;
+  MRL_CUDA_OK(cudaMemsetAsync(w.zt, 0, (size_t)N * sizeof(float), st));
+
+  // ---- forward: per-tile log-sum-exp partials and the target logit, logits never stored
+  {
+    GemmParams p = {};
+    p.M = (int)N;
+    p.N = V;
+    p.K = H;
+    p.status = status;
+    p.partial = w.partial;
+    p.part_ld = w.part_ld;
+    p.ids = ids;
+    p.zt = w.zt;
+    p.col0 = 0;
+    rc = launch_gemm<EPI_LSE>(hid, H, Wm, H, p, st);
+    if (rc != MRL_OK) return rc;
+  }
+  lmhead_rows_kernel<<<(unsigned)((N + 255) / 256), 256, 0, st>>>(N, V, w.n_tiles_fwd, w.partial, w.part_ld, w.zt, ids,
+                                                                  mask, rw.rowA, rw.rowcu, rw.rowcn, logp_old,
+                                                                  lp->eps_lo, lp->eps_hi, rw.row_m2, rw.row_s,
+                                                                  rw.row_zt, rw.rowstat, w.g, w.lse2);
+  MRL_CUDA_OK(cudaGetLastError());
+  rc = mrl_rows_finish(rw, N, logp_old, lp, logp, loss, stats, st);
+  if (rc != MRL_OK) return rc;
+  if (dHidden == nullptr) return MRL_OK;
+
+  // ---- backward
+  rc = launch_transpose(Wm, V, H, H, w.WT, w.ldWT, st);
+  if (rc != MRL_OK) return rc;
+  rc = launch_transpose(hid, N, H, H, w.HT, w.ldHT, st);
+  if (rc != MRL_OK) return rc;
+  for (int ch = 0; ch < w.n_chunks; ++ch) {
+    const int v0 = ch * w.vchunk;
+    const int vc = V - v0 < w.vchunk ? V - v0 : w.vchunk;
+    {  // D = g (softmax - onehot) of the chunk's columns, both orientations
+      GemmParams p = {};
+      p.M = (int)N;
+      p.N = vc;
+      p.K = H;
+      p.status = status;
+      p.ids = ids;
+      p.col0 = v0;
+      p.g = w.g;
+      p.lse2 = w.lse2;
+      p.D = w.D;
+      p.ldD = w.ldD;
+      p.DT = w.DT;
+      p.ldDT = w.ldDT;
+      rc = launch_gemm<EPI_DZ>(hid, H, Wm + (size_t)v0 * H, H, p, st);
+      if (rc != MRL_OK) return rc;
+    }
+    {  // dHidden (+)= D[N, vc] * (W^T[H, v0 : v0 + vc])^T
+      int mode = C_BF16;
+      if (w.n_chunks > 1) mode = ch == 0 ? C_F32 : (ch == w.n_chunks - 1 ? C_BF16_FROM_ACC : C_F32_ADD);
+      void* C = (mode == C_BF16 || mode == C_BF16_FROM_ACC) ? dHidden : static_cast<void*>(w.dH_acc);
+      rc = mrl_lmhead_gemm_tn(w.D, w.ldD, w.WT + v0, w.ldWT, (int)N, H, vc, C, H, mode, w.dH_acc, H, status, st);
+      if (rc != MRL_OK) return rc;
+    }
+    {  // dW[v0 : v0 + vc, :] = D^T[vc, N] * (hidden^T[H, N])^T
+      void* C = accum_dw ? static_cast<void*>(static_cast<float*>(dW) + (size_t)v0 * H)
+                         : static_cast<void*>(static_cast<__nv_bfloat16*>(dW) + (size_t)v0 * H);
+      rc = mrl_lmhead_gemm_tn(w.DT, w.ldDT, w.HT, w.ldHT, vc, H, (int)N, C, H, accum_dw ? C_F32_ADD : C_BF16, nullptr,
+                              0, status, st);
+      if (rc != MRL_OK) return rc;
+    }
+  }
+  return MRL_OK;
 }

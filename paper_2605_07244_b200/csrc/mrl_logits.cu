@@ -24,7 +24,7 @@ constexpr int kMaxPartBytes = 76000;  // slice size that still lets three CTAs s
 constexpr uint32_t kSpinLimit = 1u << 20;
 
 // rowstat bits
-constexpr uint8_t kStatValid = 1, kStatClipped = 2, kStatRead = 4;
+constexpr uint8_t kStatValid = MRL_ROW_VALID, kStatClipped = MRL_ROW_CLIPPED, kStatRead = MRL_ROW_READ;
 
 struct RowParams {
   const void* logits;
@@ -555,18 +555,9 @@ __global__ void __launch_bounds__(1024) finalize_kernel(const double* __restrict
   }
 }
 
-struct LossWorkspace {
-  float *rowA, *rowcu, *rowcn, *row_m2, *row_s, *row_zt;
-  double *pg_term, *nll_term;
-  uint8_t* rowstat;
-  int32_t* seq_cnt;
-  unsigned long long* totals;
-  size_t bytes;
-};
-
-LossWorkspace carve_loss_ws(void* ws, long long N, int S) {
+MrlLossWs carve_loss_ws(void* ws, long long N, int S) {
   MrlCarver c(ws);
-  LossWorkspace w;
+  MrlLossWs w;
   w.totals = c.take<unsigned long long>(4);
   w.rowA = c.take<float>((size_t)N);
   w.rowcu = c.take<float>((size_t)N);
@@ -637,6 +628,37 @@ bool dtype_ok(int dtype) { return dtype == MRL_BF16 || dtype == MRL_F32; }
 
 size_t mrl_policy_loss_workspace_bytes(long long N, int S) { return carve_loss_ws(nullptr, N, S).bytes; }
 
+// Per-sequence bookkeeping shared by the logits-in and the hidden-in pass: carves the per-row scratch, counts the
+// valid tokens of every sequence and fills A_t, c_t u_t and cn_t of every row.
+int mrl_rows_prepare(void* workspace, long long N, int V, int S, const int32_t* ids, const uint8_t* mask,
+                     const int32_t* cu_seqlens, const float* adv_seq, const float* tok_weight,
+                     const float* nll_weight, const mrl_loss_params* lp, int32_t* status, cudaStream_t st,
+                     MrlLossWs* out) {
+  MrlLossWs w = carve_loss_ws(workspace, N, S);
+  // rows no sequence covers must contribute nothing: clear the coefficient arrays and the totals
+  MRL_CUDA_OK(cudaMemsetAsync(w.totals, 0, (size_t)((char*)w.row_m2 - (char*)w.totals), st));
+  seq_count_kernel<<<S, 128, 0, st>>>(cu_seqlens, S, N, V, ids, mask, w.seq_cnt, w.totals, status);
+  MRL_CUDA_OK(cudaGetLastError());
+  row_coef_kernel<<<S, 128, 0, st>>>(cu_seqlens, S, N, V, ids, mask, adv_seq, tok_weight, nll_weight, w.seq_cnt,
+                                     w.totals, *lp, w.rowA, w.rowcu, w.rowcn);
+  MRL_CUDA_OK(cudaGetLastError());
+  *out = w;
+  return MRL_OK;
+}
+
+// Float64 loss terms from the per-row reduction triples, then the fixed-order sums into loss / stats.
+int mrl_rows_finish(const MrlLossWs& w, long long N, const float* logp_old, const mrl_loss_params* lp, float* logp,
+                    float* loss, int64_t* stats, cudaStream_t st) {
+  row_terms_kernel<<<(unsigned)((N + 255) / 256), 256, 0, st>>>(N, w.row_m2, w.row_s, w.row_zt, w.rowstat, w.rowA,
+                                                                w.rowcu, w.rowcn, logp_old, lp->eps_lo, lp->eps_hi,
+                                                                w.pg_term, w.nll_term, logp);
+  MRL_CUDA_OK(cudaGetLastError());
+  finalize_kernel<<<1, 1024, 0, st>>>(w.pg_term, w.nll_term, w.rowstat, N, w.totals, lp->flags, loss,
+                                      reinterpret_cast<long long*>(stats));
+  MRL_CUDA_OK(cudaGetLastError());
+  return MRL_OK;
+}
+
 extern "C" int mrl_token_logprobs(const void* logits, int32_t dtype, int64_t N, int32_t V, int64_t ld,
                                   const int32_t* ids, const uint8_t* mask, float* logp, float* lse, int32_t* status,
                                   void* workspace, size_t workspace_bytes, void* stream) {
@@ -686,15 +708,10 @@ extern "C" int mrl_policy_loss_fwd_bwd(const void* logits, int32_t dtype, int64_
   const size_t need = mrl_policy_loss_workspace_bytes(N, S);
   if (workspace == nullptr || workspace_bytes < need) return MRL_ERR_WORKSPACE_TOO_SMALL;
   if ((reinterpret_cast<uintptr_t>(workspace) & 255) != 0) return MRL_ERR_INVALID_ARG;
-  LossWorkspace w = carve_loss_ws(workspace, N, S);
-
-  // rows no sequence covers must contribute nothing: clear the coefficient arrays and the totals
-  MRL_CUDA_OK(cudaMemsetAsync(w.totals, 0, (size_t)((char*)w.row_m2 - (char*)w.totals), st));
-  seq_count_kernel<<<S, 128, 0, st>>>(cu_seqlens, S, N, V, ids, mask, w.seq_cnt, w.totals, status);
-  MRL_CUDA_OK(cudaGetLastError());
-  row_coef_kernel<<<S, 128, 0, st>>>(cu_seqlens, S, N, V, ids, mask, adv_seq, tok_weight, nll_weight, w.seq_cnt,
-                                     w.totals, *lp, w.rowA, w.rowcu, w.rowcn);
-  MRL_CUDA_OK(cudaGetLastError());
+  MrlLossWs w;
+  int rc = mrl_rows_prepare(workspace, N, V, S, ids, mask, cu_seqlens, adv_seq, tok_weight, nll_weight, lp, status, st,
+                            &w);
+  if (rc != MRL_OK) return rc;
 
   RowParams p = {};
   p.logits = logits;
@@ -718,16 +735,9 @@ extern "C" int mrl_policy_loss_fwd_bwd(const void* logits, int32_t dtype, int64_
   p.row_zt = w.row_zt;
   p.rowstat = w.rowstat;
   p.status = status;
-  const int rc = launch_rows(p, dtype, st);
+  rc = launch_rows(p, dtype, st);
   if (rc != MRL_OK) return rc;
-  row_terms_kernel<<<(unsigned)((N + 255) / 256), 256, 0, st>>>(N, w.row_m2, w.row_s, w.row_zt, w.rowstat, w.rowA,
-                                                                w.rowcu, w.rowcn, logp_old, lp->eps_lo, lp->eps_hi,
-                                                                w.pg_term, w.nll_term, logp);
-  MRL_CUDA_OK(cudaGetLastError());
-  finalize_kernel<<<1, 1024, 0, st>>>(w.pg_term, w.nll_term, w.rowstat, N, w.totals, lp->flags, loss,
-                                      reinterpret_cast<long long*>(stats));
-  MRL_CUDA_OK(cudaGetLastError());
-  return MRL_OK;
+  return mrl_rows_finish(w, N, logp_old, lp, logp, loss, stats, st);
 }
 
 // ------------------------------------------------------------------------------------------------

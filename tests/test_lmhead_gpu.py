@@ -1,0 +1,199 @@
+"""GPU parity of the hidden-in path (mrl_fused_lmhead_loss_fwd_bwd) against the CPU float64 oracle:
+log-probs, loss terms, statistics, dHidden and dW on the same seeded inputs, through the C ABI."""
+import pytest
+import torch
+
+from oracle import mrl_oracle as O
+from paper_2605_07244_b200 import binding as B
+from paper_2605_07244_b200 import build, synth
+
+from helpers import GRAD_REL_L2_BF16, LOGP_ATOL, LOSS_RTOL, TIE_MARGIN, dev, make_lp, oracle_lp, rel_l2
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+    B.lib()
+
+
+def run_gpu_lmhead(hidden, W, ids, mask, cu, adv, logp_old, tok_weight, nll_weight, lp, want_grads=True,
+                   dW_init=None):
+    """CPU tensors in, CPU results of the CUDA path out."""
+    h, w = dev(hidden), dev(W)
+    N, H = h.shape
+    V = w.shape[0]
+    S = cu.numel() - 1
+    ws = torch.empty(max(B.workspace_bytes(B.WS_FUSED_LMHEAD, N, V, H, B.BF16, S), 256), dtype=torch.uint8,
+                     device="cuda")
+    dH = dW = None
+    if want_grads:
+        dH = torch.full((N, H), float("nan"), dtype=torch.bfloat16, device="cuda")
+        if lp.flags & B.FLAG_ACCUMULATE_DW:
+            dW = dev(dW_init, torch.float32)
+        else:
+            dW = torch.full((V, H), float("nan"), dtype=torch.bfloat16, device="cuda")
+    logp = torch.full((N,), float("nan"), device="cuda")
+    loss = torch.full((2,), float("nan"), device="cuda")
+    stats = torch.full((4,), -1, dtype=torch.int64, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    B.mrl_fused_lmhead_loss_fwd_bwd(h, w, dev(ids, torch.int32), dev(mask, torch.uint8), dev(cu, torch.int32),
+                                    dev(adv, torch.float32), dev(logp_old, torch.float32),
+                                    dev(tok_weight, torch.float32), dev(nll_weight, torch.float32), lp, dH, dW, logp,
+                                    loss, stats, status, ws)
+    torch.cuda.synchronize()
+    return dict(logp=logp.cpu(), loss=loss.cpu(), stats=stats.cpu(), status=int(status.cpu()),
+                dH=None if dH is None else dH.cpu(), dW=None if dW is None else dW.cpu())
+
+
+def toy(N, H, V, S, seed, mask_p=None, h_std=1.0, w_std=None, noise=0.1):
+    g = torch.Generator().manual_seed(seed)
+    w_std = w_std if w_std is not None else 2.0 / H ** 0.5       # logits of a few units, like an LM head
+    hidden = (torch.randn(N, H, generator=g) * h_std).to(torch.bfloat16)
+    W = (torch.randn(V, H, generator=g) * w_std).to(torch.bfloat16)
+    ids = torch.randint(0, V, (N,), generator=g, dtype=torch.int32)
+    if N > 1:
+        ids[0], ids[-1] = 0, V - 1
+    cuts = sorted(torch.randperm(N - 1, generator=g)[:S - 1].add(1).tolist()) if S > 1 else []
+    cu = torch.tensor([0] + cuts + [N], dtype=torch.int32)
+    adv = torch.randn(S, generator=g)
+    mask = None if mask_p is None else (torch.rand(N, generator=g) < mask_p).to(torch.uint8)
+    z = hidden.double() @ W.double().T
+    logp, _, _ = O.token_logprobs(z, ids, mask)
+    logp_old = (logp + torch.randn(N, generator=g, dtype=torch.float64) * noise).float()
+    return hidden, W, ids, mask, cu, adv, logp_old, g
+
+
+def compare(got, ref, check_grads=True, dW_base=None):
+    assert got["status"] == 0
+    assert torch.isfinite(got["logp"]).all()
+    err = (got["logp"].double() - ref["logp"]).abs().max()
+    assert err <= LOGP_ATOL, f"logp abs err {err}"
+    # Group-centred advantages make the policy-gradient term a cancelling sum (|L| can be 1e-3 of the sum of
+    # |terms|), and here the logits themselves are float32-accumulated dot products (|d logp| ~ 1e-6), so the
+    # relative tolerance is taken against max(|L|, a tenth of the sum of |terms|).
+    for k, name, terms in ((0, "loss_pg", "pg_term"), (1, "loss_nll", "nll_term")):
+        L = ref[name]
+        scale = max(abs(L), 0.1 * float(ref[terms].abs().sum()))
+        assert abs(float(got["loss"][k]) - L) <= LOSS_RTOL * scale + 1e-12, f"{name}: {float(got['loss'][k])} vs {L}"
+    tie = ref["valid"] & (ref["margin"] < TIE_MARGIN)
+    assert int(got["stats"][0]) == ref["stats"][0]
+    assert abs(int(got["stats"][1]) - ref["stats"][1]) <= int(tie.sum())
+    if not check_grads:
+        return
+    assert not tie.any(), "a row sits on the clip boundary: pick another seed for a gradient comparison"
+    dH, dW = got["dH"].double(), got["dW"].double()
+    assert torch.isfinite(dH).all() and torch.isfinite(dW).all()
+    want_dW = ref["dW"] if dW_base is None else ref["dW"] + dW_base.double()
+    e_h, e_w = rel_l2(dH, ref["dHidden"]), rel_l2(dW, want_dW)
+    assert e_h <= GRAD_REL_L2_BF16, f"dHidden rel L2 {e_h}"
+    assert e_w <= GRAD_REL_L2_BF16, f"dW rel L2 {e_w}"
+    # rows without gradient are exactly zero
+    zero_rows = ref["g"] == 0
+    if zero_rows.any():
+        assert dH[zero_rows].abs().max() == 0
+    # no row of dHidden hides behind the global norm
+    live = ref["g"] != 0
+    if live.any():
+        num = (dH[live] - ref["dHidden"][live]).norm(dim=1)
+        den = ref["dHidden"][live].norm(dim=1)
+        assert (num / den).max() <= 4 * GRAD_REL_L2_BF16
+
+
+CASES = [
+    # N, H, V, S, mask_p                      what it exercises
+    (300, 128, 1000, 5, None),      # ragged row tile, ragged column tile, one chunk
+    (128, 64, 256, 1, None),        # exactly one tile
+    (1, 64, 37, 1, None),           # N = 1, V below one vector
+    (260, 192, 40000, 7, 0.8),      # three vocabulary chunks with a ragged last one, masked rows
+    (700, 256, 16384 + 8, 3, None),  # second chunk of 8 columns
+]
+
+
+@pytest.mark.parametrize("agg", [B.AGG_TOKEN_MEAN, B.AGG_SEQ_MEAN_TOKEN_MEAN])
+@pytest.mark.parametrize("N,H,V,S,mask_p", CASES)
+def test_fused_lmhead_matches_oracle(N, H, V, S, mask_p, agg):
+    hidden, W, ids, mask, cu, adv, logp_old, g = toy(N, H, V, S, seed=N + V + agg, mask_p=mask_p)
+    tokw = torch.exp(torch.randn(N, generator=g) * 0.5)
+    nllw = (torch.rand(N, generator=g) < 0.2).float()
+    lp = make_lp(agg=agg, nll_coeff=0.05)
+    got = run_gpu_lmhead(hidden, W, ids, mask, cu, adv, logp_old, tokw, nllw, lp)
+    ref = O.fused_lmhead_loss(hidden, W, ids, mask, cu, adv, logp_old, tokw, nllw, oracle_lp(lp))
+    compare(got, ref)
+
+
+def test_forward_only_and_dw_accumulation_in_float32():
+    N, H, V, S = 200, 128, 3000, 4
+    hidden, W, ids, mask, cu, adv, logp_old, g = toy(N, H, V, S, seed=9)
+    lp = make_lp()
+    ref = O.fused_lmhead_loss(hidden, W, ids, mask, cu, adv, logp_old, None, None, oracle_lp(lp))
+    fwd = run_gpu_lmhead(hidden, W, ids, mask, cu, adv, logp_old, None, None, lp, want_grads=False)
+    compare(fwd, ref, check_grads=False)
+    base = torch.randn(V, H, generator=g) * float(ref["dW"].abs().mean())
+    lp_acc = make_lp(flags=B.FLAG_ACCUMULATE_DW)
+    got = run_gpu_lmhead(hidden, W, ids, mask, cu, adv, logp_old, None, None, lp_acc, dW_init=base)
+    assert got["dW"].dtype == torch.float32
+    compare(got, ref, dW_base=base)
+
+
+def test_degenerate_batches():
+    N, H, V, S = 96, 64, 500, 3
+    hidden, W, ids, mask, cu, adv, logp_old, g = toy(N, H, V, S, seed=21)
+    lp = make_lp()
+    # every row masked: zero loss, zero gradients
+    zeros = torch.zeros(N, dtype=torch.uint8)
+    got = run_gpu_lmhead(hidden, W, ids, zeros, cu, adv, logp_old, None, None, lp)
+    assert got["status"] == 0 and float(got["loss"].abs().max()) == 0
+    assert float(got["dH"].float().abs().max()) == 0 and float(got["dW"].float().abs().max()) == 0
+    assert got["stats"][0] == 0
+    # a bad id is reported, masked, and changes nothing else
+    bad = ids.clone()
+    bad[5] = V + 3
+    got = run_gpu_lmhead(hidden, W, bad, None, cu, adv, logp_old, None, None, lp)
+    assert got["status"] & B.DEV_BAD_TOKEN_ID
+    ref = O.fused_lmhead_loss(hidden, W, bad, None, cu, adv, logp_old, None, None, oracle_lp(lp))
+    got["status"] = 0
+    compare(got, ref)
+    # ratio one (no behaviour trace): loss = - masked mean of A
+    got = run_gpu_lmhead(hidden, W, ids, None, cu, adv, None, None, None, lp)
+    lens = (cu[1:] - cu[:-1]).double()
+    want = -float((adv.double() * lens).sum() / lens.sum())
+    assert abs(float(got["loss"][0]) - want) <= LOSS_RTOL * abs(want)
+
+
+def test_dW_columns_sum_to_zero_and_matches_logits_in_path():
+    """dz rows sum to zero, so sum_v dW[v, :] = 0 up to rounding; and the log-probs agree with the logits-in
+    kernel fed the bf16-rounded logits only to that rounding (a cross-check of the two kernel families)."""
+    N, H, V, S = 512, 256, 4096, 8
+    hidden, W, ids, mask, cu, adv, logp_old, g = toy(N, H, V, S, seed=33)
+    lp = make_lp()
+    got = run_gpu_lmhead(hidden, W, ids, None, cu, adv, logp_old, None, None, lp)
+    col = got["dW"].double().sum(dim=0)
+    scale = got["dW"].double().abs().sum(dim=0)
+    assert (col.abs() <= 2e-2 * scale + 1e-12).all()
+
+
+def test_config5_reduced_twin():
+    """Config 5's recipe at N = 4,096, H = 1,024, V = 32,768 (two vocabulary chunks), checked in full."""
+    w = synth.scaled(synth.C5, P=16, G=16, own_len=(16, 16), V=32768, H=1024)
+    meta = synth.make_meta(w, seed=3)
+    batch = synth.make_batch(meta)
+    N = batch.N
+    assert N == 4096
+    hidden = batch.hidden_rows(0, N)
+    W = batch.lm_head()
+    adv, _ = O.group_advantages(meta.rewards)
+    adv_seq = adv[batch.seq_p.long(), batch.seq_m.long(), batch.seq_g.long()].float()
+    z = hidden.double() @ W.double().T
+    logp, _, _ = O.token_logprobs(z, batch.ids)
+    logp_old = (logp + batch.noise.double()).float()
+    lp = make_lp()
+    got = run_gpu_lmhead(hidden, W, batch.ids, None, batch.cu_seqlens, adv_seq, logp_old, None, None, lp)
+    ref = O.fused_lmhead_loss(hidden, W, batch.ids, None, batch.cu_seqlens, adv_seq, logp_old, None, None,
+                              oracle_lp(lp))
+    tie = ref["valid"] & (ref["margin"] < TIE_MARGIN)
+    if tie.any():        # rows on the clip boundary may go either way: compare everything but the gradients
+        compare(got, ref, check_grads=False)
+    else:
+        compare(got, ref)
