@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the policy-loss hot path on B200 (one process per GPU).
 
-    python bench.py --gpus N --steps K --warmup W [--impl reference] [--workload C2|C5]
+    python bench.py --gpus N --steps K --warmup W [--impl reference] [--workload C2|C2s|C5]
 
 A step is one pass of the whole hot path over one batch of synthetic input: group advantages and
 SGT gate (mrl_group_advantages), then log-probs, ratio, clipped surrogate, aggregation and dlogits
@@ -33,6 +33,8 @@ METRIC = "policy_loss_fwd_bwd_tokens_per_s"
 UNIT = "tokens/s"
 ORACLE_ROWS = 2048          # rows of the workload the CPU baseline is timed on
 REFERENCE_ROWS = 1024       # rows per step of the --impl reference arm
+LMHEAD_ORACLE_ROWS = 128    # rows of config 5 the CPU baseline is timed on (full V and H)
+LMHEAD_SUB_STEPS = 5        # timed steps of the config-5 leg inside the default (config 2) run
 
 
 # ------------------------------------------------------------------------------------------ helpers
@@ -178,6 +180,7 @@ class LogitsInWorkload:
         self.logp_old = self.logp + b.noise.to(dev)
         torch.cuda.synchronize()
         self.kernels_per_step = 6    # adv_prompt, seq_count, row_coef, row (cluster), row_terms, finalize
+        self.dominant_per_step = 1
         self.bytes_per_token = 2 * self.V * self.z.element_size()   # read V + write V elements
 
     def step(self, z=None, dz=None):
@@ -221,6 +224,21 @@ class LogitsInWorkload:
         self.h_logp.copy_(self.logp, non_blocking=True)
         self.h_loss.copy_(self.loss, non_blocking=True)
 
+    def roofline(self, kernel_ms, peaks):
+        k_avg_ms = sum(kernel_ms) / len(kernel_ms)
+        alg_bytes = self.bytes_per_token * self.tokens()
+        achieved = alg_bytes / (k_avg_ms * 1e-3) / 1e9
+        per_token = profile_traffic("row_cluster_kernel_dram_bytes_per_token_V151936")
+        return {"bound": "hbm", "kernel": "row_cluster_kernel", "achieved": achieved, "peak": peaks["hbm_gbs"],
+                "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                "peak_source": peaks["source"] + " (copy, burst)", "algorithmic_bytes_per_launch": alg_bytes,
+                "kernel_ms": k_avg_ms, "traffic": None if per_token is None else per_token * self.tokens()}
+
+    def time_oracle(self):
+        O, oargs, n = self.oracle_sample(ORACLE_ROWS)
+        dt = time_oracle(O, oargs)
+        return n, dt, f"first {n} rows of the same batch, full V, fwd+bwd, float64, {dt:.1f} s"
+
     # ---- CPU baseline: the oracle on the first ORACLE_ROWS rows of the same batch
     def oracle_sample(self, rows):
         from oracle import mrl_oracle as O
@@ -234,6 +252,128 @@ class LogitsInWorkload:
         adv_seq = adv[b.seq_p.long(), b.seq_m.long(), b.seq_g.long()][:s_end]
         args = (z, b.ids[:n], None, b.cu_seqlens[:s_end + 1], adv_seq, self.logp_old[:n].cpu())
         return O, args, n
+
+
+class LmheadWorkload:
+    """Config 5: N = 65,536 response tokens, H = 4,096, V = 151,936, bf16 hidden and LM-head weight; the logits
+    are never stored; outputs logp, loss, dHidden, dW."""
+
+    def __init__(self, w: synth.Workload, seed: int, device):
+        from paper_2605_07244_b200 import binding as B
+        self.B = B
+        self.w = w
+        self.meta = synth.make_meta(w, seed)
+        self.batch = synth.make_batch(self.meta)
+        b = self.batch
+        self.N, self.V, self.H, self.S = b.N, w.V, w.H, b.S
+        P, M, G = w.P, w.M, w.G
+        dev = device
+        self.hidden = torch.empty(self.N, self.H, dtype=w.dtype, device=dev)
+        for a in range(0, self.N, w.rows_per_block):
+            e = min(self.N, a + w.rows_per_block)
+            self.hidden[a:e] = b.hidden_rows(a, e, device=dev)
+        self.W = b.lm_head(device=dev)
+        self.dH = torch.empty_like(self.hidden)
+        self.dW = torch.empty_like(self.W)
+        self.ids = b.ids.to(dev)
+        self.cu = b.cu_seqlens.to(dev)
+        self.rewards = self.meta.rewards.to(dev)
+        self.seq_len = self.meta.seq_len.to(dev)
+        self.adv_own = torch.empty(P, M, G, device=dev)
+        self.adv_pool = torch.empty(P, M, G, device=dev)
+        self.rescue = torch.empty(P, dtype=torch.uint8, device=dev)
+        self.pick = torch.empty(P, dtype=torch.int32, device=dev)
+        self.nllw_seq = torch.empty(P, M, G, device=dev)
+        self.n_gated = torch.empty(1, dtype=torch.int32, device=dev)
+        self.logp = torch.empty(self.N, device=dev)
+        self.loss = torch.zeros(2, device=dev)
+        self.stats = torch.zeros(4, dtype=torch.int64, device=dev)
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.ws = torch.empty(B.workspace_bytes(B.WS_FUSED_LMHEAD, self.N, self.V, self.H, B.BF16, self.S),
+                              dtype=torch.uint8, device=dev)
+        self.ap = B.AdvParams(B.ADV_GROUP_ZNORM, 0, 1e-6, 0.8, 0.2, B.PICK_SHORTEST, 0)
+        self.lp = B.LossParams(0.2, 0.2, B.AGG_TOKEN_MEAN, 0, 0.0, 0.0, 0.0, 0)
+        # behaviour trace: logp_old = logp + N(0, 0.1); logp from a forward-only call (input preparation)
+        B.mrl_group_advantages(self.rewards, self.seq_len, 0, self.ap, self.adv_own, self.adv_pool, self.rescue,
+                               self.pick, self.nllw_seq, self.n_gated)
+        B.mrl_fused_lmhead_loss_fwd_bwd(self.hidden, self.W, self.ids, None, self.cu, self.adv_own, None, None, None,
+                                        self.lp, None, None, self.logp, self.loss, self.stats, self.status, self.ws)
+        self.logp_old = self.logp + b.noise.to(dev)
+        torch.cuda.synchronize()
+        chunks = -(-self.V // 16384)
+        self.dominant_per_step = 1 + 3 * chunks          # forward GEMM, then (dZ, dHidden, dW) per vocabulary chunk
+        # adv, seq_count, row_coef, forward GEMM, rows, row_terms, finalize, two transposes, 3 GEMMs per chunk
+        self.kernels_per_step = 9 + 3 * chunks
+        self.flops_executed = 8.0 * self.N * self.H * self.V      # forward, recompute, dHidden, dW
+        self.flops_algorithmic = 6.0 * self.N * self.H * self.V   # without the recompute
+
+    def step(self):
+        B = self.B
+        B.mrl_group_advantages(self.rewards, self.seq_len, 0, self.ap, self.adv_own, self.adv_pool, self.rescue,
+                               self.pick, self.nllw_seq, self.n_gated)
+        B.mrl_fused_lmhead_loss_fwd_bwd(self.hidden, self.W, self.ids, None, self.cu, self.adv_own, self.logp_old,
+                                        None, None, self.lp, self.dH, self.dW, self.logp, self.loss, self.stats,
+                                        self.status, self.ws)
+
+    def tokens(self):
+        return self.N
+
+    def describe(self):
+        return {"workload": f"{self.w.name}: fused LM-head, hidden-in: N={self.N} response tokens ({self.w.P} prompts x "
+                            f"G=16 x T=64), H={self.H} bf16 hidden N(0,1), W[V={self.V},H] bf16 N(0,0.02^2), logits never "
+                            "materialised, GRPO clipped surrogate, binary rewards, fwd+bwd -> dHidden, dW",
+                "rows": self.N, "sequences": self.S, "V": self.V, "H": self.H,
+                "l2": "operands (1.8 GB) and scratch exceed the 126 MB L2; no flush needed"}
+
+    def roofline(self, kernel_ms, peaks):
+        """All tensor-core launches of a step against the bf16 rate cuBLAS sustains inside a long step."""
+        per_step_ms = sum(kernel_ms) / (len(kernel_ms) / self.dominant_per_step)
+        achieved = self.flops_executed / (per_step_ms * 1e-3) / 1e12
+        peak = peaks["bf16_tflops_sustained"]
+        return {"bound": "tensor", "kernel": "lmhead_gemm_kernel (forward, dZ recompute, dHidden, dW launches)",
+                "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                "peak_source": peaks["source"] + " (cuBLAS bf16, sustained)",
+                "flops_per_step_executed": self.flops_executed, "flops_per_step_algorithmic": self.flops_algorithmic,
+                "achieved_algorithmic": self.flops_algorithmic / (per_step_ms * 1e-3) / 1e12,
+                "kernel_ms": per_step_ms, "launches_per_step": self.dominant_per_step, "traffic": None}
+
+    def e2e_setup(self):
+        self.h_hidden = self.hidden.cpu().pin_memory()
+        self.h_W = self.W.cpu().pin_memory()
+        self.h_dH = torch.empty(self.hidden.shape, dtype=self.hidden.dtype, pin_memory=True)
+        self.h_dW = torch.empty(self.W.shape, dtype=self.W.dtype, pin_memory=True)
+        self.h_small_in = [t.cpu().pin_memory() for t in (self.ids, self.cu, self.rewards, self.seq_len, self.logp_old)]
+        self.d_small_in = [self.ids, self.cu, self.rewards, self.seq_len, self.logp_old]
+        self.h_logp = torch.empty(self.N, pin_memory=True)
+        self.h_loss = torch.empty(2, pin_memory=True)
+        h2d = (self.h_hidden.numel() + self.h_W.numel()) * 2 + sum(t.numel() * t.element_size() for t in self.h_small_in)
+        d2h = (self.h_dH.numel() + self.h_dW.numel()) * 2 + self.N * 4 + 8
+        return h2d, d2h
+
+    def e2e_step(self):
+        for h, d in zip(self.h_small_in, self.d_small_in):
+            d.copy_(h, non_blocking=True)
+        self.hidden.copy_(self.h_hidden, non_blocking=True)
+        self.W.copy_(self.h_W, non_blocking=True)
+        self.step()
+        self.h_dH.copy_(self.dH, non_blocking=True)
+        self.h_dW.copy_(self.dW, non_blocking=True)
+        self.h_logp.copy_(self.logp, non_blocking=True)
+        self.h_loss.copy_(self.loss, non_blocking=True)
+
+    def time_oracle(self):
+        from oracle import mrl_oracle as O
+        b = self.batch
+        n_seq = max(1, LMHEAD_ORACLE_ROWS // int(b.cu_seqlens[1]))
+        n = int(b.cu_seqlens[n_seq])
+        adv, _ = O.group_advantages(self.meta.rewards)
+        adv_seq = adv[b.seq_p.long(), b.seq_m.long(), b.seq_g.long()][:n_seq]
+        args = (self.hidden[:n].cpu(), self.W.cpu(), b.ids[:n], None, b.cu_seqlens[:n_seq + 1], adv_seq,
+                self.logp_old[:n].cpu())
+        t0 = time.perf_counter()
+        O.fused_lmhead_loss(*args, None, None, O.LossParams())
+        dt = time.perf_counter() - t0
+        return n, dt, f"first {n} rows of the same batch, full V and H, fwd+bwd incl. dW, float64, {dt:.1f} s"
 
 
 def time_oracle(O, args, repeats=1):
@@ -307,6 +447,42 @@ def run_e2e(args, wl, world):
                     "included) and of dlogits, logp and loss"}
 
 
+def measure(wl, steps, warmup, world, local_rank, rank, peaks, with_e2e, with_cpu, args):
+    """Warm up, time `steps` steps with CUDA events (max over ranks), and build the result fields."""
+    B = wl.B
+    for _ in range(max(warmup, 3)):
+        wl.step()
+    torch.cuda.synchronize()
+    timer = B.DominantKernelTimer(steps * wl.dominant_per_step)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier(world)
+    torch.cuda.synchronize()
+    with ClockSampler(local_rank) as clocks, timer:
+        ev0.record()
+        for _ in range(steps):
+            wl.step()
+        ev1.record()
+        torch.cuda.synchronize()
+    barrier(world)
+    local_ms = ev0.elapsed_time(ev1)
+    kernel_ms = timer.elapsed_ms(steps * wl.dominant_per_step)
+    status = int(wl.status.cpu())
+    if status != 0:
+        raise SystemExit(f"device status word is {status} after the timed region")
+    total_ms, total_tokens = aggregate_over_ranks(local_ms, wl.tokens() * steps, world)
+    out = {"value": total_tokens / (total_ms * 1e-3), "ms_per_step": total_ms / steps, "steps": steps,
+           "config": dict(wl.describe(), parallelism=f"replicas x{world}"), "clocks": clocks.summary(),
+           "gpu_launches": wl.kernels_per_step * steps, "roofline": wl.roofline(kernel_ms, peaks)}
+    # end to end: pinned host buffers -> device -> kernels -> pinned host buffers
+    out["e2e"] = run_e2e(args, wl, world) if with_e2e else None
+    out["cpu_baseline"] = None
+    if with_cpu and rank == 0 and world == 1:
+        n, dt, sample = wl.time_oracle()
+        out["cpu_baseline"] = {"value": n / dt, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
+                               "sample": sample}
+    return out
+
+
 def run_ours(args, rank, world, local_rank):
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
@@ -316,67 +492,39 @@ def run_ours(args, rank, world, local_rank):
     from paper_2605_07244_b200 import build
     build.build()
     B.lib()
-    if args.workload not in ("C2", "C2s"):
-        raise SystemExit("bench.py times config 2 (logits-in); C2s is its small profiling case; "
-                         "other configs are parity-test cases")
-    wl = LogitsInWorkload(synth.CONFIGS[args.workload], args.seed + rank, device)
+    if args.workload not in ("C2", "C2s", "C5", "C5s"):
+        raise SystemExit("bench.py times config 2 (logits-in; C2s is its small profiling case) and config 5 "
+                         "(fused LM head); the other configs are parity-test cases")
     peaks = measured_peaks()
+    lmhead_main = args.workload in ("C5", "C5s")
+    cls = LmheadWorkload if lmhead_main else LogitsInWorkload
+    wl = cls(synth.CONFIGS[args.workload], args.seed + rank, device)
+    res = measure(wl, args.steps, args.warmup, world, local_rank, rank, peaks, not args.no_e2e,
+                  not args.no_cpu_baseline, args)
+    del wl
+    torch.cuda.empty_cache()
 
-    for _ in range(max(args.warmup, 3)):
-        wl.step()
-    torch.cuda.synchronize()
-
-    timer = B.DominantKernelTimer(args.steps)
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier(world)
-    torch.cuda.synchronize()
-    with ClockSampler(local_rank) as clocks, timer:
-        ev0.record()
-        for _ in range(args.steps):
-            wl.step()
-        ev1.record()
-        torch.cuda.synchronize()
-    barrier(world)
-    local_ms = ev0.elapsed_time(ev1)
-    kernel_ms = timer.elapsed_ms(args.steps)
-    status = int(wl.status.cpu())
-    if status != 0:
-        raise SystemExit(f"device status word is {status} after the timed region")
-    total_ms, total_tokens = aggregate_over_ranks(local_ms, wl.tokens() * args.steps, world)
-    value = total_tokens / (total_ms * 1e-3)
-
-    # dominant kernel against the HBM roofline
-    k_avg_ms = sum(kernel_ms) / len(kernel_ms)
-    alg_bytes = wl.bytes_per_token * wl.tokens()
-    achieved = alg_bytes / (k_avg_ms * 1e-3) / 1e9
-    per_token = profile_traffic("row_cluster_kernel_dram_bytes_per_token_V151936")
-    roofline = {"bound": "hbm", "kernel": "row_cluster_kernel", "achieved": achieved, "peak": peaks["hbm_gbs"],
-                "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"] + " (copy, burst)",
-                "algorithmic_bytes_per_launch": alg_bytes, "kernel_ms": k_avg_ms,
-                "traffic": None if per_token is None else per_token * wl.tokens()}
-
-    # end to end: pinned host buffers -> device -> kernels -> pinned host buffers
-    e2e = None
-    if not args.no_e2e:
-        e2e = run_e2e(args, wl, world)
-
-
-    cpu_baseline = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        O, oargs, n = wl.oracle_sample(ORACLE_ROWS)
-        dt = time_oracle(O, oargs)
-        cpu_baseline = {"value": n / dt, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
-                        "sample": f"first {n} rows of the same batch, full V, fwd+bwd, float64, {dt:.1f} s"}
+    # the tensor-core family beside the headline: a short config-5 leg in the default run
+    lmhead = None
+    if args.workload == "C2" and not args.no_lmhead:
+        wl5 = LmheadWorkload(synth.CONFIGS["C5"], args.seed + rank, device)
+        r5 = measure(wl5, min(args.steps, LMHEAD_SUB_STEPS), 3, world, local_rank, rank, peaks, False,
+                     not args.no_cpu_baseline, args)
+        lmhead = {"metric": METRIC, "unit": UNIT, **{k: r5[k] for k in ("value", "ms_per_step", "steps", "config",
+                                                                         "gpu_launches", "roofline", "cpu_baseline")}}
+        del wl5
 
     if rank == 0:
-        print(json.dumps({
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": dict(wl.describe(), parallelism=f"replicas x{world}"),
-            "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": wl.kernels_per_step * args.steps,
-            "roofline": roofline, "cpu_baseline": cpu_baseline,
-        }))
+        line = {
+            "metric": METRIC, "value": res["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": res["ms_per_step"], "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if lmhead_main else "f32", "data": "synthetic",
+            "config": res["config"], "clocks": res["clocks"], "e2e": res["e2e"], "gpu_launches": res["gpu_launches"],
+            "roofline": res["roofline"], "cpu_baseline": res["cpu_baseline"],
+        }
+        if lmhead is not None:
+            line["lmhead"] = lmhead
+        print(json.dumps(line))
 
 
 def main():
@@ -389,6 +537,7 @@ def main():
     ap.add_argument("--seed", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="profiling runs only: skip the host-buffer leg")
+    ap.add_argument("--no-lmhead", action="store_true", help="skip the short config-5 leg of the default run")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

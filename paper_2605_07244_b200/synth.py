@@ -50,7 +50,9 @@ C5 = Workload("C5-fused-lmhead", P=64, M=1, G=16, V=151936, dtype=torch.bfloat16
               reward_beta=False, H=4096)
 # config 2 with a quarter of the prompts: still far larger than L2, small enough for a profiler capture
 C2_SMALL = replace(C2, name="C2-qwen-vocab-2-prompts", P=2)
-CONFIGS = {"C1": C1, "C2": C2, "C3": C3, "C4": C4, "C5": C5, "C2s": C2_SMALL}
+# config 5 with an eighth of the rows and two vocabulary chunks: operands and scratch still exceed L2
+C5_SMALL = replace(C5, name="C5-fused-lmhead-8k-rows-32k-vocab", P=8, V=32768)
+CONFIGS = {"C1": C1, "C2": C2, "C3": C3, "C4": C4, "C5": C5, "C2s": C2_SMALL, "C5s": C5_SMALL}
 
 
 def scaled(w: Workload, **kw) -> Workload:
