@@ -2,17 +2,14 @@
 //
 // Fast kernel (bf16, 16-byte aligned rows): one thread-block cluster per logits row.  Each CTA of
 // the cluster pulls its slice of the row into shared memory with bulk asynchronous copies (four
-// chunks, one mbarrier each), reduces max / sum-of-exponentials as the chunks land, exchanges one
-// (max, sum, target-logit) triple per CTA through distributed shared memory, evaluates the ratio /
-// clip / loss scalars, and writes g * (softmax - onehot) straight from the resident slice.  The row
-// is read from HBM exactly once and written exactly once; nothing is shared between clusters.
+// chunks, one mbarrier each), reduces max / sum-of-exponentials as the chunks land while caching the
+// exponentials in place, exchanges one (max, sum, target-logit) triple per CTA through distributed
+// shared memory, evaluates the ratio / clip / loss scalars, and writes g * (softmax - onehot) from
+// the cached slice.  The row is read from HBM exactly once and written exactly once; nothing is
+// shared between clusters.
 // General kernel (any dtype, any V, any alignment): one CTA per row, three passes over global
 // memory; used for small or unaligned problems.
-#include <cooperative_groups.h>
-
 #include "mrl_common.cuh"
-
-namespace cg = cooperative_groups;
 
 namespace {
 
@@ -90,13 +87,6 @@ __device__ __forceinline__ void st_global_v4(void* p, uint4 v) {
   asm volatile("st.global.cs.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 
-__device__ __forceinline__ float max8_bf16(uint4 v) {
-  __nv_bfloat162 a = *reinterpret_cast<__nv_bfloat162*>(&v.x), b = *reinterpret_cast<__nv_bfloat162*>(&v.y);
-  __nv_bfloat162 c = *reinterpret_cast<__nv_bfloat162*>(&v.z), d = *reinterpret_cast<__nv_bfloat162*>(&v.w);
-  __nv_bfloat162 m = __hmax2(__hmax2(a, b), __hmax2(c, d));
-  return fmaxf(__low2float(m), __high2float(m));
-}
-
 // Everything the loss needs from one row besides the logits.
 struct RowCtx {
   int id;
@@ -148,12 +138,57 @@ __device__ __forceinline__ void write_row_scalars(const RowParams& p, long long 
 }
 
 // ------------------------------------------------------------------------------------------------
-// Fast kernel: bf16, one cluster per row, slice resident in shared memory.
-// Dynamic shared memory: [slice bytes | 4 mbarriers | 64 floats reduce scratch | 8 float4 exchange | 4 floats bcast]
+// Fast kernel: bf16, one thread-block cluster per row, each CTA's slice of the row resident in shared memory.
+//
+// A CTA pulls its slice in with four bulk asynchronous copies (an mbarrier each) and works on it as the copies
+// land.  Pass 1, in steps of 1,024 vectors: each thread takes the maximum of its own 32 logits of the step as
+// reference, turns them into 2^(x - ref), sums them in float32 and writes them back over the logits as bf16, so
+// that pass 2 needs no exponential; the references stay in registers.  The CTA's (max, sum, target logit) is
+// pushed to every other CTA of the cluster through distributed shared memory (a remote store and a remote
+// mbarrier arrive per peer); warp 0 alone waits for the peers, forms the row's scalars and hands them to the
+// block.  Pass 2: every cached value times g 2^(ref - lse) as two packed bf16 FMAs (scale = hi + lo, one
+// rounding of the result), streamed out with 128-bit stores.  Full steps run without per-vector bounds checks;
+// only the last step of a slice can be ragged.  Slices are at most 76,000 bytes, so three CTAs of different rows
+// share an SM and one CTA's copy latency, exchange and stores overlap the others' arithmetic.
+// A row is read from HBM once and written once; nothing is shared between clusters.
+// Dynamic shared memory: [slice | 4 copy barriers, 1 exchange barrier | exchange | per-warp scratch | row scalars]
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kThreads) row_cluster_kernel(const RowParams p) {
+constexpr int kStepVecs = kThreads * kUnroll;                                // vectors per step of a CTA
+constexpr int kMaxSteps = (kMaxPartBytes / 16 + kStepVecs - 1) / kStepVecs;  // 5
+constexpr int kWarps = kThreads / 32;
+constexpr size_t kTailBytes = 64 + kMaxCluster * 16 + 2 * kWarps * 4 + 32;
+
+__device__ __forceinline__ uint32_t mapa_u32(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// packed arithmetic on two bf16
+__device__ __forceinline__ uint32_t hmax2_u32(uint32_t a, uint32_t b) {
+  uint32_t r;
+  asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+  return r;
+}
+__device__ __forceinline__ uint32_t hfma2_u32(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t r;
+  asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(c));
+  return r;
+}
+
+__global__ void __launch_bounds__(kThreads, 3) row_cluster_kernel(const RowParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int C = p.cluster;
   const long long row = blockIdx.x / C;
   const int rank = blockIdx.x % C;  // equals the rank in the cluster for a 1-D cluster
@@ -163,14 +198,16 @@ __global__ void __launch_bounds__(kThreads) row_cluster_kernel(const RowParams p
   const size_t slice_bytes = (size_t)p.part_elems * 2;
 
   uint4* slice = reinterpret_cast<uint4*>(smem);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + slice_bytes);
-  float* scratch = reinterpret_cast<float*>(smem + slice_bytes + kChunks * 8);
-  float4* xchg = reinterpret_cast<float4*>(smem + slice_bytes + kChunks * 8 + 64 * 4);
-  float* bcast = reinterpret_cast<float*>(smem + slice_bytes + kChunks * 8 + 64 * 4 + kMaxCluster * 16);
+  unsigned char* tail = smem + slice_bytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(tail);                    // [kChunks] copies, then the exchange
+  float4* xchg = reinterpret_cast<float4*>(tail + 64);                   // [kMaxCluster]
+  float* red = reinterpret_cast<float*>(tail + 64 + kMaxCluster * 16);   // [2][kWarps]
+  float* fin = red + 2 * kWarps;                                         // lse2, g, target-column value, ok
+  float* tgt = fin + 4;                                                  // target logit, has-target
 
+  const bool want_grad = p.dlogits != nullptr;
   const __nv_bfloat16* grow = static_cast<const __nv_bfloat16*>(p.logits) + row * p.ld + part_off;
-  __nv_bfloat16* orow =
-      p.dlogits ? static_cast<__nv_bfloat16*>(p.dlogits) + row * p.ld_out + part_off : nullptr;
+  __nv_bfloat16* orow = want_grad ? static_cast<__nv_bfloat16*>(p.dlogits) + row * p.ld_out + part_off : nullptr;
 
   // Rows that may be dead are decided before anything is fetched; otherwise fetch first.
   const bool may_be_dead = p.mask != nullptr || (p.flags & MRL_FLAG_SKIP_ZERO_ROWS);
@@ -185,15 +222,15 @@ __global__ void __launch_bounds__(kThreads) row_cluster_kernel(const RowParams p
     }
   }
 
-  const int vpc = (nvec + kChunks - 1) / kChunks;  // vectors per chunk
+  const int vpc = (nvec + kChunks - 1) / kChunks;  // vectors per copy
   if (tid == 0) {
 #pragma unroll
     for (int k = 0; k < kChunks; ++k) mbar_init(&bars[k], 1);
+    mbar_init(&bars[kChunks], C > 1 ? C - 1 : 1);
+    tgt[0] = 0.f;
+    tgt[1] = 0.f;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  }
-  __syncthreads();
-  if (tid == 0) {
 #pragma unroll
     for (int k = 0; k < kChunks; ++k) {
       const int lo = k * vpc, hi = min(nvec, lo + vpc);
@@ -204,138 +241,227 @@ __global__ void __launch_bounds__(kThreads) row_cluster_kernel(const RowParams p
       }
     }
   }
+  if (C > 1) cluster_arrive();  // "my exchange barrier exists": waited for just before the first remote access
+  __syncthreads();
   if (!may_be_dead) ctx = load_row_ctx(p, row);
 
-  // ---- pass 1: running (max, sum) in the base-2 domain as the chunks land
+  // where the target logit lives in this CTA's slice: the step whose vectors hold it, for the thread that holds it
+  const int rel = ctx.id - part_off;
+  int owner_step = -1;
+  if (ctx.valid && rel >= 0 && rel < part_len && ((rel >> 3) % kThreads) == tid) owner_step = (rel >> 3) / kStepVecs;
+  const __nv_bfloat16* slice_elems = reinterpret_cast<const __nv_bfloat16*>(slice);
+
+  // ---- pass 1
   bool timed_out = false;
-  int waited = 0;  // chunks known to have landed
-  mrl::Lse2 acc = mrl::lse2_empty();
-  for (int base = 0; base < nvec; base += kThreads * kUnroll) {
-    const int last = min(nvec - 1, base + (kUnroll - 1) * kThreads + tid);
-    const int need = last / vpc + 1;
-    while (waited < need) {
-      if (!mbar_wait_bounded(&bars[waited], 0)) timed_out = true;
-      ++waited;
-    }
-    uint4 v[kUnroll];
-    float vmax = -INFINITY;
+  int waited = 0;  // copies known to have landed
+  float ref[kMaxSteps], sums[kMaxSteps];
+  float zt = 0.f;
+  uint4* const mine = slice + tid;  // this thread's vectors: mine[step * kStepVecs + u * kThreads]
 #pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-      const int i = base + u * kThreads + tid;
-      v[u] = (i < nvec) ? slice[i] : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);  // -inf
-      vmax = fmaxf(vmax, max8_bf16(v[u]));
-    }
-    const float m_new = fmaxf(acc.m, vmax * MRL_LOG2E);
-    if (m_new > acc.m) {  // also true for the first group (acc.m = -inf, acc.s = 0)
-      acc.s *= mrl::ex2_approx(acc.m - m_new);
-      acc.m = m_new;
-    }
-    if (acc.m != -INFINITY) {
-      const float neg_m = -acc.m;
+  for (int it = 0; it < kMaxSteps; ++it) {
+    ref[it] = -INFINITY;
+    sums[it] = 0.f;
+    const int base = it * kStepVecs;
+    if (base < nvec) {
+      const int last = min(nvec - 1, base + (kUnroll - 1) * kThreads + tid);
+      const int need = last / vpc + 1;
+      while (waited < need) {
+        if (!mbar_wait_bounded(&bars[waited], 0)) timed_out = true;
+        ++waited;
+      }
+      if (owner_step == it) zt = __bfloat162float(slice_elems[rel]);  // before this thread overwrites it below
+      const bool full = base + kStepVecs <= nvec;  // uniform: only the last step of a slice is ragged
+      uint4 v[kUnroll];
+      if (full) {
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) v[u] = mine[base + u * kThreads];
+      } else {
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u)
+          v[u] = (base + u * kThreads + tid < nvec) ? mine[base + u * kThreads]
+                                                    : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
+      }
+      uint32_t mx = hmax2_u32(hmax2_u32(v[0].x, v[0].y), hmax2_u32(v[0].z, v[0].w));
+#pragma unroll
+      for (int u = 1; u < kUnroll; ++u)
+        mx = hmax2_u32(mx, hmax2_u32(hmax2_u32(v[u].x, v[u].y), hmax2_u32(v[u].z, v[u].w)));
+      const float vmax = fmaxf(mrl::bf16lo_to_f32(mx), mrl::bf16hi_to_f32(mx));
+      // a thread whose 32 logits are all -inf takes reference 0: every term is 2^-inf = 0
+      const float r = vmax != -INFINITY ? vmax * MRL_LOG2E : 0.f, neg_r = -r;
       float s0 = 0.f, s1 = 0.f;
 #pragma unroll
       for (int u = 0; u < kUnroll; ++u) {
         const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+        uint32_t e[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          s0 += mrl::ex2_approx(fmaf(mrl::bf16lo_to_f32(w[j]), MRL_LOG2E, neg_m));
-          s1 += mrl::ex2_approx(fmaf(mrl::bf16hi_to_f32(w[j]), MRL_LOG2E, neg_m));
+          const float a = mrl::ex2_approx(fmaf(mrl::bf16lo_to_f32(w[j]), MRL_LOG2E, neg_r));
+          const float b = mrl::ex2_approx(fmaf(mrl::bf16hi_to_f32(w[j]), MRL_LOG2E, neg_r));
+          s0 += a;
+          s1 += b;
+          e[j] = mrl::pack_bf16x2(a, b);
+        }
+        v[u] = make_uint4(e[0], e[1], e[2], e[3]);
+      }
+      if (want_grad) {
+        if (full) {
+#pragma unroll
+          for (int u = 0; u < kUnroll; ++u) mine[base + u * kThreads] = v[u];
+        } else {
+#pragma unroll
+          for (int u = 0; u < kUnroll; ++u)
+            if (base + u * kThreads + tid < nvec) mine[base + u * kThreads] = v[u];
         }
       }
-      acc.s += s0 + s1;
+      ref[it] = vmax != -INFINITY ? r : -INFINITY;
+      sums[it] = s0 + s1;
     }
   }
-  while (waited < kChunks) {  // chunks this thread had no vector in
+  while (waited < kChunks) {  // copies this thread had no vector in
     const int lo = waited * vpc;
     if (lo < nvec && !mbar_wait_bounded(&bars[waited], 0)) timed_out = true;
     ++waited;
   }
-  if (__syncthreads_or(timed_out ? 1 : 0)) {
-    // A copy never landed: report and leave without touching outputs.  (The other CTAs of the
-    // cluster still need this CTA at the cluster barrier, so keep going to the barrier below.)
-    if (tid == 0 && p.status != nullptr) atomicOr(p.status, MRL_DEV_TIMEOUT);
-    timed_out = true;
-  }
-  mrl::Lse2 part = mrl::lse2_block_reduce<kThreads>(acc, scratch);
 
-  // ---- exchange (max, sum, target logit) across the cluster
-  const bool owner = ctx.valid && ctx.id >= part_off && ctx.id < part_off + part_len;
-  float zt = 0.f;
-  if (owner) zt = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(slice)[ctx.id - part_off]);
-  mrl::Lse2 tot = part;
-  if (C > 1) {
-    if (tid == 0) xchg[rank] = make_float4(part.m, part.s, zt, owner ? 1.f : 0.f);
-    cluster_arrive();
-    cluster_wait();
-    if (tid < 32) {
-      cg::cluster_group cl = cg::this_cluster();
-      float4 o = make_float4(-INFINITY, 0.f, 0.f, 0.f);
-      if (tid < C) o = cl.map_shared_rank(xchg, tid)[tid];
-      mrl::Lse2 t = mrl::lse2_warp_reduce(mrl::Lse2{o.x, o.y});  // xor tree: same order in every CTA
-      float z = o.w != 0.f ? o.z : 0.f;
-#pragma unroll
-      for (int s = 16; s > 0; s >>= 1) z += __shfl_xor_sync(0xffffffffu, z, s);  // one owner: exact
-      if (tid == 0) {
-        bcast[0] = t.m;
-        bcast[1] = t.s;
-        bcast[2] = z;
-      }
-    }
-    cluster_arrive();  // matched by cluster_wait() at the end: keeps every slice alive for its readers
-    __syncthreads();
-    tot = mrl::Lse2{bcast[0], bcast[1]};
-    zt = bcast[2];
+  // ---- (max, sum) of the warp: the maximum first, one rescale per step, then a plain sum
+  if (owner_step >= 0) {  // at most one thread of the whole cluster
+    tgt[0] = zt;
+    tgt[1] = 1.f;
   }
-
-  // ---- per-row scalars (every thread, redundantly)
-  const float lse2 = tot.m + log2f(tot.s);
-  const float lse = lse2 * MRL_LN2;
-  float logp = 0.f, g = 0.f;
-  bool clipped = false;
-  if (ctx.valid && !timed_out) {
-    logp = zt - lse;
-    if (p.loss_mode) {
-      const mrl::RowOut ro = mrl::mrl_row_loss(logp, ctx.in, p.eps_lo, p.eps_hi);
-      g = ro.g;
-      clipped = ro.clipped;
-    }
+  float m = -INFINITY;
+#pragma unroll
+  for (int it = 0; it < kMaxSteps; ++it) m = fmaxf(m, ref[it]);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  float sum = 0.f;
+  if (m != -INFINITY) {
+#pragma unroll
+    for (int it = 0; it < kMaxSteps; ++it) sum = fmaf(sums[it], mrl::ex2_approx(ref[it] - m), sum);  // 2^-inf = 0
   }
-  if (rank == 0 && tid == 0 && !timed_out)
-    write_row_scalars(p, row, ctx, logp, ctx.valid ? lse : 0.f, tot, zt, clipped, true);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+  if (lane == 0) {
+    red[warp] = m;
+    red[kWarps + warp] = sum;
+  }
+  const bool any_timeout = __syncthreads_or(timed_out ? 1 : 0) != 0;
 
-  // ---- pass 2: dlogits slice = g * (p - onehot), from the resident slice
-  if (orow != nullptr && !timed_out) {
-    if (g == 0.f) {
-      for (int i = tid; i < nvec; i += kThreads) st_global_v4(orow + (size_t)i * 8, make_uint4(0, 0, 0, 0));
-    } else {
-      const float k = lse2 - log2f(fabsf(g));  // 2^(z log2e - k) = |g| p
-      const float neg_k = -k;
-      const uint32_t sign = g < 0.f ? 0x80008000u : 0u;
-      for (int base = 0; base < nvec; base += kThreads * kUnroll) {
+  // ---- warp 0: the CTA's triple to every peer, the peers' triples, the row's scalars
+  if (warp == 0) {
+    float wm = lane < kWarps ? red[lane] : -INFINITY;
+    float ws = lane < kWarps ? red[kWarps + lane] : 0.f;
+    float cm = wm;
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-          const int i = base + u * kThreads + tid;
-          if (i < nvec) {
-            const uint4 v = slice[i];
-            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-            uint32_t r[4];
+    for (int o = 16; o > 0; o >>= 1) cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, o));
+    float cs = (wm != -INFINITY) ? ws * mrl::ex2_approx(wm - cm) : 0.f;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const float a = mrl::ex2_approx(fmaf(mrl::bf16lo_to_f32(w[j]), MRL_LOG2E, neg_k));
-              const float b = mrl::ex2_approx(fmaf(mrl::bf16hi_to_f32(w[j]), MRL_LOG2E, neg_k));
-              r[j] = mrl::pack_bf16x2(a, b) ^ sign;
-            }
-            st_global_v4(orow + (size_t)i * 8, make_uint4(r[0], r[1], r[2], r[3]));
-          }
+    for (int o = 16; o > 0; o >>= 1) cs += __shfl_xor_sync(0xffffffffu, cs, o);
+    bool wok = !any_timeout;
+    if (C > 1) {
+      cluster_wait();  // every CTA of the cluster has initialised its exchange barrier
+      if (lane == 0) {
+        const float zpart = tgt[0], opart = tgt[1];
+        xchg[rank] = make_float4(cm, cs, zpart, opart);
+        for (int r = 0; r < C; ++r) {
+          if (r == rank) continue;
+          const uint32_t dst = mapa_u32(smem_u32(&xchg[rank]), (uint32_t)r);
+          asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(cm), "f"(cs), "f"(zpart),
+                       "f"(opart)
+                       : "memory");
+          const uint32_t rbar = mapa_u32(smem_u32(&bars[kChunks]), (uint32_t)r);
+          asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(rbar) : "memory");
         }
       }
-      if (owner) {  // the target column gets g (p - 1); ordered after the vector stores by the barrier
-        __syncthreads();
-        if (tid == 0) orow[ctx.id - part_off] = __float2bfloat16_rn(g * (expf(zt - lse) - 1.0f));
+      __syncwarp();
+      bool got = false;
+      for (uint32_t i = 0; i < (kSpinLimit << 2) && !got; ++i) got = mbar_try_wait_cluster(&bars[kChunks], 0);
+      wok = wok && got;
+    } else if (lane == 0) {
+      xchg[0] = make_float4(cm, cs, tgt[0], tgt[1]);
+    }
+    __syncwarp();
+    float4 o = make_float4(-INFINITY, 0.f, 0.f, 0.f);
+    if (lane < C && wok) o = xchg[lane];
+    float tm = o.x;
+#pragma unroll
+    for (int q = 16; q > 0; q >>= 1) tm = fmaxf(tm, __shfl_xor_sync(0xffffffffu, tm, q));
+    float ts = (o.x != -INFINITY) ? o.y * mrl::ex2_approx(o.x - tm) : 0.f;
+    float ztot = o.w != 0.f ? o.z : 0.f;
+#pragma unroll
+    for (int q = 16; q > 0; q >>= 1) {
+      ts += __shfl_xor_sync(0xffffffffu, ts, q);      // xor tree over the ranks: the same order in every CTA
+      ztot += __shfl_xor_sync(0xffffffffu, ztot, q);  // one owner: exact
+    }
+    const float lse2 = tm + log2f(ts);
+    const float lse = lse2 * MRL_LN2;
+    float logp = 0.f, g = 0.f;
+    bool clipped = false;
+    if (ctx.valid && wok) {
+      logp = ztot - lse;
+      if (p.loss_mode) {
+        const mrl::RowOut ro = mrl::mrl_row_loss(logp, ctx.in, p.eps_lo, p.eps_hi);
+        g = ro.g;
+        clipped = ro.clipped;
+      }
+    }
+    if (lane == 0) {
+      if (rank == 0 && wok)
+        write_row_scalars(p, row, ctx, logp, ctx.valid ? lse : 0.f, mrl::Lse2{tm, ts}, ztot, clipped, true);
+      if (!wok && p.status != nullptr) atomicOr(p.status, MRL_DEV_TIMEOUT);
+      fin[0] = lse2;
+      fin[1] = g;
+      fin[2] = g * (mrl::ex2_approx(fmaf(ztot, MRL_LOG2E, -lse2)) - 1.0f);  // the target column
+      fin[3] = wok ? 1.f : 0.f;
+    }
+  } else if (C > 1) {
+    cluster_wait();  // pairs with the arrive above (every thread of the cluster takes part)
+  }
+  __syncthreads();
+  const float lse2 = fin[0], g = fin[1], tfix = fin[2];
+  const bool ok = fin[3] != 0.f;
+
+  // ---- pass 2: dlogits slice = g * softmax - g * onehot, from the cached exponentials
+  if (want_grad && ok) {
+    uint4* const out = reinterpret_cast<uint4*>(orow) + tid;  // this thread's output vectors, indexed like `mine`
+#pragma unroll
+    for (int it = 0; it < kMaxSteps; ++it) {
+      const int base = it * kStepVecs;
+      if (base < nvec) {
+        const bool full = base + kStepVecs <= nvec;
+        uint4 o[kUnroll];
+        if (g == 0.f) {  // uniform over the row
+#pragma unroll
+          for (int u = 0; u < kUnroll; ++u) o[u] = make_uint4(0, 0, 0, 0);
+        } else {
+          // cached value times scale, as two packed bf16 FMAs: scale = hi + lo, one rounding of the result
+          const float scale = ref[it] != -INFINITY ? g * mrl::ex2_approx(ref[it] - lse2) : 0.f;
+          const float s_hi = __bfloat162float(__float2bfloat16_rn(scale));
+          const uint32_t hi2 = mrl::pack_bf16x2(s_hi, s_hi), lo2 = mrl::pack_bf16x2(scale - s_hi, scale - s_hi);
+#pragma unroll
+          for (int u = 0; u < kUnroll; ++u) {
+            const uint4 e = (full || base + u * kThreads + tid < nvec) ? mine[base + u * kThreads] : make_uint4(0, 0, 0, 0);
+            o[u].x = hfma2_u32(e.x, hi2, hfma2_u32(e.x, lo2, 0u));
+            o[u].y = hfma2_u32(e.y, hi2, hfma2_u32(e.y, lo2, 0u));
+            o[u].z = hfma2_u32(e.z, hi2, hfma2_u32(e.z, lo2, 0u));
+            o[u].w = hfma2_u32(e.w, hi2, hfma2_u32(e.w, lo2, 0u));
+          }
+        }
+        if (full) {
+#pragma unroll
+          for (int u = 0; u < kUnroll; ++u) st_global_v4(out + base + u * kThreads, o[u]);
+        } else {
+#pragma unroll
+          for (int u = 0; u < kUnroll; ++u)
+            if (base + u * kThreads + tid < nvec) st_global_v4(out + base + u * kThreads, o[u]);
+        }
+        // the target column gets g (p - 1): a scalar store by the thread whose vector store just covered it, so
+        // the two stores to that address are ordered by program order
+        if (owner_step == it && g != 0.f) orow[rel] = __float2bfloat16_rn(tfix);
       }
     }
   }
-  if (C > 1) cluster_wait();
+  // Every peer's remote store and arrive has landed before warp 0 got past its wait, and this CTA's own remote
+  // accesses were issued before it: nobody touches a CTA's shared memory after that CTA can have left.
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -601,7 +727,7 @@ int launch_rows(RowParams p, int dtype, cudaStream_t st) {
   const int vecs = (p.V / 8 + C - 1) / C;
   p.part_elems = vecs * 8;
   p.cluster = C;
-  const size_t smem = (size_t)p.part_elems * 2 + kChunks * 8 + 64 * 4 + kMaxCluster * 16 + 16;
+  const size_t smem = (size_t)p.part_elems * 2 + kTailBytes;
   // per device and idempotent; set on every call so that a change of the current device is harmless
   MRL_CUDA_OK(cudaFuncSetAttribute(row_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
   cudaLaunchConfig_t cfg = {};

@@ -281,9 +281,11 @@ def test_clip_boundary_neighbourhood():
     lp = make_lp()
     got = run_gpu_policy_loss(z, ids, None, cu, adv, old.float(), None, None, lp)
     ref = O.policy_loss(z, ids, None, cu, adv, old.float(), None, None, oracle_lp(lp))
-    # the rows come in +A / -A pairs, so the loss cancels to ~1e-5 of its terms by construction:
-    # the relative tolerance is taken against 1e-3 of the sum of |terms| instead of the residue
-    compare_policy_loss(got, ref, V, torch.bfloat16, loss_floor=1e-3 * float(ref["pg_term"].abs().sum()))
+    # The rows come in +A / -A pairs, so the loss cancels to ~1e-5 of its terms by construction.  A float32 sum
+    # of 2^x carries ~1e-7 relative error, hence each term ~1e-7 of itself and the loss ~1e-7 of the sum of |terms|
+    # whatever the residue is: "1e-5 relative under float32 accumulation" can only be asked down to a residue of
+    # 1e-2 of the sum of |terms|, which is the floor used here.
+    compare_policy_loss(got, ref, V, torch.bfloat16, loss_floor=1e-2 * float(ref["pg_term"].abs().sum()))
 
 
 def test_prop1_bandit_on_gpu():
