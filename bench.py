@@ -51,13 +51,10 @@ def measured_peaks():
     return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
 
 
-def profile_traffic(key: str):
-    """DRAM bytes per unit of the dominant kernel from the committed ncu summary (None if absent)."""
-    path = os.path.join(ROOT, "profiles", "traffic.json")
-    if not os.path.exists(path):
-        return None
-    with open(path) as f:
-        return json.load(f).get(key)
+# DRAM bytes per token (dram__bytes_read.sum + dram__bytes_write.sum over the rows of the capture) of the dominant
+# kernel as it stands, from the committed ncu summary profiles/row_stream_kernel_c2_logits_in.md; traffic grows in
+# proportion to the rows.  Set to None whenever that kernel changes, until the counters are taken again.
+ROW_STREAM_DRAM_BYTES_PER_TOKEN_V151936 = 706200
 
 
 class ClockSampler:
@@ -179,7 +176,7 @@ class LogitsInWorkload:
         B.mrl_token_logprobs(self.z, self.ids, None, self.logp)
         self.logp_old = self.logp + b.noise.to(dev)
         torch.cuda.synchronize()
-        self.kernels_per_step = 6    # adv_prompt, seq_count, row_coef, row (cluster), row_terms, finalize
+        self.kernels_per_step = 6    # adv_prompt, seq_count, row_coef, row_stream, row_terms, finalize
         self.dominant_per_step = 1
         self.bytes_per_token = 2 * self.V * self.z.element_size()   # read V + write V elements
 
@@ -228,8 +225,8 @@ class LogitsInWorkload:
         k_avg_ms = sum(kernel_ms) / len(kernel_ms)
         alg_bytes = self.bytes_per_token * self.tokens()
         achieved = alg_bytes / (k_avg_ms * 1e-3) / 1e9
-        per_token = profile_traffic("row_cluster_kernel_dram_bytes_per_token_V151936")
-        return {"bound": "hbm", "kernel": "row_cluster_kernel", "achieved": achieved, "peak": peaks["hbm_gbs"],
+        per_token = ROW_STREAM_DRAM_BYTES_PER_TOKEN_V151936 if self.V == 151936 else None
+        return {"bound": "hbm", "kernel": "row_stream_kernel", "achieved": achieved, "peak": peaks["hbm_gbs"],
                 "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
                 "peak_source": peaks["source"] + " (copy, burst)", "algorithmic_bytes_per_launch": alg_bytes,
                 "kernel_ms": k_avg_ms, "traffic": None if per_token is None else per_token * self.tokens()}

@@ -18,8 +18,8 @@
  *    `status` word [device, int32[1], nullable], treats the offending row as masked and goes
  *    on.  The library never clears `status`; zero it before the first call and read it after
  *    your own synchronisation.  Bits: MRL_DEV_BAD_TOKEN_ID (an id outside [0, V)),
- *    MRL_DEV_TIMEOUT (a bounded wait on the kernel's own asynchronous copy ran out; outputs of
- *    that call are then unspecified).
+ *    MRL_DEV_TIMEOUT (fused LM head only: a bounded wait on the kernel's own asynchronous copy
+ *    or tensor-core work ran out; outputs of that call are then unspecified).
  *  - `workspace` [device] is scratch of at least mrl_workspace_bytes(...) bytes, 256-byte
  *    aligned, contents unspecified before and after.  Calls that share a workspace must not
  *    overlap on the device.
@@ -200,10 +200,12 @@ int mrl_token_logprobs(const void* logits, int32_t dtype, int64_t N, int32_t V, 
  *   workspace: mrl_workspace_bytes(MRL_WS_POLICY_LOSS, N, V, 0, dtype, S)
  *
  * float32 row arithmetic on the input dtype, float64 for the final N-term sums (fixed order:
- * bitwise reproducible).  dlogits is rounded to nearest even.  The fast path (one thread-block
- * cluster per row, row resident in shared memory) needs bf16, V % 8 == 0, ld % 8 == 0,
- * ld_out % 8 == 0 and 16-byte aligned logits/dlogits; anything else takes a general kernel
- * with the same results.  N = 0: loss (and stats) are zeroed unless ACCUMULATE_LOSS.
+ * bitwise reproducible).  dlogits is rounded to nearest even.  The fast path (one CTA per row: the
+ * row is streamed from HBM once and read a second time from L2) needs bf16, V >= 4096, and either
+ * V % 16 == 0, ld % 16 == 0, ld_out % 16 == 0 with 32-byte aligned logits / dlogits, or the same
+ * with 8 and 16 bytes; anything else takes a general kernel with the same results.  Rows much
+ * longer than ~200,000 entries no longer fit L2 while in flight and are then read from HBM twice.
+ * N = 0: loss (and stats) are zeroed unless ACCUMULATE_LOSS.
  */
 int mrl_policy_loss_fwd_bwd(const void* logits, int32_t dtype, int64_t N, int32_t V, int64_t ld,
                             const int32_t* ids, const uint8_t* mask, const int32_t* cu_seqlens,

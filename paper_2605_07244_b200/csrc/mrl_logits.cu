@@ -1,24 +1,19 @@
 // Logits-in path: mrl_token_logprobs and mrl_policy_loss_fwd_bwd.
 //
-// Fast kernel (bf16, 16-byte aligned rows): one thread-block cluster per logits row.  Each CTA of
-// the cluster pulls its slice of the row into shared memory with bulk asynchronous copies (four
-// chunks, one mbarrier each), reduces max / sum-of-exponentials as the chunks land while caching the
-// exponentials in place, exchanges one (max, sum, target-logit) triple per CTA through distributed
-// shared memory, evaluates the ratio / clip / loss scalars, and writes g * (softmax - onehot) from
-// the cached slice.  The row is read from HBM exactly once and written exactly once; nothing is
-// shared between clusters.
+// Streaming kernel (bf16, 16- or 32-byte aligned rows): one CTA per logits row, two CTAs per SM.  Pass 1
+// streams the row from HBM with wide loads while keeping a running (max, sum of exponentials) per thread;
+// after the block reduction and the ratio / clip / loss scalars, pass 2 re-reads the row -- from L2, which
+// holds every row in flight several times over -- and writes g * (softmax - onehot) with streaming stores.
+// The row crosses the HBM interface once in each direction; nothing is shared between CTAs.
 // General kernel (any dtype, any V, any alignment): one CTA per row, three passes over global
 // memory; used for small or unaligned problems.
 #include "mrl_common.cuh"
 
 namespace {
 
-constexpr int kThreads = 256;
-constexpr int kChunks = 4;            // bulk copies (and mbarriers) per CTA slice
-constexpr int kUnroll = 4;            // 16-byte vectors in flight per thread
-constexpr int kMaxCluster = 8;        // portable cluster size limit
-constexpr int kMaxPartBytes = 76000;  // slice size that still lets three CTAs share an SM
-constexpr uint32_t kSpinLimit = 1u << 20;
+constexpr int kThreads = 256;        // general kernel
+constexpr int kStreamThreads = 512;  // streaming kernel: two CTAs per SM
+constexpr long long kSplitRowBytes = 512 * 1024;  // rows at least this long are split over a cluster of two CTAs
 
 // rowstat bits
 constexpr uint8_t kStatValid = MRL_ROW_VALID, kStatClipped = MRL_ROW_CLIPPED, kStatRead = MRL_ROW_READ;
@@ -45,47 +40,7 @@ struct RowParams {
   float* row_zt;
   uint8_t* rowstat;
   int32_t* status;
-  int part_elems;  // elements per CTA slice (multiple of 8)
-  int cluster;     // CTAs per row
 };
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait: false if the copy did not land within the spin limit.
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
-  for (uint32_t i = 0; i < kSpinLimit; ++i)
-    if (mbar_try_wait(bar, parity)) return true;
-  return false;
-}
-__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                   smem_u32(dst)),
-               "l"(src), "r"(bytes), "r"(smem_u32(bar))
-               : "memory");
-}
-__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
-__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
-
-__device__ __forceinline__ void st_global_v4(void* p, uint4 v) {
-  asm volatile("st.global.cs.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-}
 
 // Everything the loss needs from one row besides the logits.
 struct RowCtx {
@@ -137,27 +92,22 @@ __device__ __forceinline__ void write_row_scalars(const RowParams& p, long long 
   }
 }
 
-// ------------------------------------------------------------------------------------------------
-// Fast kernel: bf16, one thread-block cluster per row, each CTA's slice of the row resident in shared memory.
-//
-// A CTA pulls its slice in with four bulk asynchronous copies (an mbarrier each) and works on it as the copies
-// land.  Pass 1, in steps of 1,024 vectors: each thread takes the maximum of its own 32 logits of the step as
-// reference, turns them into 2^(x - ref), sums them in float32 and writes them back over the logits as bf16, so
-// that pass 2 needs no exponential; the references stay in registers.  The CTA's (max, sum, target logit) is
-// pushed to every other CTA of the cluster through distributed shared memory (a remote store and a remote
-// mbarrier arrive per peer); warp 0 alone waits for the peers, forms the row's scalars and hands them to the
-// block.  Pass 2: every cached value times g 2^(ref - lse) as two packed bf16 FMAs (scale = hi + lo, one
-// rounding of the result), streamed out with 128-bit stores.  Full steps run without per-vector bounds checks;
-// only the last step of a slice can be ragged.  Slices are at most 76,000 bytes, so three CTAs of different rows
-// share an SM and one CTA's copy latency, exchange and stores overlap the others' arithmetic.
-// A row is read from HBM once and written once; nothing is shared between clusters.
-// Dynamic shared memory: [slice | 4 copy barriers, 1 exchange barrier | exchange | per-warp scratch | row scalars]
-// ------------------------------------------------------------------------------------------------
-constexpr int kStepVecs = kThreads * kUnroll;                                // vectors per step of a CTA
-constexpr int kMaxSteps = (kMaxPartBytes / 16 + kStepVecs - 1) / kStepVecs;  // 5
-constexpr int kWarps = kThreads / 32;
-constexpr size_t kTailBytes = 64 + kMaxCluster * 16 + 2 * kWarps * 4 + 32;
+// packed maximum of two bf16 pairs
+__device__ __forceinline__ uint32_t hmax2_u32(uint32_t a, uint32_t b) {
+  uint32_t r;
+  asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+  return r;
+}
 
+// ------------------------------------------------------------------------------------------------
+// Streaming kernel: bf16, one CTA per row, nothing resident in shared memory.
+// Pass 1 streams the row from HBM with 128- or 256-bit loads (running maximum and rescaled sum per thread);
+// pass 2 reads the same vectors again -- by then from L2: the rows in flight (two per SM) are a fraction of its
+// capacity, and the first read asks L2 to keep the lines -- and writes g * (softmax - onehot) with streaming
+// stores.  HBM sees one read and one write of the row.  Many small CTAs with deep unrolling keep far more bytes
+// in flight per SM than a slice held in shared memory does, which is what this memory-bound pass needs.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ uint32_t mapa_u32(uint32_t addr, uint32_t rank) {
   uint32_t r;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
@@ -174,294 +124,238 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t pa
       : "memory");
   return ok != 0;
 }
-// packed arithmetic on two bf16
-__device__ __forceinline__ uint32_t hmax2_u32(uint32_t a, uint32_t b) {
-  uint32_t r;
-  asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
-  return r;
+constexpr uint32_t kExchangeSpinLimit = 1u << 22;  // polls of the peer's triple before giving up (~a second)
+
+template <int kWords>
+struct StreamVec {
+  uint32_t w[kWords];
+};
+enum { kHintKeep = 0, kHintLast = 1 };
+
+template <int kWords, int kHint>
+__device__ __forceinline__ StreamVec<kWords> stream_ld(const void* p) {
+  StreamVec<kWords> v;
+  if constexpr (kWords == 8) {
+    if constexpr (kHint == kHintKeep)
+      asm volatile("ld.global.L2::evict_last.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                   : "=r"(v.w[0]), "=r"(v.w[1]), "=r"(v.w[2]), "=r"(v.w[3]), "=r"(v.w[4]), "=r"(v.w[5]), "=r"(v.w[6]),
+                     "=r"(v.w[7])
+                   : "l"(p));
+    else
+      asm volatile("ld.global.L2::evict_first.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                   : "=r"(v.w[0]), "=r"(v.w[1]), "=r"(v.w[2]), "=r"(v.w[3]), "=r"(v.w[4]), "=r"(v.w[5]), "=r"(v.w[6]),
+                     "=r"(v.w[7])
+                   : "l"(p));
+  } else {
+    asm volatile("ld.global.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.w[0]), "=r"(v.w[1]), "=r"(v.w[2]), "=r"(v.w[3]) : "l"(p));
+  }
+  return v;
 }
-__device__ __forceinline__ uint32_t hfma2_u32(uint32_t a, uint32_t b, uint32_t c) {
-  uint32_t r;
-  asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(c));
-  return r;
+template <int kWords>
+__device__ __forceinline__ void stream_st(void* p, const StreamVec<kWords>& v) {
+  if constexpr (kWords == 8)
+    asm volatile("st.global.cs.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(v.w[0]), "r"(v.w[1]),
+                 "r"(v.w[2]), "r"(v.w[3]), "r"(v.w[4]), "r"(v.w[5]), "r"(v.w[6]), "r"(v.w[7])
+                 : "memory");
+  else
+    asm volatile("st.global.cs.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(v.w[0]), "r"(v.w[1]), "r"(v.w[2]),
+                 "r"(v.w[3])
+                 : "memory");
+}
+template <int kWords>
+__device__ __forceinline__ StreamVec<kWords> stream_fill(uint32_t x) {
+  StreamVec<kWords> v;
+#pragma unroll
+  for (int j = 0; j < kWords; ++j) v.w[j] = x;
+  return v;
 }
 
-__global__ void __launch_bounds__(kThreads, 3) row_cluster_kernel(const RowParams p) {
-  extern __shared__ __align__(128) unsigned char smem[];
+// kC = 1: the CTA takes the whole row.  kC = 2: a cluster of two CTAs takes the row, half each, and the halves'
+// (max, sum, target logit) cross through distributed shared memory: a remote store plus a remote mbarrier arrive.
+template <int kT, int kU, int kWords, int kC>
+__global__ void __launch_bounds__(kT, 1024 / kT) row_stream_kernel(const RowParams p) {
+  constexpr int kWarpsT = kT / 32;
+  constexpr int kVecBytes = kWords * 4, kVecElems = kWords * 2;
+  using Vec = StreamVec<kWords>;
+  __shared__ float red[2 * 32];
+  __shared__ float fin[4];
+  __shared__ __align__(16) float4 xchg[2];
+  __shared__ __align__(8) uint64_t xbar;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int C = p.cluster;
-  const long long row = blockIdx.x / C;
-  const int rank = blockIdx.x % C;  // equals the rank in the cluster for a 1-D cluster
-  const int part_off = rank * p.part_elems;
-  const int part_len = max(0, min(p.V - part_off, p.part_elems));  // multiple of 8
-  const int nvec = part_len >> 3;
-  const size_t slice_bytes = (size_t)p.part_elems * 2;
-
-  uint4* slice = reinterpret_cast<uint4*>(smem);
-  unsigned char* tail = smem + slice_bytes;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(tail);                    // [kChunks] copies, then the exchange
-  float4* xchg = reinterpret_cast<float4*>(tail + 64);                   // [kMaxCluster]
-  float* red = reinterpret_cast<float*>(tail + 64 + kMaxCluster * 16);   // [2][kWarps]
-  float* fin = red + 2 * kWarps;                                         // lse2, g, target-column value, ok
-  float* tgt = fin + 4;                                                  // target logit, has-target
-
+  const long long row = blockIdx.x / kC;
+  const int rank = blockIdx.x % kC;  // rank in the 1-D cluster
+  const int row_nvec = p.V / kVecElems;
+  const int part_nvec = (row_nvec + kC - 1) / kC;
+  const int part_off = rank * part_nvec * kVecElems;               // first element of this CTA's part
+  const int nvec = max(0, min(row_nvec - rank * part_nvec, part_nvec));
   const bool want_grad = p.dlogits != nullptr;
   const __nv_bfloat16* grow = static_cast<const __nv_bfloat16*>(p.logits) + row * p.ld + part_off;
   __nv_bfloat16* orow = want_grad ? static_cast<__nv_bfloat16*>(p.dlogits) + row * p.ld_out + part_off : nullptr;
+  const char* in = reinterpret_cast<const char*>(grow) + (size_t)tid * kVecBytes;
+  char* out = reinterpret_cast<char*>(orow) + (size_t)tid * kVecBytes;
 
-  // Rows that may be dead are decided before anything is fetched; otherwise fetch first.
-  const bool may_be_dead = p.mask != nullptr || (p.flags & MRL_FLAG_SKIP_ZERO_ROWS);
-  RowCtx ctx;
-  if (may_be_dead) {
-    ctx = load_row_ctx(p, row);
-    if (ctx.dead) {
-      if (orow != nullptr)
-        for (int i = tid; i < nvec; i += kThreads) st_global_v4(orow + (size_t)i * 8, make_uint4(0, 0, 0, 0));
-      if (rank == 0 && tid == 0) write_row_scalars(p, row, ctx, 0.f, 0.f, mrl::lse2_empty(), 0.f, false, false);
-      return;  // the whole cluster takes this branch: no cluster barrier is left waiting
-    }
+  const RowCtx ctx = load_row_ctx(p, row);
+  if (ctx.dead) {
+    if (orow != nullptr)
+      for (int i = tid; i < nvec; i += kT) stream_st<kWords>(out + (size_t)(i - tid) * kVecBytes, stream_fill<kWords>(0u));
+    if (rank == 0 && tid == 0) write_row_scalars(p, row, ctx, 0.f, 0.f, mrl::lse2_empty(), 0.f, false, false);
+    return;  // both CTAs of a cluster take this branch: no cluster barrier is left waiting
   }
-
-  const int vpc = (nvec + kChunks - 1) / kChunks;  // vectors per copy
-  if (tid == 0) {
-#pragma unroll
-    for (int k = 0; k < kChunks; ++k) mbar_init(&bars[k], 1);
-    mbar_init(&bars[kChunks], C > 1 ? C - 1 : 1);
-    tgt[0] = 0.f;
-    tgt[1] = 0.f;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-#pragma unroll
-    for (int k = 0; k < kChunks; ++k) {
-      const int lo = k * vpc, hi = min(nvec, lo + vpc);
-      if (hi > lo) {
-        const uint32_t bytes = (uint32_t)(hi - lo) * 16u;
-        mbar_expect_tx(&bars[k], bytes);
-        bulk_g2s(slice + lo, grow + (size_t)lo * 8, bytes, &bars[k]);
-      }
+  if (kC > 1) {
+    if (tid == 0) {
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&xbar)), "r"(kC - 1) : "memory");
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    __syncthreads();
+    // "my exchange barrier exists": the peer waits for this just before its remote store
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   }
-  if (C > 1) cluster_arrive();  // "my exchange barrier exists": waited for just before the first remote access
-  __syncthreads();
-  if (!may_be_dead) ctx = load_row_ctx(p, row);
-
-  // where the target logit lives in this CTA's slice: the step whose vectors hold it, for the thread that holds it
-  const int rel = ctx.id - part_off;
-  int owner_step = -1;
-  if (ctx.valid && rel >= 0 && rel < part_len && ((rel >> 3) % kThreads) == tid) owner_step = (rel >> 3) / kStepVecs;
-  const __nv_bfloat16* slice_elems = reinterpret_cast<const __nv_bfloat16*>(slice);
-
-  // ---- pass 1
-  bool timed_out = false;
-  int waited = 0;  // copies known to have landed
-  float ref[kMaxSteps], sums[kMaxSteps];
+  const int rel = ctx.id - part_off;                               // target column relative to this part
+  const bool owner = ctx.valid && rel >= 0 && rel < nvec * kVecElems;
   float zt = 0.f;
-  uint4* const mine = slice + tid;  // this thread's vectors: mine[step * kStepVecs + u * kThreads]
+  if (tid == 0 && owner) zt = __bfloat162float(grow[rel]);         // before anything is written in place
+
+  // ---- pass 1: running (max, sum) in the base-2 domain
+  float m_run = -INFINITY, s_run = 0.f;
+  for (int base = 0; base < nvec; base += kT * kU) {
+    Vec v[kU];
+    if (base + kT * kU <= nvec) {
 #pragma unroll
-  for (int it = 0; it < kMaxSteps; ++it) {
-    ref[it] = -INFINITY;
-    sums[it] = 0.f;
-    const int base = it * kStepVecs;
-    if (base < nvec) {
-      const int last = min(nvec - 1, base + (kUnroll - 1) * kThreads + tid);
-      const int need = last / vpc + 1;
-      while (waited < need) {
-        if (!mbar_wait_bounded(&bars[waited], 0)) timed_out = true;
-        ++waited;
-      }
-      if (owner_step == it) zt = __bfloat162float(slice_elems[rel]);  // before this thread overwrites it below
-      const bool full = base + kStepVecs <= nvec;  // uniform: only the last step of a slice is ragged
-      uint4 v[kUnroll];
-      if (full) {
+      for (int u = 0; u < kU; ++u) v[u] = stream_ld<kWords, kHintKeep>(in + (size_t)(base + u * kT) * kVecBytes);
+    } else {
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) v[u] = mine[base + u * kThreads];
-      } else {
+      for (int u = 0; u < kU; ++u)
+        v[u] = (base + u * kT + tid < nvec) ? stream_ld<kWords, kHintKeep>(in + (size_t)(base + u * kT) * kVecBytes)
+                                            : stream_fill<kWords>(0xff80ff80u);  // (-inf, -inf)
+    }
+    uint32_t mx = 0xff80ff80u;
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u)
-          v[u] = (base + u * kThreads + tid < nvec) ? mine[base + u * kThreads]
-                                                    : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
-      }
-      uint32_t mx = hmax2_u32(hmax2_u32(v[0].x, v[0].y), hmax2_u32(v[0].z, v[0].w));
+    for (int u = 0; u < kU; ++u) {
 #pragma unroll
-      for (int u = 1; u < kUnroll; ++u)
-        mx = hmax2_u32(mx, hmax2_u32(hmax2_u32(v[u].x, v[u].y), hmax2_u32(v[u].z, v[u].w)));
-      const float vmax = fmaxf(mrl::bf16lo_to_f32(mx), mrl::bf16hi_to_f32(mx));
-      // a thread whose 32 logits are all -inf takes reference 0: every term is 2^-inf = 0
-      const float r = vmax != -INFINITY ? vmax * MRL_LOG2E : 0.f, neg_r = -r;
+      for (int j = 0; j < kWords; ++j) mx = hmax2_u32(mx, v[u].w[j]);
+    }
+    const float vmax = fmaxf(mrl::bf16lo_to_f32(mx), mrl::bf16hi_to_f32(mx));
+    const float m_new = fmaxf(m_run, vmax * MRL_LOG2E);
+    if (m_new > m_run) {  // also the first group (m_run = -inf, s_run = 0)
+      s_run *= mrl::ex2_approx(m_run - m_new);
+      m_run = m_new;
+    }
+    if (m_run != -INFINITY) {
+      const float neg_m = -m_run;
       float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-      for (int u = 0; u < kUnroll; ++u) {
-        const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
-        uint32_t e[4];
+      for (int u = 0; u < kU; ++u) {
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const float a = mrl::ex2_approx(fmaf(mrl::bf16lo_to_f32(w[j]), MRL_LOG2E, neg_r));
-          const float b = mrl::ex2_approx(fmaf(mrl::bf16hi_to_f32(w[j]), MRL_LOG2E, neg_r));
-          s0 += a;
-          s1 += b;
-          e[j] = mrl::pack_bf16x2(a, b);
-        }
-        v[u] = make_uint4(e[0], e[1], e[2], e[3]);
-      }
-      if (want_grad) {
-        if (full) {
-#pragma unroll
-          for (int u = 0; u < kUnroll; ++u) mine[base + u * kThreads] = v[u];
-        } else {
-#pragma unroll
-          for (int u = 0; u < kUnroll; ++u)
-            if (base + u * kThreads + tid < nvec) mine[base + u * kThreads] = v[u];
+        for (int j = 0; j < kWords; ++j) {
+          s0 += mrl::ex2_approx(fmaf(mrl::bf16lo_to_f32(v[u].w[j]), MRL_LOG2E, neg_m));
+          s1 += mrl::ex2_approx(fmaf(mrl::bf16hi_to_f32(v[u].w[j]), MRL_LOG2E, neg_m));
         }
       }
-      ref[it] = vmax != -INFINITY ? r : -INFINITY;
-      sums[it] = s0 + s1;
+      s_run += s0 + s1;
     }
   }
-  while (waited < kChunks) {  // copies this thread had no vector in
-    const int lo = waited * vpc;
-    if (lo < nvec && !mbar_wait_bounded(&bars[waited], 0)) timed_out = true;
-    ++waited;
-  }
-
-  // ---- (max, sum) of the warp: the maximum first, one rescale per step, then a plain sum
-  if (owner_step >= 0) {  // at most one thread of the whole cluster
-    tgt[0] = zt;
-    tgt[1] = 1.f;
-  }
-  float m = -INFINITY;
-#pragma unroll
-  for (int it = 0; it < kMaxSteps; ++it) m = fmaxf(m, ref[it]);
+  // ---- block totals: maximum first, one rescale, then a plain sum (fixed order: reproducible)
+  float m = m_run;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-  float sum = 0.f;
-  if (m != -INFINITY) {
-#pragma unroll
-    for (int it = 0; it < kMaxSteps; ++it) sum = fmaf(sums[it], mrl::ex2_approx(ref[it] - m), sum);  // 2^-inf = 0
-  }
+  float sum = m_run != -INFINITY ? s_run * mrl::ex2_approx(m_run - m) : 0.f;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
   if (lane == 0) {
     red[warp] = m;
-    red[kWarps + warp] = sum;
+    red[32 + warp] = sum;
   }
-  const bool any_timeout = __syncthreads_or(timed_out ? 1 : 0) != 0;
-
-  // ---- warp 0: the CTA's triple to every peer, the peers' triples, the row's scalars
+  __syncthreads();
   if (warp == 0) {
-    float wm = lane < kWarps ? red[lane] : -INFINITY;
-    float ws = lane < kWarps ? red[kWarps + lane] : 0.f;
-    float cm = wm;
+    const float wm = lane < kWarpsT ? red[lane] : -INFINITY, ws = lane < kWarpsT ? red[32 + lane] : 0.f;
+    float tm = wm;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, o));
-    float cs = (wm != -INFINITY) ? ws * mrl::ex2_approx(wm - cm) : 0.f;
+    for (int o = 16; o > 0; o >>= 1) tm = fmaxf(tm, __shfl_xor_sync(0xffffffffu, tm, o));
+    float ts = wm != -INFINITY ? ws * mrl::ex2_approx(wm - tm) : 0.f;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) cs += __shfl_xor_sync(0xffffffffu, cs, o);
-    bool wok = !any_timeout;
-    if (C > 1) {
-      cluster_wait();  // every CTA of the cluster has initialised its exchange barrier
+    for (int o = 16; o > 0; o >>= 1) ts += __shfl_xor_sync(0xffffffffu, ts, o);
+    bool ok = true;
+    if (kC > 1) {
+      asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");  // the peer's barrier is initialised
       if (lane == 0) {
-        const float zpart = tgt[0], opart = tgt[1];
-        xchg[rank] = make_float4(cm, cs, zpart, opart);
-        for (int r = 0; r < C; ++r) {
-          if (r == rank) continue;
-          const uint32_t dst = mapa_u32(smem_u32(&xchg[rank]), (uint32_t)r);
-          asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(cm), "f"(cs), "f"(zpart),
-                       "f"(opart)
-                       : "memory");
-          const uint32_t rbar = mapa_u32(smem_u32(&bars[kChunks]), (uint32_t)r);
-          asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(rbar) : "memory");
+        xchg[rank] = make_float4(tm, ts, zt, owner ? 1.f : 0.f);
+        const uint32_t peer = (uint32_t)(rank ^ 1);
+        const uint32_t dst = mapa_u32(smem_u32(&xchg[rank]), peer);
+        asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(tm), "f"(ts), "f"(zt),
+                     "f"(owner ? 1.f : 0.f)
+                     : "memory");
+        asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(mapa_u32(smem_u32(&xbar), peer))
+                     : "memory");
+        bool got = false;
+        for (uint32_t i = 0; i < kExchangeSpinLimit && !got; ++i) got = mbar_try_wait_cluster(&xbar, 0);
+        ok = got;
+        if (got) {  // rank order, so both CTAs form the same sums
+          const float4 a = xchg[0], b = xchg[1];
+          tm = fmaxf(a.x, b.x);
+          ts = (a.x != -INFINITY ? a.y * mrl::ex2_approx(a.x - tm) : 0.f) +
+               (b.x != -INFINITY ? b.y * mrl::ex2_approx(b.x - tm) : 0.f);
+          zt = a.w != 0.f ? a.z : (b.w != 0.f ? b.z : 0.f);
+        } else if (p.status != nullptr) {
+          atomicOr(p.status, MRL_DEV_TIMEOUT);
         }
-      }
-      __syncwarp();
-      bool got = false;
-      for (uint32_t i = 0; i < (kSpinLimit << 2) && !got; ++i) got = mbar_try_wait_cluster(&bars[kChunks], 0);
-      wok = wok && got;
-    } else if (lane == 0) {
-      xchg[0] = make_float4(cm, cs, tgt[0], tgt[1]);
-    }
-    __syncwarp();
-    float4 o = make_float4(-INFINITY, 0.f, 0.f, 0.f);
-    if (lane < C && wok) o = xchg[lane];
-    float tm = o.x;
-#pragma unroll
-    for (int q = 16; q > 0; q >>= 1) tm = fmaxf(tm, __shfl_xor_sync(0xffffffffu, tm, q));
-    float ts = (o.x != -INFINITY) ? o.y * mrl::ex2_approx(o.x - tm) : 0.f;
-    float ztot = o.w != 0.f ? o.z : 0.f;
-#pragma unroll
-    for (int q = 16; q > 0; q >>= 1) {
-      ts += __shfl_xor_sync(0xffffffffu, ts, q);      // xor tree over the ranks: the same order in every CTA
-      ztot += __shfl_xor_sync(0xffffffffu, ztot, q);  // one owner: exact
-    }
-    const float lse2 = tm + log2f(ts);
-    const float lse = lse2 * MRL_LN2;
-    float logp = 0.f, g = 0.f;
-    bool clipped = false;
-    if (ctx.valid && wok) {
-      logp = ztot - lse;
-      if (p.loss_mode) {
-        const mrl::RowOut ro = mrl::mrl_row_loss(logp, ctx.in, p.eps_lo, p.eps_hi);
-        g = ro.g;
-        clipped = ro.clipped;
       }
     }
     if (lane == 0) {
-      if (rank == 0 && wok)
-        write_row_scalars(p, row, ctx, logp, ctx.valid ? lse : 0.f, mrl::Lse2{tm, ts}, ztot, clipped, true);
-      if (!wok && p.status != nullptr) atomicOr(p.status, MRL_DEV_TIMEOUT);
+      const float lse2 = tm + log2f(ts);
+      const float lse = lse2 * MRL_LN2;
+      float logp = 0.f, g = 0.f;
+      bool clipped = false;
+      if (ctx.valid && ok) {
+        logp = zt - lse;
+        if (p.loss_mode) {
+          const mrl::RowOut ro = mrl::mrl_row_loss(logp, ctx.in, p.eps_lo, p.eps_hi);
+          g = ro.g;
+          clipped = ro.clipped;
+        }
+      }
+      if (rank == 0 && ok) write_row_scalars(p, row, ctx, logp, ctx.valid ? lse : 0.f, mrl::Lse2{tm, ts}, zt, clipped, true);
       fin[0] = lse2;
       fin[1] = g;
-      fin[2] = g * (mrl::ex2_approx(fmaf(ztot, MRL_LOG2E, -lse2)) - 1.0f);  // the target column
-      fin[3] = wok ? 1.f : 0.f;
+      fin[2] = g * (mrl::ex2_approx(fmaf(zt, MRL_LOG2E, -lse2)) - 1.0f);
+      fin[3] = ok ? 1.f : 0.f;
     }
-  } else if (C > 1) {
-    cluster_wait();  // pairs with the arrive above (every thread of the cluster takes part)
+  } else if (kC > 1) {
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");  // pairs with the arrive above
   }
   __syncthreads();
+  // After the wait above the peer's remote store and arrive have landed and this CTA's own were issued before:
+  // nobody touches a CTA's shared memory once that CTA can have left.
+  if (!want_grad || fin[3] == 0.f) return;
   const float lse2 = fin[0], g = fin[1], tfix = fin[2];
-  const bool ok = fin[3] != 0.f;
 
-  // ---- pass 2: dlogits slice = g * softmax - g * onehot, from the cached exponentials
-  if (want_grad && ok) {
-    uint4* const out = reinterpret_cast<uint4*>(orow) + tid;  // this thread's output vectors, indexed like `mine`
+  // ---- pass 2: the same vectors again (L2), dlogits = g 2^(z log2e - lse2), the target column patched after
+  if (g == 0.f) {
+    for (int i = tid; i < nvec; i += kT) stream_st<kWords>(out + (size_t)(i - tid) * kVecBytes, stream_fill<kWords>(0u));
+    return;
+  }
+  const float neg_k = -(lse2 - log2f(fabsf(g)));  // 2^(z log2e - k) = |g| softmax(z)
+  const uint32_t sign = g < 0.f ? 0x80008000u : 0u;
+  for (int base = 0; base < nvec; base += kT * kU) {
+    const bool full = base + kT * kU <= nvec;
+    Vec v[kU];
 #pragma unroll
-    for (int it = 0; it < kMaxSteps; ++it) {
-      const int base = it * kStepVecs;
-      if (base < nvec) {
-        const bool full = base + kStepVecs <= nvec;
-        uint4 o[kUnroll];
-        if (g == 0.f) {  // uniform over the row
+    for (int u = 0; u < kU; ++u)
+      v[u] = (full || base + u * kT + tid < nvec) ? stream_ld<kWords, kHintLast>(in + (size_t)(base + u * kT) * kVecBytes)
+                                                  : stream_fill<kWords>(0u);
 #pragma unroll
-          for (int u = 0; u < kUnroll; ++u) o[u] = make_uint4(0, 0, 0, 0);
-        } else {
-          // cached value times scale, as two packed bf16 FMAs: scale = hi + lo, one rounding of the result
-          const float scale = ref[it] != -INFINITY ? g * mrl::ex2_approx(ref[it] - lse2) : 0.f;
-          const float s_hi = __bfloat162float(__float2bfloat16_rn(scale));
-          const uint32_t hi2 = mrl::pack_bf16x2(s_hi, s_hi), lo2 = mrl::pack_bf16x2(scale - s_hi, scale - s_hi);
+    for (int u = 0; u < kU; ++u) {
+      Vec r;
 #pragma unroll
-          for (int u = 0; u < kUnroll; ++u) {
-            const uint4 e = (full || base + u * kThreads + tid < nvec) ? mine[base + u * kThreads] : make_uint4(0, 0, 0, 0);
-            o[u].x = hfma2_u32(e.x, hi2, hfma2_u32(e.x, lo2, 0u));
-            o[u].y = hfma2_u32(e.y, hi2, hfma2_u32(e.y, lo2, 0u));
-            o[u].z = hfma2_u32(e.z, hi2, hfma2_u32(e.z, lo2, 0u));
-            o[u].w = hfma2_u32(e.w, hi2, hfma2_u32(e.w, lo2, 0u));
-          }
-        }
-        if (full) {
-#pragma unroll
-          for (int u = 0; u < kUnroll; ++u) st_global_v4(out + base + u * kThreads, o[u]);
-        } else {
-#pragma unroll
-          for (int u = 0; u < kUnroll; ++u)
-            if (base + u * kThreads + tid < nvec) st_global_v4(out + base + u * kThreads, o[u]);
-        }
-        // the target column gets g (p - 1): a scalar store by the thread whose vector store just covered it, so
-        // the two stores to that address are ordered by program order
-        if (owner_step == it && g != 0.f) orow[rel] = __float2bfloat16_rn(tfix);
+      for (int j = 0; j < kWords; ++j) {
+        const float a = mrl::ex2_approx(fmaf(mrl::bf16lo_to_f32(v[u].w[j]), MRL_LOG2E, neg_k));
+        const float b = mrl::ex2_approx(fmaf(mrl::bf16hi_to_f32(v[u].w[j]), MRL_LOG2E, neg_k));
+        r.w[j] = mrl::pack_bf16x2(a, b) ^ sign;
       }
+      if (full || base + u * kT + tid < nvec) stream_st<kWords>(out + (size_t)(base + u * kT) * kVecBytes, r);
     }
   }
-  // Every peer's remote store and arrive has landed before warp 0 got past its wait, and this CTA's own remote
-  // accesses were issued before it: nobody touches a CTA's shared memory after that CTA can have left.
+  // the thread whose vector store covered the target column patches it (program order on one address)
+  if (owner && tid == (rel / kVecElems) % kT) orow[rel] = __float2bfloat16_rn(tfix);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -699,41 +593,40 @@ MrlLossWs carve_loss_ws(void* ws, long long N, int S) {
   return w;
 }
 
-// Picks the fast path when its alignment rules hold; returns the cluster size (0 = general kernel).
-int pick_cluster(const RowParams& p, int dtype) {
+// Which kernel takes the rows: 0 = general, 4 = streaming with 128-bit accesses, 8 = with 256-bit accesses.
+int pick_stream_words(const RowParams& p, int dtype) {
   if (dtype != MRL_BF16) return 0;
-  if (p.V % 8 != 0 || p.ld % 8 != 0) return 0;
-  if ((reinterpret_cast<uintptr_t>(p.logits) & 15) != 0) return 0;
-  if (p.dlogits != nullptr && (p.ld_out % 8 != 0 || (reinterpret_cast<uintptr_t>(p.dlogits) & 15) != 0)) return 0;
   if (p.V < 4096) return 0;  // short rows: the general kernel's three passes stay in cache
-  int C = 1;
-  while ((long long)p.V * 2 > (long long)C * kMaxPartBytes) C *= 2;
-  return C <= kMaxCluster ? C : 0;
+  const uintptr_t in = reinterpret_cast<uintptr_t>(p.logits), out = reinterpret_cast<uintptr_t>(p.dlogits);
+  const bool grad = p.dlogits != nullptr;
+  if (p.V % 16 == 0 && p.ld % 16 == 0 && (in & 31) == 0 && (!grad || (p.ld_out % 16 == 0 && (out & 31) == 0))) return 8;
+  if (p.V % 8 == 0 && p.ld % 8 == 0 && (in & 15) == 0 && (!grad || (p.ld_out % 8 == 0 && (out & 15) == 0))) return 4;
+  return 0;
 }
 
 int launch_rows(RowParams p, int dtype, cudaStream_t st) {
   if (p.N == 0) return MRL_OK;
-  if (p.N > 0x7fffffffll / kMaxCluster) return MRL_ERR_UNSUPPORTED_SHAPE;
-  const int C = pick_cluster(p, dtype);
-  if (C == 0) {
+  if (p.N > 0x7fffffffll) return MRL_ERR_UNSUPPORTED_SHAPE;
+  const int words = pick_stream_words(p, dtype);
+  const unsigned n = (unsigned)p.N;
+  if (words == 0) {
     mrl_profile_before(st);
     if (dtype == MRL_BF16)
-      row_general_kernel<__nv_bfloat16><<<(unsigned)p.N, kThreads, 0, st>>>(p);
+      row_general_kernel<__nv_bfloat16><<<n, kThreads, 0, st>>>(p);
     else
-      row_general_kernel<float><<<(unsigned)p.N, kThreads, 0, st>>>(p);
+      row_general_kernel<float><<<n, kThreads, 0, st>>>(p);
     mrl_profile_after(st);
     return cudaGetLastError() == cudaSuccess ? MRL_OK : MRL_ERR_CUDA;
   }
-  const int vecs = (p.V / 8 + C - 1) / C;
-  p.part_elems = vecs * 8;
-  p.cluster = C;
-  const size_t smem = (size_t)p.part_elems * 2 + kTailBytes;
-  // per device and idempotent; set on every call so that a change of the current device is harmless
-  MRL_CUDA_OK(cudaFuncSetAttribute(row_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+  // Two CTAs per SM stream one row each, or -- for rows so long that two rows per SM would be evicted from L2
+  // before the second pass reads them back -- the two halves of one row as a cluster of two.  (At 300 KB rows the
+  // split reads HBM 1.01x instead of 1.34x but is 4 % slower: its per-CTA fixed work is spread over half the bytes.)
+  const bool split = (long long)p.V * 2 >= kSplitRowBytes && p.N <= 0x3fffffffll;
+  const int C = split ? 2 : 1;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(p.N * C));
-  cfg.blockDim = dim3(kThreads);
-  cfg.dynamicSmemBytes = smem;
+  cfg.gridDim = dim3(n * (unsigned)C);
+  cfg.blockDim = dim3(kStreamThreads);
+  cfg.dynamicSmemBytes = 0;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -743,9 +636,15 @@ int launch_rows(RowParams p, int dtype, cudaStream_t st) {
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   mrl_profile_before(st);
-  MRL_CUDA_OK(cudaLaunchKernelEx(&cfg, row_cluster_kernel, p));
+  cudaError_t e;
+  if (words == 8)
+    e = split ? cudaLaunchKernelEx(&cfg, row_stream_kernel<kStreamThreads, 4, 8, 2>, p)
+              : cudaLaunchKernelEx(&cfg, row_stream_kernel<kStreamThreads, 4, 8, 1>, p);
+  else
+    e = split ? cudaLaunchKernelEx(&cfg, row_stream_kernel<kStreamThreads, 8, 4, 2>, p)
+              : cudaLaunchKernelEx(&cfg, row_stream_kernel<kStreamThreads, 8, 4, 1>, p);
   mrl_profile_after(st);
-  return MRL_OK;
+  return e == cudaSuccess ? MRL_OK : MRL_ERR_CUDA;
 }
 
 bool dtype_ok(int dtype) { return dtype == MRL_BF16 || dtype == MRL_F32; }

@@ -91,10 +91,12 @@ def test_sgt_gate_is_bit_exact(pick, P, M, G, learner):
 @pytest.mark.parametrize("N,V,dtype,pad", [
     (1024, 1024, torch.float32, 0),      # config 1 shape
     (7, 1, torch.float32, 0), (5, 3, torch.bfloat16, 0), (9, 1000, torch.bfloat16, 3),   # general kernel
-    (37, 4096, torch.bfloat16, 0), (19, 4104, torch.bfloat16, 8),                         # cluster of 1
-    (11, 40008, torch.bfloat16, 0),                                                       # cluster of 2
-    (9, 100008, torch.bfloat16, 0), (6, 151936, torch.bfloat16, 0), (5, 128256, torch.bfloat16, 0),  # 4
-    (3, 200008, torch.bfloat16, 0),                                                       # cluster of 8
+    (37, 4096, torch.bfloat16, 0), (19, 4104, torch.bfloat16, 8),                         # 256-bit path, one step; 128-bit path with a padded row
+    (11, 40008, torch.bfloat16, 0),                                                       # 128-bit path, ragged last step
+    (9, 100008, torch.bfloat16, 0), (6, 151936, torch.bfloat16, 0), (5, 128256, torch.bfloat16, 0),
+    (13, 8208, torch.bfloat16, 0), (4, 65552, torch.bfloat16, 16),                        # 256-bit path, ragged last step
+    (3, 262160, torch.bfloat16, 0), (2, 300008, torch.bfloat16, 0),                       # rows split over a cluster of two CTAs
+    (3, 200008, torch.bfloat16, 0),                                                       # long row, 128-bit path
 ])
 def test_token_logprobs(N, V, dtype, pad):
     z, ids, _, _, _, _, g = toy_inputs(N, V, 1, dtype, seed=N + V, pad=pad)
@@ -145,6 +147,10 @@ CASES = [
     (12, 151936, 3, torch.bfloat16, 0, 0.9),
     (7, 128256, 2, torch.bfloat16, 0, None),
     (3, 200008, 1, torch.bfloat16, 0, None),
+    (17, 8208, 3, torch.bfloat16, 0, 0.8),      # 256-bit accesses, ragged last step
+    (5, 65552, 2, torch.bfloat16, 16, None),    # 256-bit accesses, padded rows
+    (4, 262160, 2, torch.bfloat16, 0, None),    # row split over a cluster of two CTAs, 256-bit accesses
+    (3, 262152, 1, torch.bfloat16, 0, 0.7),     # the same with 128-bit accesses and a masked row
 ]
 
 
@@ -386,7 +392,7 @@ def test_config4_twin_xgrpo_baseline_with_sgt_rows():
 
 def test_config2_full_size_sampled_rows():
     """Config 2 at full size, in the launch configuration the benchmark times (packed rows, bf16,
-    V = 151,936, cluster kernel): the oracle checks every scalar and gradient row of a seeded row
+    V = 151,936, streaming kernel): the oracle checks every scalar and gradient row of a seeded row
     sample; the loss is checked through a size-independent property (rho = 1 gives minus the
     token-weighted mean advantage, computed from the oracle's advantages)."""
     w = synth.C2

@@ -64,7 +64,7 @@ def _run(entry, inp, workspace):
 
 @pytest.mark.gpu
 def test_static_scratch_variant_matches_the_workspace_variant_on_two_calls_in_a_row():
-    # first a larger problem whose rows span a four-CTA cluster, then a smaller, differently cut one:
+    # first a larger problem with full-vocabulary rows, then a smaller, differently cut one:
     # the second call finds the first call's per-row scratch still in the array
     shapes = [(300, 151936, 7, True), (97, 32768, 3, False)]
     for k, (N, V, S, with_mask) in enumerate(shapes):
