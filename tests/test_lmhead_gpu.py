@@ -197,3 +197,112 @@ def test_config5_reduced_twin():
         compare(got, ref, check_grads=False)
     else:
         compare(got, ref)
+
+
+# ------------------------------------------------------------------ config 5 at full size
+
+def _c5_device_inputs(seed):
+    """Config 5's hidden states and LM-head weight drawn on the device (the generator is seeded per block, so the
+    same bits come out on either device type); returns the packed batch description as well."""
+    w = synth.C5
+    meta = synth.make_meta(w, seed)
+    batch = synth.make_batch(meta)
+    hidden = torch.empty(batch.N, w.H, dtype=w.dtype, device="cuda")
+    for a in range(0, batch.N, w.rows_per_block):
+        e = min(batch.N, a + w.rows_per_block)
+        hidden[a:e] = batch.hidden_rows(a, e, device="cuda")
+    W = batch.lm_head(device="cuda")
+    adv, _ = O.group_advantages(meta.rewards)
+    adv_seq = adv[batch.seq_p.long(), batch.seq_m.long(), batch.seq_g.long()].float()
+    return w, batch, hidden, W, adv_seq
+
+
+def _call_lmhead_on_device(hidden, W, ids, mask, cu, adv_seq, logp_old, lp):
+    N, H = hidden.shape
+    V = W.shape[0]
+    S = cu.numel() - 1
+    ws = torch.empty(B.workspace_bytes(B.WS_FUSED_LMHEAD, N, V, H, B.BF16, S), dtype=torch.uint8, device="cuda")
+    out = dict(dH=torch.full((N, H), float("nan"), dtype=torch.bfloat16, device="cuda"),
+               dW=torch.full((V, H), float("nan"), dtype=torch.bfloat16, device="cuda"),
+               logp=torch.full((N,), float("nan"), device="cuda"), loss=torch.full((2,), float("nan"), device="cuda"),
+               stats=torch.full((4,), -1, dtype=torch.int64, device="cuda"),
+               status=torch.zeros(1, dtype=torch.int32, device="cuda"))
+    B.mrl_fused_lmhead_loss_fwd_bwd(hidden, W, dev(ids, torch.int32), dev(mask, torch.uint8), dev(cu, torch.int32),
+                                    dev(adv_seq, torch.float32), dev(logp_old, torch.float32), None, None, lp,
+                                    out["dH"], out["dW"], out["logp"], out["loss"], out["stats"], out["status"], ws)
+    torch.cuda.synchronize()
+    del ws
+    return out
+
+
+def test_config5_full_size_with_a_sparse_mask_is_checked_in_full():
+    """N = 65,536, H = 4,096, V = 151,936 as the benchmark launches it, with all but 192 rows masked: every output
+    then depends on those rows only, which the oracle can afford in float64 -- loss, log-probs, the 192 dHidden
+    rows and the whole of dW are compared; masked rows must come out exactly zero."""
+    w, batch, hidden, W, adv_seq = _c5_device_inputs(seed=11)
+    N, V, H = batch.N, w.V, w.H
+    g = torch.Generator().manual_seed(5)
+    keep = torch.sort(torch.randperm(N, generator=g)[:192]).values
+    mask = torch.zeros(N, dtype=torch.uint8)
+    mask[keep] = 1
+    # the oracle's view: the kept rows as a packed batch of their own (same sequences, same advantages)
+    seq_of_row = torch.repeat_interleave(torch.arange(batch.S), (batch.cu_seqlens[1:] - batch.cu_seqlens[:-1]).long())
+    counts = torch.bincount(seq_of_row[keep], minlength=batch.S)
+    sub_cu = torch.zeros(batch.S + 1, dtype=torch.int32)
+    sub_cu[1:] = torch.cumsum(counts, 0)
+    h_sub, W_cpu, ids_sub = hidden[keep.cuda()].cpu(), W.cpu(), batch.ids[keep]
+    z_sub = h_sub.double() @ W_cpu.double().T
+    logp_sub, _, _ = O.token_logprobs(z_sub, ids_sub)
+    del z_sub
+    old_sub = (logp_sub + batch.noise[keep].double()).float()
+    logp_old = torch.zeros(N)
+    logp_old[keep] = old_sub
+    lp = make_lp()
+    got = _call_lmhead_on_device(hidden, W, batch.ids, mask, batch.cu_seqlens, adv_seq, logp_old, lp)
+    ref = O.fused_lmhead_loss(h_sub, W_cpu, ids_sub, None, sub_cu, adv_seq, old_sub, None, None, oracle_lp(lp))
+    assert int(got["status"].cpu()) == 0
+    assert int(got["stats"].cpu()[0]) == 192
+    logp = got["logp"].cpu()
+    assert (logp[keep].double() - ref["logp"]).abs().max() <= LOGP_ATOL
+    assert float(logp[mask == 0].abs().max()) == 0
+    L = ref["loss_pg"]
+    scale = max(abs(L), 0.1 * float(ref["pg_term"].abs().sum()))
+    assert abs(float(got["loss"].cpu()[0]) - L) <= LOSS_RTOL * scale
+    tie = ref["margin"] < TIE_MARGIN
+    assert not tie.any(), "a kept row sits on the clip boundary: change the seed"
+    dH = got["dH"].cpu()
+    assert float(dH[mask == 0].float().abs().max()) == 0
+    assert rel_l2(dH[keep], ref["dHidden"]) <= GRAD_REL_L2_BF16
+    assert rel_l2(got["dW"].cpu(), ref["dW"]) <= GRAD_REL_L2_BF16
+
+
+def test_config5_full_size_unmasked_sampled_rows_and_invariants():
+    """The same launch with every row live and ratio one (no behaviour trace): the loss has the closed form
+    -mean A; log-probs and dHidden are checked on 48 sampled rows the oracle evaluates one by one (g_t = A_t / N
+    needs nothing from other rows); dz rows sum to zero, so the columns of dW must sum to ~0."""
+    w, batch, hidden, W, adv_seq = _c5_device_inputs(seed=12)
+    N, V, H = batch.N, w.V, w.H
+    lp = make_lp()
+    got = _call_lmhead_on_device(hidden, W, batch.ids, None, batch.cu_seqlens, adv_seq, None, lp)
+    assert int(got["status"].cpu()) == 0 and int(got["stats"].cpu()[0]) == N
+    lens = (batch.cu_seqlens[1:] - batch.cu_seqlens[:-1]).double()
+    want_loss = -float((adv_seq.double() * lens).sum() / lens.sum())
+    terms = float((adv_seq.double().abs() * lens).sum() / lens.sum())
+    assert abs(float(got["loss"].cpu()[0]) - want_loss) <= LOSS_RTOL * max(abs(want_loss), 0.1 * terms)
+    g = torch.Generator().manual_seed(6)
+    rows = torch.sort(torch.randperm(N, generator=g)[:48]).values
+    seq_of_row = torch.repeat_interleave(torch.arange(batch.S), lens.long())
+    W64 = W.cpu().double()
+    z = hidden[rows.cuda()].cpu().double() @ W64.T
+    logp, lse, _ = O.token_logprobs(z, batch.ids[rows])
+    assert (got["logp"].cpu()[rows].double() - logp).abs().max() <= LOGP_ATOL
+    gt = adv_seq.double()[seq_of_row[rows]] / N                       # rho = 1, token mean over all N rows
+    dz = torch.exp(z - lse[:, None])
+    dz[torch.arange(48), batch.ids[rows].long()] -= 1.0
+    dz *= gt[:, None]
+    want_dH = dz @ W64
+    assert rel_l2(got["dH"].cpu()[rows], want_dH) <= GRAD_REL_L2_BF16
+    dW = got["dW"].cpu().double()
+    assert torch.isfinite(dW).all()
+    col, mag = dW.sum(dim=0), dW.abs().sum(dim=0)
+    assert (col.abs() <= 2e-2 * mag + 1e-12).all()
