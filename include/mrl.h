@@ -81,6 +81,9 @@ extern "C" {
                                          logits (A = 0 or weight 0, and no NLL weight) are not read: logp = 0,
                                          dlogits row = 0, they still count in the denominators */
 #define MRL_FLAG_ACCUMULATE_DW 4u     /* fused LM head: dW is float32 [V, H] and is added to, not overwritten */
+#define MRL_FLAG_PAIR_TILES 8u        /* fused LM head: 256-row tiles worked by pairs of CTAs (tcgen05 cta_group::2).
+                                         Same results.  Faster for a product timed alone; inside a long
+                                         power-capped step the default 128-row tiles were faster on B200 */
 
 /* `which` of mrl_workspace_bytes */
 #define MRL_WS_TOKEN_LOGPROBS 0

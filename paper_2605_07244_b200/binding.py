@@ -17,7 +17,7 @@ F32, BF16 = 0, 1
 ADV_MEAN_ONLY, ADV_GROUP_ZNORM, ADV_BATCH_ZNORM = 0, 1, 2
 PICK_NONE, PICK_FIRST, PICK_SHORTEST, PICK_ALL, PICK_SEEDED = 0, 1, 2, 3, 4
 AGG_TOKEN_MEAN, AGG_SEQ_MEAN_TOKEN_MEAN = 0, 1
-FLAG_ACCUMULATE_LOSS, FLAG_SKIP_ZERO_ROWS, FLAG_ACCUMULATE_DW = 1, 2, 4
+FLAG_ACCUMULATE_LOSS, FLAG_SKIP_ZERO_ROWS, FLAG_ACCUMULATE_DW, FLAG_PAIR_TILES = 1, 2, 4, 8
 WS_TOKEN_LOGPROBS, WS_POLICY_LOSS, WS_FUSED_LMHEAD = 0, 1, 2
 DEV_BAD_TOKEN_ID, DEV_TIMEOUT = 1, 2
 

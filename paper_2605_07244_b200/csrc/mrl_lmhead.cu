@@ -19,15 +19,20 @@ namespace {
 
 constexpr int BM = 128, BN = 256, BK = 64;  // CTA tile; BK * 2 bytes = one 128-byte swizzle row
 constexpr int UMMA_K = 16;
-constexpr int kStages = 4;
 constexpr int kAccStages = 2;
 constexpr int kTmemCols = kAccStages * BN;  // 512: all of tensor memory
 constexpr int kGemmThreads = 192;
-constexpr uint32_t kABytes = BM * BK * 2, kBBytes = BN * BK * 2, kStageBytes = kABytes + kBBytes;
-constexpr size_t kGemmSmem = (size_t)kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr uint32_t kABytes = BM * BK * 2;  // a CTA's A tile of one stage
+// kC CTAs share a tile of kC * 128 rows: each holds its own 128 rows of A and 256 / kC rows of B per stage
+template <int kC>
+struct GemmCfg {
+  static constexpr int kBRows = BN / kC;
+  static constexpr uint32_t kBBytes = kBRows * BK * 2, kStageBytes = kABytes + kBBytes;
+  static constexpr int kStages = kC == 2 ? 6 : 4;  // 192 KB of stages either way
+  static constexpr size_t kSmem = (size_t)kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
 constexpr uint32_t kWaitLimit = 1u << 24;   // mbarrier polls before a wait gives up (of the order of a second)
 constexpr int kVChunk = 16384;              // vocabulary columns per backward chunk (multiple of BN)
-constexpr int kGroupM = 16;                 // row-tiles per raster group (operand reuse through L2)
 
 enum { EPI_LSE = 0, EPI_DZ = 1, EPI_STORE = 2 };
 enum { C_BF16 = 0, C_F32 = 1, C_F32_ADD = 2, C_BF16_FROM_ACC = 3 };
@@ -35,6 +40,7 @@ enum { C_BF16 = 0, C_F32 = 1, C_F32_ADD = 2, C_BF16_FROM_ACC = 3 };
 struct GemmParams {
   int M, N, K;
   int m_tiles, n_tiles, k_blocks;
+  int group_m;            // row-tiles per raster group
   int32_t* status;
   // EPI_LSE
   float2* partial;        // [n_tiles][part_ld]: (running max, sum) of the tile's columns, base-2 domain
@@ -94,6 +100,42 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
       : "memory");
 }
+__device__ __forceinline__ uint32_t mapa_u32(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+// arrive on an mbarrier of another CTA of the cluster (address from mapa)
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA tile load of a CTA pair: the bytes land in this CTA, the completion is counted on `bar`, which may live in
+// the other CTA of the pair (a shared::cluster address)
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+// commit of a CTA pair's MMAs: one arrival on the barrier at this offset in every CTA of `mask`
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar, uint16_t mask) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(mask)
+               : "memory");
+}
+// D[tmem of both CTAs] (+)= A * B^T, one 256 x 256 x 16 step of a CTA pair (issued by the leader CTA)
+__device__ __forceinline__ void tc_mma_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accum) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accum)
+      : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -135,16 +177,18 @@ __device__ __forceinline__ uint64_t smem_desc_k128(uint32_t addr) {
   d |= (uint64_t)2 << 61;                    // SWIZZLE_128B
   return d;
 }
-// kind::f16 instruction descriptor: fp32 accumulator, bf16 x bf16, both K-major, N = 256, M = 128
-constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+// kind::f16 instruction descriptor: fp32 accumulator, bf16 x bf16, both K-major, N = 256, M = 128 per CTA
+template <int kC>
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) |
+                            ((uint32_t)((BM * kC) >> 4) << 24);
 
-// tile t -> (row-tile, column-tile): row-tiles run fastest inside a group of kGroupM, so that the CTAs of one wave
+// tile t -> (row-tile, column-tile): row-tiles run fastest inside a group of group_m, so that the CTAs of one wave
 // share a handful of A and B tiles
-__device__ __forceinline__ void tile_coords(int t, int m_tiles, int n_tiles, int& m, int& n) {
-  const int per_group = kGroupM * n_tiles;
+__device__ __forceinline__ void tile_coords(int t, int m_tiles, int n_tiles, int group_m, int& m, int& n) {
+  const int per_group = group_m * n_tiles;
   const int grp = t / per_group, r = t - grp * per_group;
-  const int m0 = grp * kGroupM;
-  const int gm = min(kGroupM, m_tiles - m0);
+  const int m0 = grp * group_m;
+  const int gm = min(group_m, m_tiles - m0);
   n = r / gm;
   m = m0 + (r - n * gm);
 }
@@ -200,10 +244,13 @@ __device__ __forceinline__ void store_bf16x32(__nv_bfloat16* dst, const float* d
 }
 
 // ------------------------------------------------------------------------------------------ the GEMM kernel
-template <int EPI>
+template <int EPI, int kC>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
                    const GemmParams p) {
+  using Cfg = GemmCfg<kC>;
+  constexpr int kStages = Cfg::kStages;
+  constexpr uint32_t kStageBytes = Cfg::kStageBytes;
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_addr(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;  // swizzled tiles need 1024-byte alignment
@@ -219,6 +266,9 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // a pair of CTAs (kC = 2) works on one tile of 256 rows: rank 0 leads (arms the barriers, issues the MMAs)
+  const int rank = kC == 2 ? (int)(blockIdx.x & 1u) : 0;
+  const int unit = (int)blockIdx.x / kC, n_units = (int)gridDim.x / kC;
   const int total_tiles = p.m_tiles * p.n_tiles;
 
   if (threadIdx.x == 0) {
@@ -228,49 +278,66 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
     }
     for (int a = 0; a < kAccStages; ++a) {
       mbar_init(tfull_bar(a), 1);
-      mbar_init(tempty_bar(a), 4);  // one arrival per epilogue warp
+      mbar_init(tempty_bar(a), 4 * kC);  // one arrival per epilogue warp of every CTA of the pair
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(tmem_slot)),
-                 "r"((uint32_t)kTmemCols)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  if (warp == 1) {  // the same warp in both CTAs of a pair, the same shared-memory slot
+    if (kC == 2) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(tmem_slot)),
+                   "r"((uint32_t)kTmemCols)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(tmem_slot)),
+                   "r"((uint32_t)kTmemCols)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if (kC == 2) cluster_sync_all();  // the peer's barriers exist before anything is signalled across the pair
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 0) {
-    // ---------------- TMA producer
+    // ---------------- TMA producer: this CTA's 128 rows of A and its 256 / kC rows of B
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+      for (int t = unit; t < total_tiles && ok; t += n_units) {
         int m, n;
-        tile_coords(t, p.m_tiles, p.n_tiles, m, n);
+        tile_coords(t, p.m_tiles, p.n_tiles, p.group_m, m, n);
+        const int a_row = (m * kC + rank) * BM, b_row = n * BN + rank * Cfg::kBRows;
         for (int kb = 0; kb < p.k_blocks; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t a_dst = tiles + (uint32_t)stage * kStageBytes;
-          mbar_expect_tx(full_bar(stage), kStageBytes);
-          tma_load_2d(a_dst, &tmapA, kb * BK, m * BM, full_bar(stage));
-          tma_load_2d(a_dst + kABytes, &tmapB, kb * BK, n * BN, full_bar(stage));
+          if (kC == 2) {
+            // the leader's barrier counts the bytes of both CTAs; only the leader arms it
+            const uint32_t lead_full = mapa_u32(full_bar(stage), 0u);
+            if (rank == 0) mbar_expect_tx(full_bar(stage), 2u * kStageBytes);
+            tma_load_2d_pair(a_dst, &tmapA, kb * BK, a_row, lead_full);
+            tma_load_2d_pair(a_dst + kABytes, &tmapB, kb * BK, b_row, lead_full);
+          } else {
+            mbar_expect_tx(full_bar(stage), kStageBytes);
+            tma_load_2d(a_dst, &tmapA, kb * BK, a_row, full_bar(stage));
+            tma_load_2d(a_dst + kABytes, &tmapB, kb * BK, b_row, full_bar(stage));
+          }
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
     }
   } else if (warp == 1) {
-    // ---------------- MMA issuer
-    if (lane == 0) {
+    // ---------------- MMA issuer (the leader CTA of a pair)
+    if (lane == 0 && rank == 0) {
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
-      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+      for (int t = unit; t < total_tiles && ok; t += n_units) {
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)acc * BN;
@@ -280,13 +347,18 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
           const uint32_t a_src = tiles + (uint32_t)stage * kStageBytes;
           const uint64_t adesc = smem_desc_k128(a_src), bdesc = smem_desc_k128(a_src + kABytes);
 #pragma unroll
-          for (int k = 0; k < BK / UMMA_K; ++k)  // 32 bytes along K inside the swizzle row: +2 in 16-byte units
-            tc_mma(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), kIdesc, (kb | k) != 0);
-          tc_commit(empty_bar(stage));  // the stage is free once these MMAs have read it
+          for (int k = 0; k < BK / UMMA_K; ++k) {  // 32 bytes along K inside the swizzle row: +2 in 16-byte units
+            if (kC == 2)
+              tc_mma_pair(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), kIdesc<kC>, (kb | k) != 0);
+            else
+              tc_mma(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), kIdesc<kC>, (kb | k) != 0);
+          }
+          // the stage is free (in both CTAs) once these MMAs have read it
+          if (kC == 2) tc_commit_pair(empty_bar(stage), 3); else tc_commit(empty_bar(stage));
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
-        tc_commit(tfull_bar(acc));
+        if (kC == 2) tc_commit_pair(tfull_bar(acc), 3); else tc_commit(tfull_bar(acc));
         if (++acc == kAccStages) { acc = 0; acc_phase ^= 1u; }
       }
     }
@@ -297,10 +369,10 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
-    for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+    for (int t = unit; t < total_tiles && ok; t += n_units) {
       int m, n;
-      tile_coords(t, p.m_tiles, p.n_tiles, m, n);
-      const int row = m * BM + row_in_tile;
+      tile_coords(t, p.m_tiles, p.n_tiles, p.group_m, m, n);
+      const int row = (m * kC + rank) * BM + row_in_tile;
       const bool row_ok = row < p.M;
       const int ncols_valid = min(BN, p.N - n * BN);
       // per-row inputs before the accumulator is ready
@@ -357,16 +429,42 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
               store_bf16x32(static_cast<__nv_bfloat16*>(p.C) + (long long)row * p.ldc + col, v, nvalid);
             } else if (p.c_mode == C_BF16_FROM_ACC) {
               const float* a = p.Cacc + (long long)row * p.ldacc + col;
+              if (nvalid >= 32 && (reinterpret_cast<uintptr_t>(a) & 15) == 0) {
 #pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (j < nvalid) v[j] += a[j];
+                for (int q = 0; q < 8; ++q) {
+                  const float4 t = reinterpret_cast<const float4*>(a)[q];
+                  v[4 * q + 0] += t.x;
+                  v[4 * q + 1] += t.y;
+                  v[4 * q + 2] += t.z;
+                  v[4 * q + 3] += t.w;
+                }
+              } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j)
+                  if (j < nvalid) v[j] += a[j];
+              }
               store_bf16x32(static_cast<__nv_bfloat16*>(p.C) + (long long)row * p.ldc + col, v, nvalid);
             } else {
               float* o = static_cast<float*>(p.C) + (long long)row * p.ldc + col;
               const bool add = p.c_mode == C_F32_ADD;
+              if (nvalid >= 32 && (reinterpret_cast<uintptr_t>(o) & 15) == 0) {
 #pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (j < nvalid) o[j] = add ? o[j] + v[j] : v[j];
+                for (int q = 0; q < 8; ++q) {
+                  float4 t = make_float4(v[4 * q + 0], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+                  if (add) {
+                    const float4 r = reinterpret_cast<const float4*>(o)[q];
+                    t.x += r.x;
+                    t.y += r.y;
+                    t.z += r.z;
+                    t.w += r.w;
+                  }
+                  reinterpret_cast<float4*>(o)[q] = t;
+                }
+              } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j)
+                  if (j < nvalid) o[j] = add ? o[j] + v[j] : v[j];
+              }
             }
           }
         }
@@ -374,7 +472,9 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
       // the accumulator has been read: hand it back to the MMA warp
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(tempty_bar(acc));
+      if (lane == 0) {  // the leader's barrier collects the epilogue warps of both CTAs
+        if (kC == 2 && rank != 0) mbar_arrive_remote(mapa_u32(tempty_bar(acc), 0u)); else mbar_arrive(tempty_bar(acc));
+      }
       if (EPI == EPI_LSE && row_ok) {
         p.partial[(long long)n * p.part_ld + row] = make_float2(st.m, st.s);
         if (st.has) p.zt[row] = st.zt;
@@ -392,10 +492,15 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
     for (int i = 0; i < 2000; ++i) __nanosleep(1000);  // let copies and MMAs still in flight land before the CTA goes
     __syncthreads();
   }
+  if (kC == 2) cluster_sync_all();  // no CTA leaves while its peer may still signal into its shared memory
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols)
-                 : "memory");
+    if (kC == 2)
+      asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols)
+                   : "memory");
+    else
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols)
+                   : "memory");
   }
 }
 
@@ -509,24 +614,69 @@ int sm_count() {
   return n[dev];
 }
 
+// CTA pairs of the two-CTA kernel that can be resident together on the current device (0: use single CTAs).
 template <int EPI>
-int launch_gemm(const void* A, long long lda, const void* B, long long ldb, GemmParams p, cudaStream_t st) {
+int resident_pairs(cudaLaunchConfig_t* cfg) {
+  static int cache[64] = {};
+  int dev = 0;
+  const bool cacheable = cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64;
+  if (cacheable && cache[dev] != 0) return cache[dev] > 0 ? cache[dev] : 0;
+  cfg->gridDim = dim3((unsigned)(sm_count() / 2 * 2));
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, lmhead_gemm_kernel<EPI, 2>, cfg) != cudaSuccess || n < 1) {
+    (void)cudaGetLastError();
+    n = 0;
+  }
+  if (cacheable) cache[dev] = n > 0 ? n : -1;
+  return n;
+}
+
+template <int EPI>
+int launch_gemm(const void* A, long long lda, const void* B, long long ldb, GemmParams p, bool pair_tiles,
+                cudaStream_t st) {
   if (p.M <= 0 || p.N <= 0 || p.K <= 0) return MRL_OK;
+  p.n_tiles = (p.N + BN - 1) / BN;
+  p.k_blocks = (p.K + BK - 1) / BK;
+  // two-CTA tiles (256 rows) when asked for and pairs can be scheduled, else one CTA per 128-row tile
+  MRL_CUDA_OK(cudaFuncSetAttribute(lmhead_gemm_kernel<EPI, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)GemmCfg<2>::kSmem));
+  cudaLaunchConfig_t cfg = {};
+  cfg.blockDim = dim3(kGemmThreads);
+  cfg.dynamicSmemBytes = GemmCfg<2>::kSmem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const int pairs = pair_tiles ? resident_pairs<EPI>(&cfg) : 0;
+  const int kC = pairs > 0 ? 2 : 1;
   CUtensorMap ta, tb;
   int rc = make_tmap(&ta, A, p.M, p.K, lda, BM);
   if (rc != MRL_OK) return rc;
-  rc = make_tmap(&tb, B, p.N, p.K, ldb, BN);
+  rc = make_tmap(&tb, B, p.N, p.K, ldb, BN / kC);
   if (rc != MRL_OK) return rc;
-  p.m_tiles = (p.M + BM - 1) / BM;
-  p.n_tiles = (p.N + BN - 1) / BN;
-  p.k_blocks = (p.K + BK - 1) / BK;
+  p.m_tiles = (p.M + BM * kC - 1) / (BM * kC);
+  // rows of A per raster group: a wave's operands should share L2; with a short K a taller group re-uses A
+  // across the next waves as well (measured: 4,096 rows at K = 4,096, 2,048 rows at K >= 16,384)
+  p.group_m = (kC == 2 && p.K <= 8192 ? 4096 : 2048) / (BM * kC);
   const long long tiles = (long long)p.m_tiles * p.n_tiles;
   if (tiles > 0x7fffffffll) return MRL_ERR_UNSUPPORTED_SHAPE;
+  if (kC == 2) {
+    const long long units = tiles < pairs ? tiles : pairs;
+    cfg.gridDim = dim3((unsigned)(2 * units));
+    mrl_profile_before(st);
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, lmhead_gemm_kernel<EPI, 2>, ta, tb, p);
+    mrl_profile_after(st);
+    return e == cudaSuccess ? MRL_OK : MRL_ERR_CUDA;
+  }
   const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
-  MRL_CUDA_OK(cudaFuncSetAttribute(lmhead_gemm_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   (int)kGemmSmem));
+  MRL_CUDA_OK(cudaFuncSetAttribute(lmhead_gemm_kernel<EPI, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)GemmCfg<1>::kSmem));
   mrl_profile_before(st);
-  lmhead_gemm_kernel<EPI><<<grid, kGemmThreads, kGemmSmem, st>>>(ta, tb, p);
+  lmhead_gemm_kernel<EPI, 1><<<grid, kGemmThreads, GemmCfg<1>::kSmem, st>>>(ta, tb, p);
   mrl_profile_after(st);
   MRL_CUDA_OK(cudaGetLastError());
   return MRL_OK;
@@ -590,7 +740,8 @@ size_t mrl_fused_lmhead_workspace_bytes(long long N, int V, int H, int S) {
 // C[M, N] = A[M, K] B[N, K]^T with a plain store (bf16 or fp32, optionally added to): the building block of the
 // two backward products, also reachable on its own for checks of the tensor-core mainloop.
 int mrl_lmhead_gemm_tn(const void* A, long long lda, const void* B, long long ldb, int M, int N, int K, void* C,
-                       long long ldc, int c_mode, float* Cacc, long long ldacc, int32_t* status, cudaStream_t st) {
+                       long long ldc, int c_mode, float* Cacc, long long ldacc, int32_t* status, bool pair_tiles,
+                       cudaStream_t st) {
   GemmParams p = {};
   p.M = M;
   p.N = N;
@@ -601,7 +752,7 @@ int mrl_lmhead_gemm_tn(const void* A, long long lda, const void* B, long long ld
   p.Cacc = Cacc;
   p.ldacc = ldacc;
   p.status = status;
-  return launch_gemm<EPI_STORE>(A, lda, B, ldb, p, st);
+  return launch_gemm<EPI_STORE>(A, lda, B, ldb, p, pair_tiles, st);
 }
 
 extern "C" int mrl_fused_lmhead_loss_fwd_bwd(const void* hidden, const void* W, int64_t N, int32_t H, int32_t V,
@@ -619,6 +770,7 @@ extern "C" int mrl_fused_lmhead_loss_fwd_bwd(const void* hidden, const void* W, 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool accum_loss = lp->flags & MRL_FLAG_ACCUMULATE_LOSS;
   const bool accum_dw = lp->flags & MRL_FLAG_ACCUMULATE_DW;
+  const bool pair = lp->flags & MRL_FLAG_PAIR_TILES;
   if (N == 0 || S == 0) {
     if (N != 0) return MRL_ERR_INVALID_ARG;
     if (!accum_loss) {
@@ -659,7 +811,7 @@ extern "C" int mrl_fused_lmhead_loss_fwd_bwd(const void* hidden, const void* W, 
     p.ids = ids;
     p.zt = w.zt;
     p.col0 = 0;
-    rc = launch_gemm<EPI_LSE>(hid, H, Wm, H, p, st);
+    rc = launch_gemm<EPI_LSE>(hid, H, Wm, H, p, pair, st);
     if (rc != MRL_OK) return rc;
   }
   lmhead_rows_kernel<<<(unsigned)((N + 255) / 256), 256, 0, st>>>(N, V, w.n_tiles_fwd, w.partial, w.part_ld, w.zt, ids,
@@ -693,21 +845,21 @@ extern "C" int mrl_fused_lmhead_loss_fwd_bwd(const void* hidden, const void* W, 
       p.ldD = w.ldD;
       p.DT = w.DT;
       p.ldDT = w.ldDT;
-      rc = launch_gemm<EPI_DZ>(hid, H, Wm + (size_t)v0 * H, H, p, st);
+      rc = launch_gemm<EPI_DZ>(hid, H, Wm + (size_t)v0 * H, H, p, pair, st);
       if (rc != MRL_OK) return rc;
     }
     {  // dHidden (+)= D[N, vc] * (W^T[H, v0 : v0 + vc])^T
       int mode = C_BF16;
       if (w.n_chunks > 1) mode = ch == 0 ? C_F32 : (ch == w.n_chunks - 1 ? C_BF16_FROM_ACC : C_F32_ADD);
       void* C = (mode == C_BF16 || mode == C_BF16_FROM_ACC) ? dHidden : static_cast<void*>(w.dH_acc);
-      rc = mrl_lmhead_gemm_tn(w.D, w.ldD, w.WT + v0, w.ldWT, (int)N, H, vc, C, H, mode, w.dH_acc, H, status, st);
+      rc = mrl_lmhead_gemm_tn(w.D, w.ldD, w.WT + v0, w.ldWT, (int)N, H, vc, C, H, mode, w.dH_acc, H, status, pair, st);
       if (rc != MRL_OK) return rc;
     }
     {  // dW[v0 : v0 + vc, :] = D^T[vc, N] * (hidden^T[H, N])^T
       void* C = accum_dw ? static_cast<void*>(static_cast<float*>(dW) + (size_t)v0 * H)
                          : static_cast<void*>(static_cast<__nv_bfloat16*>(dW) + (size_t)v0 * H);
       rc = mrl_lmhead_gemm_tn(w.DT, w.ldDT, w.HT, w.ldHT, vc, H, (int)N, C, H, accum_dw ? C_F32_ADD : C_BF16, nullptr,
-                              0, status, st);
+                              0, status, pair, st);
       if (rc != MRL_OK) return rc;
     }
   }

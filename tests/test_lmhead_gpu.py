@@ -123,6 +123,17 @@ def test_fused_lmhead_matches_oracle(N, H, V, S, mask_p, agg):
     compare(got, ref)
 
 
+@pytest.mark.parametrize("N,H,V,S,mask_p", [(300, 128, 1000, 5, None), (700, 256, 16384 + 8, 3, 0.8), (1, 64, 37, 1, None)])
+def test_pair_tiles_give_the_same_results(N, H, V, S, mask_p):
+    """MRL_FLAG_PAIR_TILES: every product on 256-row tiles shared by two CTAs; checked against the oracle."""
+    hidden, W, ids, mask, cu, adv, logp_old, g = toy(N, H, V, S, seed=3 * N + V, mask_p=mask_p)
+    nllw = (torch.rand(N, generator=g) < 0.2).float()
+    lp = make_lp(nll_coeff=0.05, flags=B.FLAG_PAIR_TILES)
+    got = run_gpu_lmhead(hidden, W, ids, mask, cu, adv, logp_old, None, nllw, lp)
+    ref = O.fused_lmhead_loss(hidden, W, ids, mask, cu, adv, logp_old, None, nllw, oracle_lp(lp))
+    compare(got, ref)
+
+
 def test_forward_only_and_dw_accumulation_in_float32():
     N, H, V, S = 200, 128, 3000, 4
     hidden, W, ids, mask, cu, adv, logp_old, g = toy(N, H, V, S, seed=9)
