@@ -142,7 +142,7 @@ __device__ __forceinline__ StreamVec<kWords> stream_ld(const void* p) {
                      "=r"(v.w[7])
                    : "l"(p));
     else
-      asm volatile("ld.global.L2::evict_first.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+      asm volatile("ld.global.L1::no_allocate.L2::evict_first.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
                    : "=r"(v.w[0]), "=r"(v.w[1]), "=r"(v.w[2]), "=r"(v.w[3]), "=r"(v.w[4]), "=r"(v.w[5]), "=r"(v.w[6]),
                      "=r"(v.w[7])
                    : "l"(p));
@@ -151,16 +151,21 @@ __device__ __forceinline__ StreamVec<kWords> stream_ld(const void* p) {
   }
   return v;
 }
+// Output lines are never read again: they are marked evict-first in L2 so that they do not push out the rows that
+// wait for their second read (the `.cs` qualifier alone does not do that).
 template <int kWords>
 __device__ __forceinline__ void stream_st(void* p, const StreamVec<kWords>& v) {
-  if constexpr (kWords == 8)
-    asm volatile("st.global.cs.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(v.w[0]), "r"(v.w[1]),
-                 "r"(v.w[2]), "r"(v.w[3]), "r"(v.w[4]), "r"(v.w[5]), "r"(v.w[6]), "r"(v.w[7])
+  if constexpr (kWords == 8) {
+    asm volatile("st.global.L2::evict_first.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(v.w[0]),
+                 "r"(v.w[1]), "r"(v.w[2]), "r"(v.w[3]), "r"(v.w[4]), "r"(v.w[5]), "r"(v.w[6]), "r"(v.w[7])
                  : "memory");
-  else
-    asm volatile("st.global.cs.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(v.w[0]), "r"(v.w[1]), "r"(v.w[2]),
-                 "r"(v.w[3])
+  } else {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    asm volatile("st.global.L2::cache_hint.v4.b32 [%0], {%1, %2, %3, %4}, %5;" ::"l"(p), "r"(v.w[0]), "r"(v.w[1]),
+                 "r"(v.w[2]), "r"(v.w[3]), "l"(pol)
                  : "memory");
+  }
 }
 template <int kWords>
 __device__ __forceinline__ StreamVec<kWords> stream_fill(uint32_t x) {
