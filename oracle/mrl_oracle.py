@@ -20,6 +20,7 @@ Passages followed (by section / equation of the paper):
   * SGT gate / transfer, Eq. (2), L_SGT "averaged per token and aggregated over
     all gated examples"                                                  (Sec. 5.3, App. B)
   * softmax score  grad log pi(a_i) = e_i - pi                            (App. H, proof of Prop. 1)
+  * THL word-level trace alignment  Z_w, C_w, Z_w / C_w                    (Sec. 4.2; App. D, Alg. 3; Thm. 1)
 
 Readings taken where the paper is silent are listed in the repository's
 design notes; each is a parameter here with the default stated.
@@ -27,7 +28,8 @@ design notes; each is a parameter here with the default stated.
 Pins (tests, CPU only): closed forms (uniform logits, V = 1, binary-reward
 advantages), brute force on tiny inputs, finite differences, the printed
 three-action example of Prop. 1, the rescue-gate probability of Def. 7, and
-library special cases (scipy logsumexp, torch cross_entropy).
+library special cases (scipy logsumexp, torch cross_entropy), and for the word alignment the per-word mass
+conservation and the residual identity of Thm. 1 evaluated from its own set definitions.
 Functions without a pin: none.
 """
 from __future__ import annotations
@@ -316,3 +318,67 @@ def fused_lmhead_loss(hidden, W, ids, mask, cu_seqlens, adv_seq, logp_old, tok_w
     out["dW"] = dz.T @ h
     out["logits"] = z
     return out
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# THL WordAlignLogProbs (Sec. 4.2; App. D, Alg. 3; Thm. 1)
+# ---------------------------------------------------------------------------------------------------------------
+
+def thl_word_align_logprobs(src_logp, src_word, src_cu, tgt_word, tgt_cu, ignore_value: float = 0.0):
+    """Word-level trace alignment of App. D, Alg. 3, on packed response tokens, in the algorithm's own steps.
+
+    For sequence i the source tokens are src_cu[i] .. src_cu[i+1]-1 with log-probs `src_logp` and word ids
+    `src_word` (the token-to-word map of Alg. 1; -1 = None), the target tokens tgt_cu[i] .. with word ids
+    `tgt_word`.  (The response masks of the algorithm are already applied: only response tokens are passed.)
+      pass 1: per_word_sum[w] = sum of the source log-probs of the tokens mapped to w          (Z_w)
+      a sequence whose per_word_sum is empty is skipped: its outputs stay at ignore_value
+      pass 2: per_word_count[w] = number of target tokens mapped to w                        (C_w)
+      pass 3: every target token with a word gets per_word_sum.get(w, 0) / per_word_count[w]
+    Returns out f64[N_tgt] (ignore_value where nothing is assigned).
+    """
+    src_logp = torch.as_tensor(src_logp).to(F64)
+    src_word = torch.as_tensor(src_word).long()
+    tgt_word = torch.as_tensor(tgt_word).long()
+    src_cu = torch.as_tensor(src_cu).long()
+    tgt_cu = torch.as_tensor(tgt_cu).long()
+    out = torch.full((int(tgt_cu[-1]) if tgt_cu.numel() else 0,), float(ignore_value), dtype=F64)
+    for i in range(src_cu.numel() - 1):
+        per_word_sum = {}
+        for p in range(int(src_cu[i]), int(src_cu[i + 1])):
+            wid = int(src_word[p])
+            if wid < 0:
+                continue
+            per_word_sum[wid] = per_word_sum.get(wid, 0.0) + float(src_logp[p])
+        if not per_word_sum:
+            continue
+        per_word_count = {}
+        for p in range(int(tgt_cu[i]), int(tgt_cu[i + 1])):
+            wid = int(tgt_word[p])
+            if wid < 0:
+                continue
+            per_word_count[wid] = per_word_count.get(wid, 0) + 1
+        for p in range(int(tgt_cu[i]), int(tgt_cu[i + 1])):
+            wid = int(tgt_word[p])
+            if wid < 0:
+                continue
+            cnt = per_word_count.get(wid, 0)
+            if cnt <= 0:
+                continue
+            out[p] = per_word_sum.get(wid, 0.0) / cnt
+    return out
+
+
+def thl_sequence_totals(src_logp, src_cu, aligned, tgt_word, tgt_cu, has_source):
+    """L_mu (all source response tokens) and L~_mu (aligned values on target tokens with a word) per sequence,
+    the two sides of Thm. 1.  `has_source[i]`: sequence i was not skipped by the algorithm."""
+    src_logp = torch.as_tensor(src_logp).to(F64)
+    aligned = torch.as_tensor(aligned).to(F64)
+    tgt_word = torch.as_tensor(tgt_word).long()
+    B = len(src_cu) - 1
+    L_src, L_tgt = torch.zeros(B, dtype=F64), torch.zeros(B, dtype=F64)
+    for i in range(B):
+        L_src[i] = src_logp[int(src_cu[i]):int(src_cu[i + 1])].sum()
+        if has_source[i]:
+            a, b = int(tgt_cu[i]), int(tgt_cu[i + 1])
+            L_tgt[i] = aligned[a:b][tgt_word[a:b] >= 0].sum()
+    return L_src, L_tgt

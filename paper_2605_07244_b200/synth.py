@@ -193,3 +193,46 @@ def make_batch(meta: Meta, select: torch.Tensor | None = None) -> Batch:
         spike_col = torch.where(on_target, ids, other)
     return Batch(w, seed, seq_p, seq_m, seq_g, cu.to(torch.int32), ids, noise, tok_weight, is_peer,
                  spike_col)
+
+
+@dataclass
+class WordMaps:
+    """Token-to-word maps of one batch under two tokenizers (what Alg. 1 of App. D would return), packed."""
+    src_word: torch.Tensor   # i32 [N_src], -1 = no word
+    src_cu: torch.Tensor     # i32 [B+1]
+    tgt_word: torch.Tensor   # i32 [N_tgt]
+    tgt_cu: torch.Tensor     # i32 [B+1]
+    word_cu: torch.Tensor    # i32 [B+1]: sequence i uses word ids [0, word_cu[i+1] - word_cu[i])
+    src_logp: torch.Tensor   # f32 [N_src]
+
+
+def make_word_maps(B: int, words: tuple, seed: int, p_uncovered: float = 0.03, p_leading_none: float = 0.3,
+                   p_source_gap: float = 0.02, max_pieces: int = 4) -> WordMaps:
+    """Sequences of `words` = (lo, hi) whitespace-delimited words; every word is cut into 1..max_pieces tokens by
+    the source tokenizer and, independently, by the target tokenizer (maps are non-decreasing, as a span-by-span
+    tokenisation produces them).  With small probabilities a word has no target token (a source-covered word
+    without a target slot), a word has no source token, and a sequence starts with delimiter tokens mapped to no
+    word.  Source log-probs are -Exp(1)-like draws of the size of per-token NLLs (App. F reports 0.2 .. 1.1)."""
+    g = _gen(seed, 21)
+    sw, tw, scu, tcu, wcu = [], [], [0], [0], [0]
+    for _ in range(B):
+        nw = int(torch.randint(words[0], words[1] + 1, (1,), generator=g))
+        s_cnt = torch.randint(1, max_pieces + 1, (nw,), generator=g)
+        t_cnt = torch.randint(1, max_pieces + 1, (nw,), generator=g)
+        t_cnt[torch.rand(nw, generator=g) < p_uncovered] = 0
+        s_cnt[torch.rand(nw, generator=g) < p_source_gap] = 0
+        ids = torch.arange(nw, dtype=torch.int32)
+        s_map, t_map = torch.repeat_interleave(ids, s_cnt), torch.repeat_interleave(ids, t_cnt)
+        if float(torch.rand(1, generator=g)) < p_leading_none:
+            s_map = torch.cat([torch.full((int(torch.randint(1, 3, (1,), generator=g)),), -1, dtype=torch.int32), s_map])
+            t_map = torch.cat([torch.full((int(torch.randint(1, 3, (1,), generator=g)),), -1, dtype=torch.int32), t_map])
+        sw.append(s_map)
+        tw.append(t_map)
+        scu.append(scu[-1] + s_map.numel())
+        tcu.append(tcu[-1] + t_map.numel())
+        wcu.append(wcu[-1] + nw)
+    src_word = torch.cat(sw) if sw else torch.zeros(0, dtype=torch.int32)
+    tgt_word = torch.cat(tw) if tw else torch.zeros(0, dtype=torch.int32)
+    src_logp = torch.log(torch.rand(src_word.numel(), generator=g).clamp_min(1e-6)) * 0.7
+    i32 = lambda x: torch.tensor(x, dtype=torch.int32)
+    return WordMaps(src_word.to(torch.int32), i32(scu), tgt_word.to(torch.int32), i32(tcu), i32(wcu), src_logp.float())
