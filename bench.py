@@ -373,6 +373,49 @@ class LmheadWorkload:
         return n, dt, f"first {n} rows of the same batch, full V and H, fwd+bwd incl. dW, float64, {dt:.1f} s"
 
 
+def measure_thl_align(seed, with_cpu):
+    """THL word alignment on a batch shaped like one PRP step of App. G.1: 256 prompts x 5 peer rollouts of
+    ~630 response tokens, words cut into 1..4 tokens by each tokenizer.  It is tiny next to the loss pass (a few
+    tens of MB, L2-resident), so it is reported as time per call and tokens/s, not against a roofline."""
+    from paper_2605_07244_b200 import binding as B
+    wm = synth.make_word_maps(1280, (150, 350), seed)
+    total_words = int(wm.word_cu[-1])
+    d = {k: getattr(wm, k).cuda() for k in ("src_logp", "src_word", "src_cu", "tgt_word", "tgt_cu", "word_cu")}
+    n_src, n_tgt = int(wm.src_cu[-1]), int(wm.tgt_cu[-1])
+    out = torch.empty(n_tgt, device="cuda")
+    tot = torch.empty(2, 1280, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ws = torch.empty(B.workspace_bytes(B.WS_THL_WORD_ALIGN, total_words, 0), dtype=torch.uint8, device="cuda")
+    call = lambda: B.mrl_thl_word_align_logprobs(d["src_logp"], d["src_word"], d["src_cu"], d["tgt_word"], d["tgt_cu"],
+                                                 d["word_cu"], total_words, 0.0, out, tot[0], tot[1], status, ws)
+    for _ in range(3):
+        call()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = 50
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(reps):
+        call()
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / reps
+    alg_bytes = 8 * n_src + 8 * n_tgt      # log-prob + word id per source token, word id + output per target token
+    res = {"metric": "thl_word_align_target_tokens_per_s", "value": n_tgt / (us * 1e-6), "unit": "tokens/s",
+           "us_per_call": us, "sequences": 1280, "source_tokens": n_src, "target_tokens": n_tgt, "words": total_words,
+           "algorithmic_bytes": alg_bytes, "achieved_gbs": alg_bytes / (us * 1e-6) / 1e9, "gpu_launches": reps,
+           "status": int(status.cpu())}
+    if with_cpu:
+        from oracle import mrl_oracle as O
+        k = 32
+        t0 = time.perf_counter()
+        O.thl_word_align_logprobs(wm.src_logp[:int(wm.src_cu[k])], wm.src_word[:int(wm.src_cu[k])], wm.src_cu[:k + 1],
+                                  wm.tgt_word[:int(wm.tgt_cu[k])], wm.tgt_cu[:k + 1], 0.0)
+        dt = time.perf_counter() - t0
+        res["cpu_baseline"] = {"value": int(wm.tgt_cu[k]) / dt, "unit": "tokens/s", "cores": 1, "kind": "oracle",
+                               "sample": f"first {k} sequences, {dt:.1f} s"}
+    return res
+
+
 def time_oracle(O, args, repeats=1):
     best = None
     for _ in range(repeats):
@@ -511,6 +554,10 @@ def run_ours(args, rank, world, local_rank):
                                                                          "gpu_launches", "roofline", "cpu_baseline")}}
         del wl5
 
+    thl = None
+    if args.workload == "C2" and not args.no_lmhead and rank == 0 and world == 1:
+        thl = measure_thl_align(args.seed, not args.no_cpu_baseline)
+
     if rank == 0:
         line = {
             "metric": METRIC, "value": res["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -521,6 +568,8 @@ def run_ours(args, rank, world, local_rank):
         }
         if lmhead is not None:
             line["lmhead"] = lmhead
+        if thl is not None:
+            line["thl_align"] = thl
         print(json.dumps(line))
 
 

@@ -54,6 +54,7 @@ extern "C" {
 /* bits of the device status word */
 #define MRL_DEV_BAD_TOKEN_ID 1
 #define MRL_DEV_TIMEOUT 2
+#define MRL_DEV_BAD_WORD_MAP 4
 
 /* element types of logits / dlogits */
 #define MRL_F32 0
@@ -89,6 +90,7 @@ extern "C" {
 #define MRL_WS_TOKEN_LOGPROBS 0
 #define MRL_WS_POLICY_LOSS 1
 #define MRL_WS_FUSED_LMHEAD 2
+#define MRL_WS_THL_WORD_ALIGN 3         /* N = total number of words of the batch; V, H, dtype, S unused */
 
 typedef struct mrl_adv_params {
   int32_t mode;             /* MRL_ADV_* */
@@ -277,6 +279,40 @@ int mrl_fused_lmhead_loss_fwd_bwd(const void* hidden, const void* W, int64_t N, 
                                   const mrl_loss_params* lp, void* dHidden, void* dW, float* logp,
                                   float* loss, int64_t* stats, int32_t* status, void* workspace,
                                   size_t workspace_bytes, void* stream);
+
+/*
+ * mrl_thl_word_align_logprobs -- THL policy-distribution alignment: a peer's per-token log-prob trace mapped onto
+ * the learner's tokenisation of the same text, the denominator of PRP's THL-aligned variant.
+ *
+ * Defined by: Sec. 4.2 (Z_w = sum of the source log-probs of word w; every target token of w gets
+ * Z_w / max(1, C_w), C_w the number of target tokens of w); App. D, Alg. 3 (a sequence with no source token
+ * mapped to a word is left at ignore_value; a target word without source tokens gets 0; tokens mapped to no word
+ * get ignore_value); App. H, Thm. 1 (per-word mass is conserved wherever C_w > 0).
+ *
+ * Tokens are packed, response tokens only (the algorithm's masks already applied).  Sequence i owns source
+ * tokens [src_cu[i], src_cu[i+1]), target tokens [tgt_cu[i], tgt_cu[i+1]) and word ids [0, word_cu[i+1] - word_cu[i]).
+ *
+ *   src_logp   [device] float32 [N_src]  source-policy log-probs
+ *   src_word   [device] int32   [N_src]  word id of each source token (App. D, Alg. 1), negative = no word
+ *   tgt_word   [device] int32   [N_tgt]  the same for the learner's tokens
+ *   src_cu, tgt_cu, word_cu  [device] int32 [B+1], non-decreasing, starting at 0
+ *   total_words  word_cu[B] (sizes the workspace)
+ *   out        [device] float32 [N_tgt]  aligned trace; every element is written
+ *   src_total  [device] float32 [B], nullable: sum of all source log-probs of the sequence (L_mu of Thm. 1)
+ *   tgt_total  [device] float32 [B], nullable: sum of the aligned values written (L~_mu); the difference of the
+ *              two is the residual R_THL of Thm. 1
+ *   workspace: mrl_workspace_bytes(MRL_WS_THL_WORD_ALIGN, total_words, 0, 0, 0, 0)
+ *
+ * Equal word ids must be contiguous within a sequence (what a span-by-span tokenisation yields); then every sum
+ * is taken in token order by one thread and results are bitwise reproducible.  A word id seen in two separate
+ * runs or outside the sequence's range sets MRL_DEV_BAD_WORD_MAP in `status` (such tokens count as "no word" /
+ * their word's value is then unspecified).  float32 sums.  B = 0 is a no-op.
+ */
+int mrl_thl_word_align_logprobs(const float* src_logp, const int32_t* src_word, const int32_t* src_cu,
+                                const int32_t* tgt_word, const int32_t* tgt_cu, const int32_t* word_cu, int32_t B,
+                                int64_t total_words, float ignore_value, float* out, float* src_total,
+                                float* tgt_total, int32_t* status, void* workspace, size_t workspace_bytes,
+                                void* stream);
 
 /*
  * mrl_profile_dominant_kernel -- instrumentation for benchmarks; the paper has no counterpart.

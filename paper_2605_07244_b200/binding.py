@@ -18,12 +18,12 @@ ADV_MEAN_ONLY, ADV_GROUP_ZNORM, ADV_BATCH_ZNORM = 0, 1, 2
 PICK_NONE, PICK_FIRST, PICK_SHORTEST, PICK_ALL, PICK_SEEDED = 0, 1, 2, 3, 4
 AGG_TOKEN_MEAN, AGG_SEQ_MEAN_TOKEN_MEAN = 0, 1
 FLAG_ACCUMULATE_LOSS, FLAG_SKIP_ZERO_ROWS, FLAG_ACCUMULATE_DW, FLAG_PAIR_TILES = 1, 2, 4, 8
-WS_TOKEN_LOGPROBS, WS_POLICY_LOSS, WS_FUSED_LMHEAD = 0, 1, 2
-DEV_BAD_TOKEN_ID, DEV_TIMEOUT = 1, 2
+WS_TOKEN_LOGPROBS, WS_POLICY_LOSS, WS_FUSED_LMHEAD, WS_THL_WORD_ALIGN = 0, 1, 2, 3
+DEV_BAD_TOKEN_ID, DEV_TIMEOUT, DEV_BAD_WORD_MAP = 1, 2, 4
 
 EXPORTS = ("mrl_group_advantages", "mrl_token_logprobs", "mrl_policy_loss_fwd_bwd",
            "mrl_fused_lmhead_loss_fwd_bwd", "mrl_workspace_bytes", "mrl_status_string", "mrl_version",
-           "mrl_profile_dominant_kernel", "mrl_policy_loss_fwd_bwd_static")
+           "mrl_profile_dominant_kernel", "mrl_policy_loss_fwd_bwd_static", "mrl_thl_word_align_logprobs")
 STATIC_MAX_ROWS, STATIC_MAX_SEQS = 65536, 65536
 ERR_STATIC_SCRATCH_TOO_SMALL = 8
 
@@ -71,6 +71,8 @@ def lib() -> C.CDLL:
         L.mrl_fused_lmhead_loss_fwd_bwd.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, vp, vp, vp,
                                                     C.POINTER(LossParams), vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.mrl_fused_lmhead_loss_fwd_bwd.restype = C.c_int
+        L.mrl_thl_word_align_logprobs.argtypes = [vp, vp, vp, vp, vp, vp, i32, i64, C.c_float, vp, vp, vp, vp, vp, sz, vp]
+        L.mrl_thl_word_align_logprobs.restype = C.c_int
         L.mrl_workspace_bytes.argtypes = [i32, i64, i32, i32, i32, i32]
         L.mrl_workspace_bytes.restype = sz
         L.mrl_status_string.argtypes = [C.c_int]
@@ -181,6 +183,16 @@ def mrl_fused_lmhead_loss_fwd_bwd(hidden, W, ids, mask, cu_seqlens, adv_seq, log
                                                C.byref(lp), _p(dHidden), _p(dW), _p(logp), _p(loss), _p(stats),
                                                _p(status), _p(workspace), ws_bytes, _stream(stream)),
            "mrl_fused_lmhead_loss_fwd_bwd")
+
+
+def mrl_thl_word_align_logprobs(src_logp, src_word, src_cu, tgt_word, tgt_cu, word_cu, total_words, ignore_value,
+                                out, src_total=None, tgt_total=None, status=None, workspace=None, stream=None):
+    Bn = src_cu.numel() - 1
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib().mrl_thl_word_align_logprobs(_p(src_logp), _p(src_word), _p(src_cu), _p(tgt_word), _p(tgt_cu),
+                                             _p(word_cu), Bn, int(total_words), float(ignore_value), _p(out),
+                                             _p(src_total), _p(tgt_total), _p(status), _p(workspace), ws_bytes,
+                                             _stream(stream)), "mrl_thl_word_align_logprobs")
 
 
 class DominantKernelTimer:

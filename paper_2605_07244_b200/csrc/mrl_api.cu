@@ -3,6 +3,7 @@
 
 size_t mrl_policy_loss_workspace_bytes(long long N, int S);
 size_t mrl_fused_lmhead_workspace_bytes(long long N, int V, int H, int S);
+size_t mrl_thl_workspace_bytes(long long total_words);
 
 extern "C" size_t mrl_workspace_bytes(int32_t which, int64_t N, int32_t V, int32_t H, int32_t dtype, int32_t S) {
   (void)dtype;
@@ -14,6 +15,8 @@ extern "C" size_t mrl_workspace_bytes(int32_t which, int64_t N, int32_t V, int32
       return mrl_policy_loss_workspace_bytes(N, S);
     case MRL_WS_FUSED_LMHEAD:
       return mrl_fused_lmhead_workspace_bytes(N, V, H, S);
+    case MRL_WS_THL_WORD_ALIGN:
+      return mrl_thl_workspace_bytes(N);
     default:
       return 0;
   }
