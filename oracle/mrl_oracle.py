@@ -20,6 +20,7 @@ Passages followed (by section / equation of the paper):
   * SGT gate / transfer, Eq. (2), L_SGT "averaged per token and aggregated over
     all gated examples"                                                  (Sec. 5.3, App. B)
   * softmax score  grad log pi(a_i) = e_i - pi                            (App. H, proof of Prop. 1)
+  * response-level ratio  w = exp(L_theta - L_behavior)                     (App. H, data-level coupling)
   * THL word-level trace alignment  Z_w, C_w, Z_w / C_w                    (Sec. 4.2; App. D, Alg. 3; Thm. 1)
 
 Readings taken where the paper is silent are listed in the repository's
@@ -52,6 +53,10 @@ PICK_FIRST = 1
 PICK_SHORTEST = 2
 PICK_ALL = 3
 PICK_SEEDED = 4
+
+# importance ratio level: per token (Sec. 3, Eq. (1)) or per response (App. H, data-level coupling)
+RATIO_TOKEN = 0
+RATIO_SEQUENCE = 1
 
 # token aggregation (Eq. (1) E_tok then 1/K; or one masked mean over all tokens)
 AGG_TOKEN_MEAN = 0
@@ -198,6 +203,7 @@ class LossParams:
     pg_denominator: float = 0.0   # <= 0: number of valid tokens in this call
     seq_denominator: float = 0.0  # <= 0: number of sequences in this call
     nll_coeff: float = 0.0        # lambda_SGT / n_gated (Eq. (2); App. B)
+    ratio_level: int = RATIO_TOKEN
 
 
 def row_coefficients(valid, cu_seqlens, adv_seq, tok_weight, nll_weight, lp: LossParams):
@@ -302,6 +308,90 @@ def policy_loss(logits, ids, mask, cu_seqlens, adv_seq, logp_old, tok_weight=Non
             safe = torch.where(valid[idx], ids_l[idx], torch.zeros_like(ids_l[idx]))
             onehot.scatter_(1, safe[:, None], 1.0)
             dz[a:a + _ROW_BLOCK] = g[idx, None] * (p - onehot)
+        out["dlogits"] = dz
+    return out
+
+
+def sequence_ratio_surrogate(logp, logp_old, valid, cu_seqlens, adv_seq, nll_weight, lp: LossParams):
+    """Response-level importance ratio of App. H (data-level coupling): with L = sum_t l_t over the valid tokens
+    of a response,  w = exp(L_theta - L_behavior),  s = min(w A, clip(w, 1-eps_lo, 1+eps_hi) A), and the loss is
+    the mean of -s over the responses (the 1/K sum of Eq. (1) with E_tok replaced by the response-level term).
+    A response is clipped iff (A > 0 and w > 1+eps_hi) or (A < 0 and w < 1-eps_lo); responses without a valid
+    token contribute nothing.  The gated NLL term of Eq. (2) is unchanged (token level).
+    Returns dict: seq_term f64[S] (= -s / S_d), w f64[S], seq_clipped bool[S], seq_margin f64[S], per-row
+    g (dL/dlogp = -g), nll_term, cn.
+    """
+    logp = torch.as_tensor(logp).to(F64)
+    logp_old = torch.as_tensor(logp_old).to(F64)
+    valid = torch.as_tensor(valid).bool()
+    cu = torch.as_tensor(cu_seqlens).long()
+    S = cu.shape[0] - 1
+    N = logp.shape[0]
+    adv_seq = torch.as_tensor(adv_seq).to(F64)
+    nw = torch.zeros(N, dtype=F64) if nll_weight is None else torch.as_tensor(nll_weight).to(F64)
+    Sd = lp.seq_denominator if lp.seq_denominator > 0 else float(S)
+    lo, hi = 1.0 - lp.eps_lo, 1.0 + lp.eps_hi
+    seq_term = torch.zeros(S, dtype=F64)
+    w = torch.ones(S, dtype=F64)
+    seq_clipped = torch.zeros(S, dtype=torch.bool)
+    seq_margin = torch.full((S,), math.inf, dtype=F64)
+    g = torch.zeros(N, dtype=F64)
+    cn = torch.zeros(N, dtype=F64)
+    for s_ in range(S):
+        a, b = int(cu[s_]), int(cu[s_ + 1])
+        v = valid[a:b]
+        n_valid = int(v.sum())
+        if n_valid == 0:
+            continue
+        cn[a:b] = lp.nll_coeff * v.to(F64) * nw[a:b] / n_valid
+        A = float(adv_seq[s_])
+        L_theta = float(logp[a:b][v].sum())
+        L_beh = float(logp_old[a:b][v].sum())
+        ws = math.exp(L_theta - L_beh)
+        w[s_] = ws
+        if A == 0:
+            continue
+        sur = min(ws * A, min(max(ws, lo), hi) * A)
+        seq_term[s_] = -sur / Sd
+        clipped = (A > 0 and ws > hi) or (A < 0 and ws < lo)
+        seq_clipped[s_] = clipped
+        seq_margin[s_] = abs(ws - (hi if A > 0 else lo))
+        if not clipped:
+            g[a:b] = v.to(F64) * (A * ws / Sd)
+    nll_term = torch.where(cn != 0, -cn * logp, torch.zeros_like(logp))
+    return dict(seq_term=seq_term, w=w, seq_clipped=seq_clipped, seq_margin=seq_margin, g=g + cn, cn=cn,
+                nll_term=nll_term)
+
+
+def policy_loss_sequence_ratio(logits, ids, mask, cu_seqlens, adv_seq, logp_old, nll_weight=None,
+                               lp: LossParams | None = None, want_dlogits: bool = True):
+    """The logits-in pass with the response-level ratio: log-probs, sequence_ratio_surrogate, and
+    dlogits[t, v] = g_t (softmax(z_t)[v] - 1[v == ids_t]) with the same g for every token of a response."""
+    lp = lp or LossParams(ratio_level=RATIO_SEQUENCE)
+    logits = torch.as_tensor(logits)
+    N, V = logits.shape
+    ids_l = torch.as_tensor(ids).long()
+    logp, lse, valid = token_logprobs(logits, ids_l, mask)
+    if logp_old is None:
+        logp_old = logp
+    sur = sequence_ratio_surrogate(logp, logp_old, valid, cu_seqlens, adv_seq, nll_weight, lp)
+    out = dict(sur)
+    out.update(logp=logp, lse=lse, valid=valid)
+    out["loss_pg"] = float(sur["seq_term"].sum())
+    out["loss_nll"] = float(sur["nll_term"].sum())
+    cu = torch.as_tensor(cu_seqlens).long()
+    lens = cu[1:] - cu[:-1]
+    row_clipped = torch.repeat_interleave(sur["seq_clipped"], lens) & valid
+    out["stats"] = (int(valid.sum()), int(row_clipped.sum()))
+    if want_dlogits:
+        dz = torch.empty(N, V, dtype=F64)
+        for a in range(0, N, _ROW_BLOCK):
+            z = logits[a:a + _ROW_BLOCK].to(F64)
+            p = torch.exp(z - lse[a:a + _ROW_BLOCK, None])
+            onehot = torch.zeros_like(p)
+            safe = torch.where(valid[a:a + _ROW_BLOCK], ids_l[a:a + _ROW_BLOCK], torch.zeros_like(ids_l[a:a + _ROW_BLOCK]))
+            onehot.scatter_(1, safe[:, None], 1.0)
+            dz[a:a + _ROW_BLOCK] = sur["g"][a:a + _ROW_BLOCK, None] * (p - onehot)
         out["dlogits"] = dz
     return out
 
