@@ -139,10 +139,11 @@ def barrier(world: int):
 class LogitsInWorkload:
     """Config 2: 8 prompts x G = 8, ragged lengths in [128, 1024] packed, V = 151,936, bf16 logits."""
 
-    def __init__(self, w: synth.Workload, seed: int, device):
+    def __init__(self, w: synth.Workload, seed: int, device, ratio_level: int = 0):
         from paper_2605_07244_b200 import binding as B
         self.B = B
         self.w = w
+        self.ratio_level = ratio_level
         self.meta = synth.make_meta(w, seed)
         self.batch = synth.make_batch(self.meta)
         b = self.batch
@@ -171,14 +172,19 @@ class LogitsInWorkload:
         self.ws = torch.empty(B.workspace_bytes(B.WS_POLICY_LOSS, self.N, self.V, 0, B.BF16, self.S),
                               dtype=torch.uint8, device=dev)
         self.ap = B.AdvParams(B.ADV_GROUP_ZNORM, 0, 1e-6, 0.8, 0.2, B.PICK_SHORTEST, 0)
-        self.lp = B.LossParams(0.2, 0.2, B.AGG_TOKEN_MEAN, 0, 0.0, 0.0, 0.0, 0)
-        # behaviour trace: logp_old = logp + N(0, 0.1); logp from the library's forward (input preparation)
+        self.lp = B.LossParams(0.2, 0.2, B.AGG_TOKEN_MEAN, 0, 0.0, 0.0, 0.0, ratio_level)
+        # behaviour trace: logp_old = logp + N(0, 0.1); logp from the library's forward (input preparation).
+        # For the response-level ratio the noise is scaled by 1 / sqrt(mean length) so that w stays of order one.
         B.mrl_token_logprobs(self.z, self.ids, None, self.logp)
-        self.logp_old = self.logp + b.noise.to(dev)
+        scale = 1.0 if ratio_level == 0 else (self.S / max(self.N, 1)) ** 0.5
+        self.logp_old = self.logp + b.noise.to(dev) * scale
         torch.cuda.synchronize()
-        self.kernels_per_step = 6    # adv_prompt, seq_count, row_coef, row_stream, row_terms, finalize
-        self.dominant_per_step = 1
-        self.bytes_per_token = 2 * self.V * self.z.element_size()   # read V + write V elements
+        # adv_prompt, seq_count, row_coef, row_stream, row_terms, finalize; the response-level ratio has a forward
+        # launch, the per-response kernel and a backward launch instead of one fused row kernel
+        self.kernels_per_step = 6 if ratio_level == 0 else 7
+        self.dominant_per_step = 1 if ratio_level == 0 else 2
+        # read V + write V elements; the response-level ratio reads the row a second time from HBM
+        self.bytes_per_token = (2 if ratio_level == 0 else 3) * self.V * self.z.element_size()
 
     def step(self, z=None, dz=None):
         B = self.B
@@ -197,6 +203,7 @@ class LogitsInWorkload:
                             "ragged T in [128,1024], V=151936, bf16 logits N(0,2^2) + one +12 spike per row, "
                             "GRPO group z-norm, eps 0.2",
                 "rows": self.N, "sequences": self.S, "V": self.V, "logits_dtype": "bf16",
+                "ratio_level": "token" if self.ratio_level == 0 else "response (App. H)",
                 "l2": "inputs (%.1f GB logits) exceed the 126 MB L2; no flush needed" % (self.z.numel() * 2 / 1e9)}
 
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region
@@ -222,11 +229,18 @@ class LogitsInWorkload:
         self.h_loss.copy_(self.loss, non_blocking=True)
 
     def roofline(self, kernel_ms, peaks):
-        k_avg_ms = sum(kernel_ms) / len(kernel_ms)
+        k_avg_ms = sum(kernel_ms) / (len(kernel_ms) / self.dominant_per_step)
         alg_bytes = self.bytes_per_token * self.tokens()
+        if self.ratio_level != 0:
+            # forward reads every row, backward writes every row but reads only rows with a gradient: those of
+            # responses with A != 0 that are not clipped (stats[1] = valid rows of clipped responses)
+            lens = (self.cu[1:] - self.cu[:-1]).cpu()
+            live_rows = int(lens[(self.adv_own.reshape(-1) != 0).cpu()].sum()) - int(self.stats.cpu()[1])
+            alg_bytes = (2 * self.tokens() + live_rows) * self.V * self.z.element_size()
         achieved = alg_bytes / (k_avg_ms * 1e-3) / 1e9
-        per_token = ROW_STREAM_DRAM_BYTES_PER_TOKEN_V151936 if self.V == 151936 else None
-        return {"bound": "hbm", "kernel": "row_stream_kernel", "achieved": achieved, "peak": peaks["hbm_gbs"],
+        per_token = ROW_STREAM_DRAM_BYTES_PER_TOKEN_V151936 if self.V == 151936 and self.ratio_level == 0 else None
+        kernel = "row_stream_kernel" if self.ratio_level == 0 else "row_stream_kernel (forward) + row_backward_stream_kernel"
+        return {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peaks["hbm_gbs"],
                 "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
                 "peak_source": peaks["source"] + " (copy, burst)", "algorithmic_bytes_per_launch": alg_bytes,
                 "kernel_ms": k_avg_ms, "traffic": None if per_token is None else per_token * self.tokens()}
@@ -538,7 +552,8 @@ def run_ours(args, rank, world, local_rank):
     peaks = measured_peaks()
     lmhead_main = args.workload in ("C5", "C5s")
     cls = LmheadWorkload if lmhead_main else LogitsInWorkload
-    wl = cls(synth.CONFIGS[args.workload], args.seed + rank, device)
+    wl = (cls(synth.CONFIGS[args.workload], args.seed + rank, device) if lmhead_main else
+          cls(synth.CONFIGS[args.workload], args.seed + rank, device, 1 if args.ratio_level == "sequence" else 0))
     res = measure(wl, args.steps, args.warmup, world, local_rank, rank, peaks, not args.no_e2e,
                   not args.no_cpu_baseline, args)
     del wl
@@ -583,6 +598,8 @@ def main():
     ap.add_argument("--seed", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="profiling runs only: skip the host-buffer leg")
+    ap.add_argument("--ratio-level", default="token", choices=["token", "sequence"],
+                    help="logits-in workloads: importance ratio per token (Eq. (1), default) or per response (App. H)")
     ap.add_argument("--no-lmhead", action="store_true", help="skip the short config-5 leg of the default run")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))

@@ -76,6 +76,11 @@ extern "C" {
 #define MRL_AGG_TOKEN_MEAN 0            /* one masked mean over all tokens */
 #define MRL_AGG_SEQ_MEAN_TOKEN_MEAN 1   /* Eq. (1): E_tok within each sequence, then the mean over sequences */
 
+/* mrl_loss_params.ratio_level */
+#define MRL_RATIO_TOKEN 0      /* rho_t = exp(logp_t - logp_old_t), clipped per token               (Sec. 3, Eq. (1)) */
+#define MRL_RATIO_SEQUENCE 1   /* w = exp(sum_t logp_t - sum_t logp_old_t) over a response, clipped per
+                                  response; loss = - mean over responses of min(w A, clip(w) A)  (App. H) */
+
 /* mrl_loss_params.flags */
 #define MRL_FLAG_ACCUMULATE_LOSS 1u   /* loss[0..1] and stats += this call (micro-batch accumulation, App. A) */
 #define MRL_FLAG_SKIP_ZERO_ROWS 2u    /* rows whose gradient multiplier is known to be zero before reading the
@@ -111,7 +116,7 @@ typedef struct mrl_loss_params {
                                several calls; <= 0: the valid tokens of this call */
   double seq_denominator;   /* SEQ_MEAN_TOKEN_MEAN: number of sequences of the whole step; <= 0: S */
   float nll_coeff;          /* lambda_SGT / n_gated (Eq. (2), App. B); 0 disables the NLL term */
-  int32_t reserved;
+  int32_t ratio_level;      /* MRL_RATIO_*; 0 (token level) is the default */
 } mrl_loss_params;
 
 /*
@@ -186,6 +191,14 @@ int mrl_token_logprobs(const void* logits, int32_t dtype, int64_t N, int32_t V, 
  *   dlogits[t, v] = g_t (softmax(z_t)[v] - [v == ids_t])
  * t is clipped iff (A_t > 0 and rho_t > 1+eps_hi) or (A_t < 0 and rho_t < 1-eps_lo); equality is
  * unclipped.  Rows with c_t u_t A_t = 0 add exactly 0 to loss[0].
+ *
+ * With ratio_level = MRL_RATIO_SEQUENCE (App. H, data-level coupling) the ratio is taken per response:
+ *   w_s = exp(sum over the valid rows of s of (logp_t - logp_old_t)),  S_d = seq_denominator (<= 0: S)
+ *   loss[0] = - (1 / S_d) sum_s min(w_s A_s, clip(w_s) A_s)   over responses with a valid row
+ *   g_t = A_s w_s / S_d [s unclipped] + cn_t   for every valid row of s
+ * agg_mode and pg_denominator are not used, tok_weight must be NULL (MRL_ERR_INVALID_ARG otherwise),
+ * SKIP_ZERO_ROWS is ignored, and the gradient is a second launch that reads the logits again.  Every
+ * response must be whole inside one call.  stats[1] counts the valid rows of clipped responses.
  *
  *   logits     [device] dtype [N, ld]
  *   ids, mask  as in mrl_token_logprobs

@@ -52,6 +52,10 @@ int mrl_rows_prepare(void* workspace, long long N, int V, int S, const int32_t* 
 int mrl_rows_finish(const MrlLossWs& w, long long N, const float* logp_old, const mrl_loss_params* lp, float* logp,
                     float* loss, int64_t* stats, cudaStream_t st);
 
+int mrl_rows_finish_sequence(const MrlLossWs& w, long long N, int S, const int32_t* cu_seqlens, const float* adv_seq,
+                             const float* logp_old, const float* nll_weight, const mrl_loss_params* lp, float* logp,
+                             float* loss, int64_t* stats, float* g_out, float* lse2_out, cudaStream_t st);
+
 // Benchmark instrumentation (mrl_profile_dominant_kernel): event pairs recorded around dominant kernels.
 void mrl_profile_before(cudaStream_t st);
 void mrl_profile_after(cudaStream_t st);

@@ -767,6 +767,8 @@ extern "C" int mrl_fused_lmhead_loss_fwd_bwd(const void* hidden, const void* W, 
   if (N > 0x7fffff00ll) return MRL_ERR_UNSUPPORTED_SHAPE;
   if (lp->agg_mode != MRL_AGG_TOKEN_MEAN && lp->agg_mode != MRL_AGG_SEQ_MEAN_TOKEN_MEAN) return MRL_ERR_INVALID_ARG;
   if (!(lp->eps_lo >= 0.f) || !(lp->eps_hi >= 0.f)) return MRL_ERR_INVALID_ARG;
+  if (lp->ratio_level != MRL_RATIO_TOKEN && lp->ratio_level != MRL_RATIO_SEQUENCE) return MRL_ERR_INVALID_ARG;
+  if (lp->ratio_level == MRL_RATIO_SEQUENCE && tok_weight != nullptr) return MRL_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool accum_loss = lp->flags & MRL_FLAG_ACCUMULATE_LOSS;
   const bool accum_dw = lp->flags & MRL_FLAG_ACCUMULATE_DW;
@@ -814,12 +816,18 @@ extern "C" int mrl_fused_lmhead_loss_fwd_bwd(const void* hidden, const void* W, 
     rc = launch_gemm<EPI_LSE>(hid, H, Wm, H, p, pair, st);
     if (rc != MRL_OK) return rc;
   }
+  const bool seq_ratio = lp->ratio_level == MRL_RATIO_SEQUENCE;
   lmhead_rows_kernel<<<(unsigned)((N + 255) / 256), 256, 0, st>>>(N, V, w.n_tiles_fwd, w.partial, w.part_ld, w.zt, ids,
-                                                                  mask, rw.rowA, rw.rowcu, rw.rowcn, logp_old,
-                                                                  lp->eps_lo, lp->eps_hi, rw.row_m2, rw.row_s,
-                                                                  rw.row_zt, rw.rowstat, w.g, w.lse2);
+                                                                  mask, rw.rowA, rw.rowcu, rw.rowcn,
+                                                                  seq_ratio ? nullptr : logp_old, lp->eps_lo,
+                                                                  lp->eps_hi, rw.row_m2, rw.row_s, rw.row_zt,
+                                                                  rw.rowstat, w.g, w.lse2);
   MRL_CUDA_OK(cudaGetLastError());
-  rc = mrl_rows_finish(rw, N, logp_old, lp, logp, loss, stats, st);
+  if (seq_ratio)  // response-level ratio: g_t comes from the whole response (App. H)
+    rc = mrl_rows_finish_sequence(rw, N, S, cu_seqlens, adv_seq, logp_old, nll_weight, lp, logp, loss, stats, w.g,
+                                  w.lse2, st);
+  else
+    rc = mrl_rows_finish(rw, N, logp_old, lp, logp, loss, stats, st);
   if (rc != MRL_OK) return rc;
   if (dHidden == nullptr) return MRL_OK;
 

@@ -429,6 +429,144 @@ __global__ void __launch_bounds__(kThreads) row_general_kernel(const RowParams p
 }
 
 // ------------------------------------------------------------------------------------------------
+// Backward-only row kernels (response-level ratio): g_t is known only once the whole response has been scored, so
+// the gradient is a launch of its own that reads the row again.
+// ------------------------------------------------------------------------------------------------
+template <int kT, int kU, int kWords>
+__global__ void __launch_bounds__(kT, 1024 / kT) row_backward_stream_kernel(const RowParams p, const float* __restrict__ row_g,
+                                                                            const float* __restrict__ row_lse2,
+                                                                            const float* __restrict__ row_zt) {
+  constexpr int kVecBytes = kWords * 4, kVecElems = kWords * 2;
+  using Vec = StreamVec<kWords>;
+  const int tid = threadIdx.x;
+  const long long row = blockIdx.x;
+  const int nvec = p.V / kVecElems;
+  const char* in = reinterpret_cast<const char*>(static_cast<const __nv_bfloat16*>(p.logits) + row * p.ld) +
+                   (size_t)tid * kVecBytes;
+  __nv_bfloat16* orow = static_cast<__nv_bfloat16*>(p.dlogits) + row * p.ld_out;
+  char* out = reinterpret_cast<char*>(orow) + (size_t)tid * kVecBytes;
+  const float g = row_g[row];
+  if (g == 0.f) {
+    for (int i = tid; i < nvec; i += kT) stream_st<kWords>(out + (size_t)(i - tid) * kVecBytes, stream_fill<kWords>(0u));
+    return;
+  }
+  const float lse2 = row_lse2[row];
+  const float neg_k = -(lse2 - log2f(fabsf(g)));  // 2^(z log2e - k) = |g| softmax(z)
+  const uint32_t sign = g < 0.f ? 0x80008000u : 0u;
+  for (int base = 0; base < nvec; base += kT * kU) {
+    const bool full = base + kT * kU <= nvec;
+    Vec v[kU];
+#pragma unroll
+    for (int u = 0; u < kU; ++u)
+      v[u] = (full || base + u * kT + tid < nvec) ? stream_ld<kWords, kHintLast>(in + (size_t)(base + u * kT) * kVecBytes)
+                                                  : stream_fill<kWords>(0u);
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+      Vec r;
+#pragma unroll
+      for (int j = 0; j < kWords; ++j) {
+        const float a = mrl::ex2_approx(fmaf(mrl::bf16lo_to_f32(v[u].w[j]), MRL_LOG2E, neg_k));
+        const float b = mrl::ex2_approx(fmaf(mrl::bf16hi_to_f32(v[u].w[j]), MRL_LOG2E, neg_k));
+        r.w[j] = mrl::pack_bf16x2(a, b) ^ sign;
+      }
+      if (full || base + u * kT + tid < nvec) stream_st<kWords>(out + (size_t)(base + u * kT) * kVecBytes, r);
+    }
+  }
+  const int id = p.ids[row];  // g != 0 only on valid rows: the id is in range
+  if (tid == (id / kVecElems) % kT)
+    orow[id] = __float2bfloat16_rn(g * (mrl::ex2_approx(fmaf(row_zt[row], MRL_LOG2E, -lse2)) - 1.0f));
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads) row_backward_general_kernel(const RowParams p, const float* __restrict__ row_g,
+                                                                        const float* __restrict__ row_lse2,
+                                                                        const float* __restrict__ row_zt) {
+  const int tid = threadIdx.x;
+  const long long row = blockIdx.x;
+  const T* z = static_cast<const T*>(p.logits) + row * p.ld;
+  T* dz = static_cast<T*>(p.dlogits) + row * p.ld_out;
+  const float g = row_g[row];
+  if (g == 0.f) {
+    for (int v = tid; v < p.V; v += kThreads) st_from_f32<T>(dz + v, 0.f);
+    return;
+  }
+  const float lse2 = row_lse2[row];
+  const float neg_k = -(lse2 - log2f(fabsf(g)));
+  const float sgn = g < 0.f ? -1.f : 1.f;
+  for (int v = tid; v < p.V; v += kThreads)
+    st_from_f32<T>(dz + v, sgn * mrl::ex2_approx(fmaf(ld_as_f32<T>(z + v), MRL_LOG2E, neg_k)));
+  __syncthreads();
+  if (tid == 0) st_from_f32<T>(dz + p.ids[row], g * (mrl::ex2_approx(fmaf(row_zt[row], MRL_LOG2E, -lse2)) - 1.0f));
+}
+
+// Response-level ratio (App. H, data-level coupling): one block per response.  L_theta - L_behavior over the valid
+// tokens in float64 (fixed order), w = exp of it, the clip decision, the response's loss term (kept on its first
+// row), and for every row the gradient multiplier g_t = A w / S_d [unclipped] + cn_t and the base-2 log-sum-exp the
+// backward launch needs.  g_out / lse2_out may alias row_s / row_m2 (each thread reads its row before writing it).
+__global__ void __launch_bounds__(256) seq_ratio_kernel(const int32_t* __restrict__ cu, int S, long long N,
+                                                         const float* row_m2, const float* row_s,
+                                                         const float* __restrict__ row_zt, uint8_t* __restrict__ rowstat,
+                                                         const int32_t* __restrict__ seq_cnt,
+                                                         const float* __restrict__ adv_seq,
+                                                         const float* __restrict__ logp_old,
+                                                         const float* __restrict__ nll_weight, mrl_loss_params lp,
+                                                         double* __restrict__ pg_term, double* __restrict__ nll_term,
+                                                         float* __restrict__ logp, float* g_out, float* lse2_out) {
+  __shared__ double red[8];
+  __shared__ double diff_sh;
+  const int s = blockIdx.x, tid = threadIdx.x;
+  const long long a = max(0ll, min((long long)cu[s], N)), b = max(a, min((long long)cu[s + 1], N));
+  const double kLn2 = 0.693147180559945309417232121458;
+  double d = 0.0;
+  for (long long t = a + tid; t < b; t += 256) {
+    const uint8_t st = rowstat[t];
+    if ((st & kStatValid) && (st & kStatRead)) {
+      const double lpv = (double)row_zt[t] - ((double)row_m2[t] + log2((double)row_s[t])) * kLn2;
+      d += lpv - (logp_old ? (double)logp_old[t] : lpv);
+    }
+  }
+  for (int o = 16; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
+  if ((tid & 31) == 0) red[tid >> 5] = d;
+  __syncthreads();
+  if (tid == 0) {
+    double t = 0.0;
+    for (int k = 0; k < 8; ++k) t += red[k];
+    diff_sh = t;
+  }
+  __syncthreads();
+  const double len = (double)seq_cnt[s];
+  const double Sd = lp.seq_denominator > 0 ? lp.seq_denominator : (double)S;
+  const double A = adv_seq[s];
+  const double w = exp(diff_sh);
+  const double lo = 1.0 - (double)lp.eps_lo, hi = 1.0 + (double)lp.eps_hi;
+  const bool live = len > 0 && A != 0.0;
+  const bool clipped = live && ((A > 0 && w > hi) || (A < 0 && w < lo));
+  const double term = live ? -fmin(w * A, fmin(fmax(w, lo), hi) * A) / Sd : 0.0;
+  const float g_pg = (live && !clipped) ? (float)(A * w / Sd) : 0.f;
+  const double cn_base = len > 0 ? (double)lp.nll_coeff / len : 0.0;
+  for (long long t = a + tid; t < b; t += 256) {
+    const uint8_t st = rowstat[t];
+    const bool valid = (st & kStatValid) && (st & kStatRead);
+    double lpv = 0.0;
+    float l2 = 0.f, g = 0.f;
+    double nl = 0.0;
+    if (valid) {
+      l2 = row_m2[t] + log2f(row_s[t]);
+      lpv = (double)row_zt[t] - ((double)row_m2[t] + log2((double)row_s[t])) * kLn2;
+      const float cn = nll_weight ? (float)cn_base * nll_weight[t] : 0.f;
+      g = g_pg + cn;
+      if (cn != 0.f) nl = -(double)cn * lpv;
+      if (clipped) rowstat[t] = st | kStatClipped;
+    }
+    pg_term[t] = t == a ? term : 0.0;
+    nll_term[t] = nl;
+    if (logp != nullptr) logp[t] = (float)lpv;
+    lse2_out[t] = l2;
+    g_out[t] = g;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
 // Per-sequence bookkeeping around the row kernel.
 // ------------------------------------------------------------------------------------------------
 // valid-token count of each sequence, the total, and bad-id detection
@@ -689,6 +827,43 @@ int mrl_rows_finish(const MrlLossWs& w, long long N, const float* logp_old, cons
   return MRL_OK;
 }
 
+// Response-level ratio: loss terms, per-row gradient multipliers and log-sum-exps from the forward pass's per-row
+// triples, then the fixed-order sums.  Rows that no sequence covers keep g = 0 (the arrays are cleared first).
+int mrl_rows_finish_sequence(const MrlLossWs& w, long long N, int S, const int32_t* cu_seqlens, const float* adv_seq,
+                             const float* logp_old, const float* nll_weight, const mrl_loss_params* lp, float* logp,
+                             float* loss, int64_t* stats, float* g_out, float* lse2_out, cudaStream_t st) {
+  MRL_CUDA_OK(cudaMemsetAsync(w.pg_term, 0, (size_t)N * sizeof(double), st));
+  MRL_CUDA_OK(cudaMemsetAsync(w.nll_term, 0, (size_t)N * sizeof(double), st));
+  if (logp != nullptr) MRL_CUDA_OK(cudaMemsetAsync(logp, 0, (size_t)N * sizeof(float), st));
+  seq_ratio_kernel<<<S, 256, 0, st>>>(cu_seqlens, S, N, w.row_m2, w.row_s, w.row_zt, w.rowstat, w.seq_cnt, adv_seq,
+                                      logp_old, nll_weight, *lp, w.pg_term, w.nll_term, logp, g_out, lse2_out);
+  MRL_CUDA_OK(cudaGetLastError());
+  finalize_kernel<<<1, 1024, 0, st>>>(w.pg_term, w.nll_term, w.rowstat, N, w.totals, lp->flags, loss,
+                                      reinterpret_cast<long long*>(stats));
+  MRL_CUDA_OK(cudaGetLastError());
+  return MRL_OK;
+}
+
+namespace {
+int launch_rows_backward(const RowParams& p, int dtype, const float* g, const float* lse2, const float* zt,
+                         cudaStream_t st) {
+  if (p.N == 0) return MRL_OK;
+  const int words = pick_stream_words(p, dtype);
+  const unsigned n = (unsigned)p.N;
+  mrl_profile_before(st);
+  if (words == 8)
+    row_backward_stream_kernel<kStreamThreads, 4, 8><<<n, kStreamThreads, 0, st>>>(p, g, lse2, zt);
+  else if (words == 4)
+    row_backward_stream_kernel<kStreamThreads, 8, 4><<<n, kStreamThreads, 0, st>>>(p, g, lse2, zt);
+  else if (dtype == MRL_BF16)
+    row_backward_general_kernel<__nv_bfloat16><<<n, kThreads, 0, st>>>(p, g, lse2, zt);
+  else
+    row_backward_general_kernel<float><<<n, kThreads, 0, st>>>(p, g, lse2, zt);
+  mrl_profile_after(st);
+  return cudaGetLastError() == cudaSuccess ? MRL_OK : MRL_ERR_CUDA;
+}
+}  // namespace
+
 extern "C" int mrl_token_logprobs(const void* logits, int32_t dtype, int64_t N, int32_t V, int64_t ld,
                                   const int32_t* ids, const uint8_t* mask, float* logp, float* lse, int32_t* status,
                                   void* workspace, size_t workspace_bytes, void* stream) {
@@ -724,6 +899,8 @@ extern "C" int mrl_policy_loss_fwd_bwd(const void* logits, int32_t dtype, int64_
   if (dlogits != nullptr && ld_out < V) return MRL_ERR_INVALID_ARG;
   if (lp->agg_mode != MRL_AGG_TOKEN_MEAN && lp->agg_mode != MRL_AGG_SEQ_MEAN_TOKEN_MEAN) return MRL_ERR_INVALID_ARG;
   if (!(lp->eps_lo >= 0.f) || !(lp->eps_hi >= 0.f)) return MRL_ERR_INVALID_ARG;
+  if (lp->ratio_level != MRL_RATIO_TOKEN && lp->ratio_level != MRL_RATIO_SEQUENCE) return MRL_ERR_INVALID_ARG;
+  if (lp->ratio_level == MRL_RATIO_SEQUENCE && tok_weight != nullptr) return MRL_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool accum = lp->flags & MRL_FLAG_ACCUMULATE_LOSS;
   if (N == 0 || S == 0) {
@@ -765,6 +942,20 @@ extern "C" int mrl_policy_loss_fwd_bwd(const void* logits, int32_t dtype, int64_
   p.row_zt = w.row_zt;
   p.rowstat = w.rowstat;
   p.status = status;
+  if (lp->ratio_level == MRL_RATIO_SEQUENCE) {
+    // forward only (ratio one: no token-level clipping), then the responses' ratios, then the gradient launch
+    p.dlogits = nullptr;
+    p.logp_old = nullptr;
+    p.flags &= ~MRL_FLAG_SKIP_ZERO_ROWS;  // every valid row is needed for its response's sum
+    rc = launch_rows(p, dtype, st);
+    if (rc != MRL_OK) return rc;
+    // rows outside every sequence must come out with g = 0: the kernel below writes covered rows only
+    rc = mrl_rows_finish_sequence(w, N, S, cu_seqlens, adv_seq, logp_old, nll_weight, lp, logp, loss, stats, w.row_s,
+                                  w.row_m2, st);
+    if (rc != MRL_OK || dlogits == nullptr) return rc;
+    p.dlogits = dlogits;
+    return launch_rows_backward(p, dtype, w.row_s, w.row_m2, w.row_zt, st);
+  }
   rc = launch_rows(p, dtype, st);
   if (rc != MRL_OK) return rc;
   return mrl_rows_finish(w, N, logp_old, lp, logp, loss, stats, st);

@@ -24,15 +24,15 @@ def dev(t, dtype=None):
     return t.cuda().contiguous()
 
 
-def make_lp(eps_lo=0.2, eps_hi=0.2, agg=0, flags=0, pg_den=0.0, seq_den=0.0, nll_coeff=0.0):
-    return B.LossParams(eps_lo, eps_hi, agg, flags, pg_den, seq_den, nll_coeff, 0)
+def make_lp(eps_lo=0.2, eps_hi=0.2, agg=0, flags=0, pg_den=0.0, seq_den=0.0, nll_coeff=0.0, ratio_level=0):
+    return B.LossParams(eps_lo, eps_hi, agg, flags, pg_den, seq_den, nll_coeff, ratio_level)
 
 
 def oracle_lp(lp: B.LossParams) -> O.LossParams:
     # float32 parameters are upcast exactly, as the kernel sees them
     return O.LossParams(eps_lo=float(lp.eps_lo), eps_hi=float(lp.eps_hi), agg_mode=lp.agg_mode,
                         pg_denominator=lp.pg_denominator, seq_denominator=lp.seq_denominator,
-                        nll_coeff=float(lp.nll_coeff))
+                        nll_coeff=float(lp.nll_coeff), ratio_level=lp.ratio_level)
 
 
 def run_gpu_policy_loss(logits, ids, mask, cu, adv, logp_old, tok_weight, nll_weight, lp, V=None,
