@@ -21,6 +21,7 @@ Passages followed (by section / equation of the paper):
     all gated examples"                                                  (Sec. 5.3, App. B)
   * softmax score  grad log pi(a_i) = e_i - pi                            (App. H, proof of Prop. 1)
   * response-level ratio  w = exp(L_theta - L_behavior)                     (App. H, data-level coupling)
+  * policy entropy diagnostic  H_t = - sum_v p_v log p_v                   (Sec. 6, App. B: entropy curves)
   * THL word-level trace alignment  Z_w, C_w, Z_w / C_w                    (Sec. 4.2; App. D, Alg. 3; Thm. 1)
 
 Readings taken where the paper is silent are listed in the repository's
@@ -193,6 +194,27 @@ def token_logprobs(logits, ids, mask=None):
         tgt[a:a + _ROW_BLOCK] = z.gather(1, safe_ids[a:a + _ROW_BLOCK, None])[:, 0]
     logp = torch.where(valid, tgt - lse, torch.zeros_like(lse))
     return logp, lse, valid
+
+
+def token_entropy(logits, ids=None, mask=None):
+    """Entropy of the policy's next-token distribution at every row, H_t = - sum_v p_v log p_v with
+    p = softmax(z_t) -- the quantity behind the entropy diagnostics of Sec. 6 / App. B (Fig. 5, 6).
+    Evaluated as the definition; rows that are masked or have an out-of-range id give 0 (as for log-probs)."""
+    logits = torch.as_tensor(logits)
+    N, V = logits.shape
+    H = torch.empty(N, dtype=F64)
+    for a in range(0, N, _ROW_BLOCK):
+        z = logits[a:a + _ROW_BLOCK].to(F64)
+        logp = z - torch.logsumexp(z, dim=1, keepdim=True)
+        p = torch.exp(logp)
+        H[a:a + _ROW_BLOCK] = -(torch.where(p > 0, p * logp, torch.zeros_like(p))).sum(dim=1)
+    valid = torch.ones(N, dtype=torch.bool)
+    if ids is not None:
+        ids = torch.as_tensor(ids).long()
+        valid &= (ids >= 0) & (ids < V)
+    if mask is not None:
+        valid &= torch.as_tensor(mask) != 0
+    return torch.where(valid, H, torch.zeros_like(H))
 
 
 @dataclass
