@@ -139,7 +139,7 @@ def barrier(world: int):
 class LogitsInWorkload:
     """Config 2: 8 prompts x G = 8, ragged lengths in [128, 1024] packed, V = 151,936, bf16 logits."""
 
-    def __init__(self, w: synth.Workload, seed: int, device, ratio_level: int = 0):
+    def __init__(self, w: synth.Workload, seed: int, device, ratio_level: int = 0, with_entropy: bool = False):
         from paper_2605_07244_b200 import binding as B
         self.B = B
         self.w = w
@@ -176,6 +176,9 @@ class LogitsInWorkload:
         # behaviour trace: logp_old = logp + N(0, 0.1); logp from the library's forward (input preparation).
         # For the response-level ratio the noise is scaled by 1 / sqrt(mean length) so that w stays of order one.
         B.mrl_token_logprobs(self.z, self.ids, None, self.logp)
+        if with_entropy:     # the policy-entropy diagnostic from the same pass
+            self.entropy = torch.empty(self.N, device=dev)
+            self.lp.entropy = self.entropy.data_ptr()
         scale = 1.0 if ratio_level == 0 else (self.S / max(self.N, 1)) ** 0.5
         self.logp_old = self.logp + b.noise.to(dev) * scale
         torch.cuda.synchronize()
@@ -204,6 +207,7 @@ class LogitsInWorkload:
                             "GRPO group z-norm, eps 0.2",
                 "rows": self.N, "sequences": self.S, "V": self.V, "logits_dtype": "bf16",
                 "ratio_level": "token" if self.ratio_level == 0 else "response (App. H)",
+                "entropy_output": bool(self.lp.entropy),
                 "l2": "inputs (%.1f GB logits) exceed the 126 MB L2; no flush needed" % (self.z.numel() * 2 / 1e9)}
 
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region
@@ -553,7 +557,8 @@ def run_ours(args, rank, world, local_rank):
     lmhead_main = args.workload in ("C5", "C5s")
     cls = LmheadWorkload if lmhead_main else LogitsInWorkload
     wl = (cls(synth.CONFIGS[args.workload], args.seed + rank, device) if lmhead_main else
-          cls(synth.CONFIGS[args.workload], args.seed + rank, device, 1 if args.ratio_level == "sequence" else 0))
+          cls(synth.CONFIGS[args.workload], args.seed + rank, device, 1 if args.ratio_level == "sequence" else 0,
+              args.with_entropy))
     res = measure(wl, args.steps, args.warmup, world, local_rank, rank, peaks, not args.no_e2e,
                   not args.no_cpu_baseline, args)
     del wl
@@ -600,6 +605,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="profiling runs only: skip the host-buffer leg")
     ap.add_argument("--ratio-level", default="token", choices=["token", "sequence"],
                     help="logits-in workloads: importance ratio per token (Eq. (1), default) or per response (App. H)")
+    ap.add_argument("--with-entropy", action="store_true", help="logits-in workloads: also emit the per-row policy entropy")
     ap.add_argument("--no-lmhead", action="store_true", help="skip the short config-5 leg of the default run")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))

@@ -38,7 +38,7 @@
 extern "C" {
 #endif
 
-#define MRL_VERSION 100
+#define MRL_VERSION 101
 
 /* return codes */
 #define MRL_OK 0
@@ -117,6 +117,10 @@ typedef struct mrl_loss_params {
   double seq_denominator;   /* SEQ_MEAN_TOKEN_MEAN: number of sequences of the whole step; <= 0: S */
   float nll_coeff;          /* lambda_SGT / n_gated (Eq. (2), App. B); 0 disables the NLL term */
   int32_t ratio_level;      /* MRL_RATIO_*; 0 (token level) is the default */
+  float* entropy;           /* [device] float32 [N], nullable.  mrl_policy_loss_fwd_bwd only (must be NULL for the
+                               fused LM head): entropy - sum_v p_v log p_v of softmax(z_t) at every valid row, 0
+                               elsewhere -- the policy-entropy diagnostic of Sec. 6 / App. B, taken from the same
+                               pass over the logits (one more FMA per logit) */
 } mrl_loss_params;
 
 /*

@@ -38,7 +38,7 @@ class AdvParams(C.Structure):
 class LossParams(C.Structure):
     _fields_ = [("eps_lo", C.c_float), ("eps_hi", C.c_float), ("agg_mode", C.c_int32),
                 ("flags", C.c_uint32), ("pg_denominator", C.c_double), ("seq_denominator", C.c_double),
-                ("nll_coeff", C.c_float), ("ratio_level", C.c_int32)]
+                ("nll_coeff", C.c_float), ("ratio_level", C.c_int32), ("entropy", C.c_void_p)]
 
 
 class MrlError(RuntimeError):

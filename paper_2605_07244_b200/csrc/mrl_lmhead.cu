@@ -769,6 +769,7 @@ extern "C" int mrl_fused_lmhead_loss_fwd_bwd(const void* hidden, const void* W, 
   if (!(lp->eps_lo >= 0.f) || !(lp->eps_hi >= 0.f)) return MRL_ERR_INVALID_ARG;
   if (lp->ratio_level != MRL_RATIO_TOKEN && lp->ratio_level != MRL_RATIO_SEQUENCE) return MRL_ERR_INVALID_ARG;
   if (lp->ratio_level == MRL_RATIO_SEQUENCE && tok_weight != nullptr) return MRL_ERR_INVALID_ARG;
+  if (lp->entropy != nullptr) return MRL_ERR_INVALID_ARG;  // the entropy diagnostic is a logits-in output
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool accum_loss = lp->flags & MRL_FLAG_ACCUMULATE_LOSS;
   const bool accum_dw = lp->flags & MRL_FLAG_ACCUMULATE_DW;

@@ -35,6 +35,7 @@ struct RowParams {
   int loss_mode;  // 0: log-probs only, 1: loss (+ gradient when dlogits != null)
   float* logp;
   float* lse;
+  float* entropy;  // nullable: per-row entropy of softmax(z_t) (diagnostic)
   float* row_m2;  // loss mode: per-row (max, sum, target) of the base-2 log-sum-exp, finished in float64 later
   float* row_s;
   float* row_zt;
@@ -177,12 +178,12 @@ __device__ __forceinline__ StreamVec<kWords> stream_fill(uint32_t x) {
 
 // kC = 1: the CTA takes the whole row.  kC = 2: a cluster of two CTAs takes the row, half each, and the halves'
 // (max, sum, target logit) cross through distributed shared memory: a remote store plus a remote mbarrier arrive.
-template <int kT, int kU, int kWords, int kC>
+template <int kT, int kU, int kWords, int kC, bool kEnt>
 __global__ void __launch_bounds__(kT, 1024 / kT) row_stream_kernel(const RowParams p) {
   constexpr int kWarpsT = kT / 32;
   constexpr int kVecBytes = kWords * 4, kVecElems = kWords * 2;
   using Vec = StreamVec<kWords>;
-  __shared__ float red[2 * 32];
+  __shared__ float red[3 * 32];
   __shared__ float fin[4];
   __shared__ __align__(16) float4 xchg[2];
   __shared__ __align__(8) uint64_t xbar;
@@ -203,7 +204,10 @@ __global__ void __launch_bounds__(kT, 1024 / kT) row_stream_kernel(const RowPara
   if (ctx.dead) {
     if (orow != nullptr)
       for (int i = tid; i < nvec; i += kT) stream_st<kWords>(out + (size_t)(i - tid) * kVecBytes, stream_fill<kWords>(0u));
-    if (rank == 0 && tid == 0) write_row_scalars(p, row, ctx, 0.f, 0.f, mrl::lse2_empty(), 0.f, false, false);
+    if (rank == 0 && tid == 0) {
+      write_row_scalars(p, row, ctx, 0.f, 0.f, mrl::lse2_empty(), 0.f, false, false);
+      if (kEnt) p.entropy[row] = 0.f;
+    }
     return;  // both CTAs of a cluster take this branch: no cluster barrier is left waiting
   }
   if (kC > 1) {
@@ -221,7 +225,7 @@ __global__ void __launch_bounds__(kT, 1024 / kT) row_stream_kernel(const RowPara
   if (tid == 0 && owner) zt = __bfloat162float(grow[rel]);         // before anything is written in place
 
   // ---- pass 1: running (max, sum) in the base-2 domain
-  float m_run = -INFINITY, s_run = 0.f;
+  float m_run = -INFINITY, s_run = 0.f, u_run = 0.f;  // u: sum of 2^(x - m) z, for the entropy (kEnt only)
   for (int base = 0; base < nvec; base += kT * kU) {
     Vec v[kU];
     if (base + kT * kU <= nvec) {
@@ -242,33 +246,47 @@ __global__ void __launch_bounds__(kT, 1024 / kT) row_stream_kernel(const RowPara
     const float vmax = fmaxf(mrl::bf16lo_to_f32(mx), mrl::bf16hi_to_f32(mx));
     const float m_new = fmaxf(m_run, vmax * MRL_LOG2E);
     if (m_new > m_run) {  // also the first group (m_run = -inf, s_run = 0)
-      s_run *= mrl::ex2_approx(m_run - m_new);
+      const float f = mrl::ex2_approx(m_run - m_new);
+      s_run *= f;
+      if (kEnt) u_run *= f;
       m_run = m_new;
     }
     if (m_run != -INFINITY) {
       const float neg_m = -m_run;
-      float s0 = 0.f, s1 = 0.f;
+      float s0 = 0.f, s1 = 0.f, u0 = 0.f, u1 = 0.f;
 #pragma unroll
       for (int u = 0; u < kU; ++u) {
 #pragma unroll
         for (int j = 0; j < kWords; ++j) {
-          s0 += mrl::ex2_approx(fmaf(mrl::bf16lo_to_f32(v[u].w[j]), MRL_LOG2E, neg_m));
-          s1 += mrl::ex2_approx(fmaf(mrl::bf16hi_to_f32(v[u].w[j]), MRL_LOG2E, neg_m));
+          const float zlo = mrl::bf16lo_to_f32(v[u].w[j]), zhi = mrl::bf16hi_to_f32(v[u].w[j]);
+          const float a = mrl::ex2_approx(fmaf(zlo, MRL_LOG2E, neg_m)), b = mrl::ex2_approx(fmaf(zhi, MRL_LOG2E, neg_m));
+          s0 += a;
+          s1 += b;
+          if (kEnt) {  // a = 0 exactly where z = -inf: keep 0 * inf out of the sum
+            u0 = a != 0.f ? fmaf(a, zlo, u0) : u0;
+            u1 = b != 0.f ? fmaf(b, zhi, u1) : u1;
+          }
         }
       }
       s_run += s0 + s1;
+      if (kEnt) u_run += u0 + u1;
     }
   }
   // ---- block totals: maximum first, one rescale, then a plain sum (fixed order: reproducible)
   float m = m_run;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-  float sum = m_run != -INFINITY ? s_run * mrl::ex2_approx(m_run - m) : 0.f;
+  const float rescale = m_run != -INFINITY ? mrl::ex2_approx(m_run - m) : 0.f;
+  float sum = s_run * rescale, usum = kEnt ? u_run * rescale : 0.f;
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+  for (int o = 16; o > 0; o >>= 1) {
+    sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    if (kEnt) usum += __shfl_xor_sync(0xffffffffu, usum, o);
+  }
   if (lane == 0) {
     red[warp] = m;
     red[32 + warp] = sum;
+    if (kEnt) red[64 + warp] = usum;
   }
   __syncthreads();
   if (warp == 0) {
@@ -276,9 +294,13 @@ __global__ void __launch_bounds__(kT, 1024 / kT) row_stream_kernel(const RowPara
     float tm = wm;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) tm = fmaxf(tm, __shfl_xor_sync(0xffffffffu, tm, o));
-    float ts = wm != -INFINITY ? ws * mrl::ex2_approx(wm - tm) : 0.f;
+    const float wscale = wm != -INFINITY ? mrl::ex2_approx(wm - tm) : 0.f;
+    float ts = ws * wscale, tu = (kEnt && lane < kWarpsT) ? red[64 + lane] * wscale : 0.f;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) ts += __shfl_xor_sync(0xffffffffu, ts, o);
+    for (int o = 16; o > 0; o >>= 1) {
+      ts += __shfl_xor_sync(0xffffffffu, ts, o);
+      if (kEnt) tu += __shfl_xor_sync(0xffffffffu, tu, o);
+    }
     bool ok = true;
     if (kC > 1) {
       asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");  // the peer's barrier is initialised
@@ -319,6 +341,7 @@ __global__ void __launch_bounds__(kT, 1024 / kT) row_stream_kernel(const RowPara
         }
       }
       if (rank == 0 && ok) write_row_scalars(p, row, ctx, logp, ctx.valid ? lse : 0.f, mrl::Lse2{tm, ts}, zt, clipped, true);
+      if (kEnt) p.entropy[row] = ctx.valid ? lse - tu / ts : 0.f;  // H = lse - sum_v p_v z_v
       fin[0] = lse2;
       fin[1] = g;
       fin[2] = g * (mrl::ex2_approx(fmaf(zt, MRL_LOG2E, -lse2)) - 1.0f);
@@ -390,7 +413,10 @@ __global__ void __launch_bounds__(kThreads) row_general_kernel(const RowParams p
   if (ctx.dead) {
     if (dz != nullptr)
       for (int v = tid; v < p.V; v += kThreads) st_from_f32<T>(dz + v, 0.f);
-    if (tid == 0) write_row_scalars(p, row, ctx, 0.f, 0.f, mrl::lse2_empty(), 0.f, false, false);
+    if (tid == 0) {
+      write_row_scalars(p, row, ctx, 0.f, 0.f, mrl::lse2_empty(), 0.f, false, false);
+      if (p.entropy != nullptr) p.entropy[row] = 0.f;
+    }
     return;
   }
   const float zt = ld_as_f32<T>(z + ctx.id);  // before any in-place write
@@ -415,6 +441,25 @@ __global__ void __launch_bounds__(kThreads) row_general_kernel(const RowParams p
     clipped = ro.clipped;
   }
   if (tid == 0) write_row_scalars(p, row, ctx, logp, lse, tot, zt, clipped, true);
+  if (p.entropy != nullptr) {  // H = lse - sum_v p_v z_v, p_v = 2^(z_v log2e - lse2)
+    float u = 0.f;
+    for (int v = tid; v < p.V; v += kThreads) {
+      const float zv = ld_as_f32<T>(z + v);
+      const float pv = mrl::ex2_approx(fmaf(zv, MRL_LOG2E, -lse2));
+      u = pv != 0.f ? fmaf(pv, zv, u) : u;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) u += __shfl_xor_sync(0xffffffffu, u, o);
+    __syncthreads();
+    if ((tid & 31) == 0) scratch[tid >> 5] = u;
+    __syncthreads();
+    if (tid == 0) {
+      float t = 0.f;
+      for (int k = 0; k < kThreads / 32; ++k) t += scratch[k];
+      p.entropy[row] = lse - t;
+    }
+    __syncthreads();
+  }
   if (dz == nullptr) return;
   if (g == 0.f) {
     for (int v = tid; v < p.V; v += kThreads) st_from_f32<T>(dz + v, 0.f);
@@ -764,7 +809,9 @@ int launch_rows(RowParams p, int dtype, cudaStream_t st) {
   // Two CTAs per SM stream one row each, or -- for rows so long that two rows per SM would be evicted from L2
   // before the second pass reads them back -- the two halves of one row as a cluster of two.  (At 300 KB rows the
   // split reads HBM 1.01x instead of 1.34x but is 4 % slower: its per-CTA fixed work is spread over half the bytes.)
-  const bool split = (long long)p.V * 2 >= kSplitRowBytes && p.N <= 0x3fffffffll;
+  // (the entropy diagnostic is carried by the whole-row variant only)
+  const bool split = (long long)p.V * 2 >= kSplitRowBytes && p.N <= 0x3fffffffll && p.entropy == nullptr;
+  const bool ent = p.entropy != nullptr;
   const int C = split ? 2 : 1;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(n * (unsigned)C);
@@ -781,11 +828,13 @@ int launch_rows(RowParams p, int dtype, cudaStream_t st) {
   mrl_profile_before(st);
   cudaError_t e;
   if (words == 8)
-    e = split ? cudaLaunchKernelEx(&cfg, row_stream_kernel<kStreamThreads, 4, 8, 2>, p)
-              : cudaLaunchKernelEx(&cfg, row_stream_kernel<kStreamThreads, 4, 8, 1>, p);
+    e = split ? cudaLaunchKernelEx(&cfg, row_stream_kernel<kStreamThreads, 4, 8, 2, false>, p)
+        : ent ? cudaLaunchKernelEx(&cfg, row_stream_kernel<kStreamThreads, 4, 8, 1, true>, p)
+              : cudaLaunchKernelEx(&cfg, row_stream_kernel<kStreamThreads, 4, 8, 1, false>, p);
   else
-    e = split ? cudaLaunchKernelEx(&cfg, row_stream_kernel<kStreamThreads, 8, 4, 2>, p)
-              : cudaLaunchKernelEx(&cfg, row_stream_kernel<kStreamThreads, 8, 4, 1>, p);
+    e = split ? cudaLaunchKernelEx(&cfg, row_stream_kernel<kStreamThreads, 8, 4, 2, false>, p)
+        : ent ? cudaLaunchKernelEx(&cfg, row_stream_kernel<kStreamThreads, 8, 4, 1, true>, p)
+              : cudaLaunchKernelEx(&cfg, row_stream_kernel<kStreamThreads, 8, 4, 1, false>, p);
   mrl_profile_after(st);
   return e == cudaSuccess ? MRL_OK : MRL_ERR_CUDA;
 }
@@ -937,6 +986,7 @@ extern "C" int mrl_policy_loss_fwd_bwd(const void* logits, int32_t dtype, int64_
   p.eps_hi = lp->eps_hi;
   p.flags = lp->flags;
   p.loss_mode = 1;
+  p.entropy = lp->entropy;
   p.row_m2 = w.row_m2;
   p.row_s = w.row_s;
   p.row_zt = w.row_zt;
