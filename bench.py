@@ -454,22 +454,33 @@ def run_reference(args, rank, world):
     w = synth.CONFIGS[args.workload]
     meta = synth.make_meta(w, args.seed)
     batch = synth.make_batch(meta)
-    n_seq = 1
-    while int(batch.cu_seqlens[n_seq]) < REFERENCE_ROWS and n_seq < batch.S:
-        n_seq += 1
-    n = int(batch.cu_seqlens[n_seq])
-    z = batch.logits_rows(0, n)
     adv, _ = O.group_advantages(meta.rewards)
-    adv_seq = adv[batch.seq_p.long(), batch.seq_m.long(), batch.seq_g.long()][:n_seq]
-    logp, _, _ = O.token_logprobs(z, batch.ids[:n])
-    logp_old = (logp + batch.noise[:n].double()).float()
-    call = (z, batch.ids[:n], None, batch.cu_seqlens[:n_seq + 1], adv_seq, logp_old)
+    if w.H > 0:      # hidden-in workloads: the oracle's float64 LM head on a few sequences, full V and H
+        n_seq = max(1, LMHEAD_ORACLE_ROWS // int(batch.cu_seqlens[1]))
+        n = int(batch.cu_seqlens[n_seq])
+        hidden, W = batch.hidden_rows(0, n), batch.lm_head()
+        adv_seq = adv[batch.seq_p.long(), batch.seq_m.long(), batch.seq_g.long()][:n_seq]
+        logp, _, _ = O.token_logprobs(hidden.double() @ W.double().T, batch.ids[:n])
+        logp_old = (logp + batch.noise[:n].double()).float()
+        call = (hidden, W, batch.ids[:n], None, batch.cu_seqlens[:n_seq + 1], adv_seq, logp_old)
+        run_once = lambda: O.fused_lmhead_loss(*call, None, None, O.LossParams())
+    else:
+        n_seq = 1
+        while int(batch.cu_seqlens[n_seq]) < REFERENCE_ROWS and n_seq < batch.S:
+            n_seq += 1
+        n = int(batch.cu_seqlens[n_seq])
+        z = batch.logits_rows(0, n)
+        adv_seq = adv[batch.seq_p.long(), batch.seq_m.long(), batch.seq_g.long()][:n_seq]
+        logp, _, _ = O.token_logprobs(z, batch.ids[:n])
+        logp_old = (logp + batch.noise[:n].double()).float()
+        call = (z, batch.ids[:n], None, batch.cu_seqlens[:n_seq + 1], adv_seq, logp_old)
+        run_once = lambda: O.policy_loss(*call, None, None, O.LossParams())
     for _ in range(min(args.warmup, 1)):
-        O.policy_loss(*call, None, None, O.LossParams())
+        run_once()
     t0 = time.perf_counter()
     for _ in range(args.steps):
         O.group_advantages(meta.rewards)
-        O.policy_loss(*call, None, None, O.LossParams())
+        run_once()
     dt = time.perf_counter() - t0
     value = n * args.steps / dt
     cores = torch.get_num_threads()
@@ -478,7 +489,7 @@ def run_reference(args, rank, world):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "rows_per_step": n, "V": w.V},
+        "config": {"workload": w.name, "rows_per_step": n, "V": w.V, "H": w.H},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
