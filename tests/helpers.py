@@ -1,5 +1,5 @@
 """Shared plumbing of the GPU parity tests: run the C ABI on one set of inputs, run the oracle on the
-same inputs, compare.  Tolerances are the ones the task states: ids / masks / gate outputs bit-exact,
+same inputs, compare.  Tolerances: ids / masks / gate outputs bit-exact,
 log-probs 1e-4 absolute, loss 1e-5 relative, bf16 gradients 1e-2 relative L2 (fp32 gradients 1e-5)."""
 from __future__ import annotations
 
