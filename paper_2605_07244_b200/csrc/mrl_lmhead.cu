@@ -1,11 +1,12 @@
 // Hidden-in path (fused LM head): mrl_fused_lmhead_loss_fwd_bwd.
 //
-// Every product of the pass is a "TN" GEMM  C[M, N] = A[M, K] * B[N, K]^T  (both operands K-major, bf16, fp32
-// accumulation) on one persistent tcgen05 kernel, specialised by its epilogue:
+// Every product of the pass is  C[M, N] = A B^T  (bf16 operands, fp32 accumulation) on one persistent tcgen05
+// kernel, specialised by its epilogue and by how each operand lies in memory (K-major, or MN-major = given as the
+// [K, M] / [K, N] matrix, so that nothing ever has to be transposed in memory):
 //   forward    z = hidden W^T, tile by tile; the epilogue folds each tile into per-row (max, sum 2^x) partials and
 //              picks the target logit; the [N, V] logits are never stored
-//   backward   per vocabulary chunk: recompute the z tile, write D = g (softmax - onehot) in bf16 as D[N, Vc] and
-//              D^T[Vc, N]; dHidden (+)= D (W^T)^T; dW[chunk] = D^T (hidden^T)^T
+//   backward   per vocabulary chunk: recompute the z tile, write D = g (softmax - onehot) in bf16 as D[N, Vc];
+//              dHidden (+)= D W_chunk  (W_chunk enters MN-major);  dW[chunk] = D^T hidden  (both enter MN-major)
 // Kernel anatomy (one CTA per SM, 192 threads): warp 0 feeds a shared-memory ring with TMA tile loads
 // (128-byte swizzle, no multicast), one thread of warp 1 issues tcgen05.mma into one of two TMEM accumulators,
 // warps 2..5 drain the other accumulator with tcgen05.ld while the next tile's MMAs run.  Every mbarrier wait is
@@ -53,8 +54,6 @@ struct GemmParams {
   const float* lse2;      // [M] log2 sum_v 2^(z log2 e)
   __nv_bfloat16* D;       // [M, ldD]
   long long ldD;
-  __nv_bfloat16* DT;      // [N, ldDT]
-  long long ldDT;
   // EPI_STORE
   void* C;                // bf16 or fp32 [M, ldc]
   float* Cacc;            // fp32 [M, ldacc] running sum (C_BF16_FROM_ACC reads it, C_F32 / C_F32_ADD write C)
@@ -177,10 +176,24 @@ __device__ __forceinline__ uint64_t smem_desc_k128(uint32_t addr) {
   d |= (uint64_t)2 << 61;                    // SWIZZLE_128B
   return d;
 }
-// kind::f16 instruction descriptor: fp32 accumulator, bf16 x bf16, both K-major, N = 256, M = 128 per CTA
-template <int kC>
-constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) |
-                            ((uint32_t)((BM * kC) >> 4) << 24);
+// The same for an MN-major tile: the operand is stored with its M (or N) index contiguous, and the TMA brings it in as
+// boxes of 64 such elements (128 bytes) by BK rows of K.  Inside a box, 8 K-rows of 128 bytes form one swizzle atom
+// (1024 bytes apart: the stride byte offset); boxes of consecutive groups of 64 follow each other BK * 128 bytes
+// apart (the leading byte offset).  One MMA step of K = 16 is two atoms: + 2048 bytes in the start address.
+__device__ __forceinline__ uint64_t smem_desc_mn128(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3ffffu) >> 4);
+  d |= (uint64_t)((BK * 128) >> 4) << 16;     // leading byte offset: next group of 64 along M / N
+  d |= (uint64_t)(1024 >> 4) << 32;           // stride byte offset: next group of 8 along K
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+// kind::f16 instruction descriptor: fp32 accumulator, bf16 x bf16, N = 256, M = 128 per CTA
+// (bits 15 / 16: A / B is MN-major)
+template <int kC, bool kAMn, bool kBMn>
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((kAMn ? 1u : 0u) << 15) | ((kBMn ? 1u : 0u) << 16) |
+                            ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((BM * kC) >> 4) << 24);
 
 // tile t -> (row-tile, column-tile): row-tiles run fastest inside a group of group_m, so that the CTAs of one wave
 // share a handful of A and B tiles
@@ -244,7 +257,8 @@ __device__ __forceinline__ void store_bf16x32(__nv_bfloat16* dst, const float* d
 }
 
 // ------------------------------------------------------------------------------------------ the GEMM kernel
-template <int EPI, int kC>
+// kAMn / kBMn: the operand is stored MN-major (its M / N index contiguous, K strided) instead of K-major.
+template <int EPI, int kC, bool kAMn, bool kBMn>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
                    const GemmParams p) {
@@ -316,16 +330,24 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
         for (int kb = 0; kb < p.k_blocks; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t a_dst = tiles + (uint32_t)stage * kStageBytes;
-          if (kC == 2) {
-            // the leader's barrier counts the bytes of both CTAs; only the leader arms it
-            const uint32_t lead_full = mapa_u32(full_bar(stage), 0u);
-            if (rank == 0) mbar_expect_tx(full_bar(stage), 2u * kStageBytes);
-            tma_load_2d_pair(a_dst, &tmapA, kb * BK, a_row, lead_full);
-            tma_load_2d_pair(a_dst + kABytes, &tmapB, kb * BK, b_row, lead_full);
+          // the leader's barrier counts the bytes of both CTAs of a pair; only the leader arms it
+          const uint32_t bar = kC == 2 ? mapa_u32(full_bar(stage), 0u) : full_bar(stage);
+          if (rank == 0) mbar_expect_tx(full_bar(stage), (uint32_t)kC * kStageBytes);
+          auto load = [&](uint32_t dst, const CUtensorMap* map, int x, int y) {
+            if (kC == 2) tma_load_2d_pair(dst, map, x, y, bar); else tma_load_2d(dst, map, x, y, bar);
+          };
+          if (kAMn) {  // boxes of 64 rows-of-the-tile x BK
+#pragma unroll
+            for (int j = 0; j < BM / 64; ++j) load(a_dst + (uint32_t)j * (BK * 128), &tmapA, a_row + 64 * j, kb * BK);
           } else {
-            mbar_expect_tx(full_bar(stage), kStageBytes);
-            tma_load_2d(a_dst, &tmapA, kb * BK, a_row, full_bar(stage));
-            tma_load_2d(a_dst + kABytes, &tmapB, kb * BK, b_row, full_bar(stage));
+            load(a_dst, &tmapA, kb * BK, a_row);
+          }
+          if (kBMn) {
+#pragma unroll
+            for (int j = 0; j < Cfg::kBRows / 64; ++j)
+              load(a_dst + kABytes + (uint32_t)j * (BK * 128), &tmapB, b_row + 64 * j, kb * BK);
+          } else {
+            load(a_dst + kABytes, &tmapB, kb * BK, b_row);
           }
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
@@ -345,13 +367,16 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
           if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
           tc_fence_after();
           const uint32_t a_src = tiles + (uint32_t)stage * kStageBytes;
-          const uint64_t adesc = smem_desc_k128(a_src), bdesc = smem_desc_k128(a_src + kABytes);
+          const uint64_t adesc = kAMn ? smem_desc_mn128(a_src) : smem_desc_k128(a_src);
+          const uint64_t bdesc = kBMn ? smem_desc_mn128(a_src + kABytes) : smem_desc_k128(a_src + kABytes);
+          // one step of K = 16: 32 bytes along a K-major swizzle row, two 1024-byte atoms of an MN-major tile
+          constexpr uint64_t a_step = kAMn ? (2048 >> 4) : 2, b_step = kBMn ? (2048 >> 4) : 2;
 #pragma unroll
-          for (int k = 0; k < BK / UMMA_K; ++k) {  // 32 bytes along K inside the swizzle row: +2 in 16-byte units
+          for (int k = 0; k < BK / UMMA_K; ++k) {
             if (kC == 2)
-              tc_mma_pair(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), kIdesc<kC>, (kb | k) != 0);
+              tc_mma_pair(d_tmem, adesc + a_step * k, bdesc + b_step * k, kIdesc<kC, kAMn, kBMn>, (kb | k) != 0);
             else
-              tc_mma(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), kIdesc<kC>, (kb | k) != 0);
+              tc_mma(d_tmem, adesc + a_step * k, bdesc + b_step * k, kIdesc<kC, kAMn, kBMn>, (kb | k) != 0);
           }
           // the stage is free (in both CTAs) once these MMAs have read it
           if (kC == 2) tc_commit_pair(empty_bar(stage), 3); else tc_commit(empty_bar(stage));
@@ -417,9 +442,6 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
           if (row_ok) {
             const int nvalid = ncols_valid - c;
             store_bf16x32(p.D + (long long)row * p.ldD + (long long)n * BN + c, d, nvalid);
-#pragma unroll
-            for (int j = 0; j < 32; ++j)  // a warp writes 32 consecutive rows of one column: 64 contiguous bytes
-              if (j < nvalid) p.DT[(long long)(n * BN + c + j) * p.ldDT + row] = __float2bfloat16_rn(d[j]);
           }
         } else {
           if (row_ok) {
@@ -505,24 +527,6 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
 }
 
 // ------------------------------------------------------------------------------------------ small kernels
-// out[c, r] = in[r, c]; in [R, ld_in], out [C, ld_out]
-__global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16* __restrict__ in, long long R,
-                                                              long long C, long long ld_in,
-                                                              __nv_bfloat16* __restrict__ out, long long ld_out) {
-  __shared__ __nv_bfloat16 tile[64][66];
-  const long long r0 = (long long)blockIdx.y * 64, c0 = (long long)blockIdx.x * 64;
-  const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;
-  for (int i = ty; i < 64; i += 4) {
-    const long long r = r0 + i, c = c0 + tx;
-    tile[i][tx] = (r < R && c < C) ? in[r * ld_in + c] : __float2bfloat16(0.f);
-  }
-  __syncthreads();
-  for (int i = ty; i < 64; i += 4) {
-    const long long c = c0 + i, r = r0 + tx;
-    if (c < C && r < R) out[c * ld_out + r] = tile[tx][i];
-  }
-}
-
 // Merges the per-tile partials of every row in tile order, then the row's ratio / clip / gradient multiplier.
 __global__ void __launch_bounds__(256) lmhead_rows_kernel(long long N, int V, int n_tiles, const float2* __restrict__ partial,
                                                            long long part_ld, const float* __restrict__ zt,
@@ -615,7 +619,7 @@ int sm_count() {
 }
 
 // CTA pairs of the two-CTA kernel that can be resident together on the current device (0: use single CTAs).
-template <int EPI>
+template <int EPI, bool kAMn, bool kBMn>
 int resident_pairs(cudaLaunchConfig_t* cfg) {
   static int cache[64] = {};
   int dev = 0;
@@ -623,7 +627,7 @@ int resident_pairs(cudaLaunchConfig_t* cfg) {
   if (cacheable && cache[dev] != 0) return cache[dev] > 0 ? cache[dev] : 0;
   cfg->gridDim = dim3((unsigned)(sm_count() / 2 * 2));
   int n = 0;
-  if (cudaOccupancyMaxActiveClusters(&n, lmhead_gemm_kernel<EPI, 2>, cfg) != cudaSuccess || n < 1) {
+  if (cudaOccupancyMaxActiveClusters(&n, lmhead_gemm_kernel<EPI, 2, kAMn, kBMn>, cfg) != cudaSuccess || n < 1) {
     (void)cudaGetLastError();
     n = 0;
   }
@@ -631,14 +635,16 @@ int resident_pairs(cudaLaunchConfig_t* cfg) {
   return n;
 }
 
-template <int EPI>
+// C[M, N] = A B^T.  A K-major operand is a row-major [rows = M or N, K] matrix; an MN-major one is a row-major
+// [K, rows] matrix (what the other one would be transposed), `ld` elements between its rows either way.
+template <int EPI, bool kAMn, bool kBMn>
 int launch_gemm(const void* A, long long lda, const void* B, long long ldb, GemmParams p, bool pair_tiles,
                 cudaStream_t st) {
   if (p.M <= 0 || p.N <= 0 || p.K <= 0) return MRL_OK;
   p.n_tiles = (p.N + BN - 1) / BN;
   p.k_blocks = (p.K + BK - 1) / BK;
   // two-CTA tiles (256 rows) when asked for and pairs can be scheduled, else one CTA per 128-row tile
-  MRL_CUDA_OK(cudaFuncSetAttribute(lmhead_gemm_kernel<EPI, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  MRL_CUDA_OK(cudaFuncSetAttribute(lmhead_gemm_kernel<EPI, 2, kAMn, kBMn>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    (int)GemmCfg<2>::kSmem));
   cudaLaunchConfig_t cfg = {};
   cfg.blockDim = dim3(kGemmThreads);
@@ -651,12 +657,13 @@ int launch_gemm(const void* A, long long lda, const void* B, long long ldb, Gemm
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  const int pairs = pair_tiles ? resident_pairs<EPI>(&cfg) : 0;
+  const int pairs = pair_tiles ? resident_pairs<EPI, kAMn, kBMn>(&cfg) : 0;
   const int kC = pairs > 0 ? 2 : 1;
   CUtensorMap ta, tb;
-  int rc = make_tmap(&ta, A, p.M, p.K, lda, BM);
+  // K-major: tiles of [box rows x 64 of K]; MN-major: boxes of [64 of K rows x 64 of M / N]
+  int rc = kAMn ? make_tmap(&ta, A, p.K, p.M, lda, BK) : make_tmap(&ta, A, p.M, p.K, lda, BM);
   if (rc != MRL_OK) return rc;
-  rc = make_tmap(&tb, B, p.N, p.K, ldb, BN / kC);
+  rc = kBMn ? make_tmap(&tb, B, p.K, p.N, ldb, BK) : make_tmap(&tb, B, p.N, p.K, ldb, BN / kC);
   if (rc != MRL_OK) return rc;
   p.m_tiles = (p.M + BM * kC - 1) / (BM * kC);
   // rows of A per raster group: a wave's operands should share L2; with a short K a taller group re-uses A
@@ -668,26 +675,16 @@ int launch_gemm(const void* A, long long lda, const void* B, long long ldb, Gemm
     const long long units = tiles < pairs ? tiles : pairs;
     cfg.gridDim = dim3((unsigned)(2 * units));
     mrl_profile_before(st);
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, lmhead_gemm_kernel<EPI, 2>, ta, tb, p);
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, lmhead_gemm_kernel<EPI, 2, kAMn, kBMn>, ta, tb, p);
     mrl_profile_after(st);
     return e == cudaSuccess ? MRL_OK : MRL_ERR_CUDA;
   }
   const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
-  MRL_CUDA_OK(cudaFuncSetAttribute(lmhead_gemm_kernel<EPI, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  MRL_CUDA_OK(cudaFuncSetAttribute(lmhead_gemm_kernel<EPI, 1, kAMn, kBMn>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    (int)GemmCfg<1>::kSmem));
   mrl_profile_before(st);
-  lmhead_gemm_kernel<EPI, 1><<<grid, kGemmThreads, GemmCfg<1>::kSmem, st>>>(ta, tb, p);
+  lmhead_gemm_kernel<EPI, 1, kAMn, kBMn><<<grid, kGemmThreads, GemmCfg<1>::kSmem, st>>>(ta, tb, p);
   mrl_profile_after(st);
-  MRL_CUDA_OK(cudaGetLastError());
-  return MRL_OK;
-}
-
-int launch_transpose(const __nv_bfloat16* in, long long R, long long C, long long ld_in, __nv_bfloat16* out,
-                     long long ld_out, cudaStream_t st) {
-  if (R == 0 || C == 0) return MRL_OK;
-  dim3 grid((unsigned)((C + 63) / 64), (unsigned)((R + 63) / 64));
-  if (grid.y > 65535u) return MRL_ERR_UNSUPPORTED_SHAPE;
-  transpose_bf16_kernel<<<grid, 256, 0, st>>>(in, R, C, ld_in, out, ld_out);
   MRL_CUDA_OK(cudaGetLastError());
   return MRL_OK;
 }
@@ -698,9 +695,9 @@ struct LmheadWs {
   void* rows;            // per-row scratch of the loss (MrlLossWs)
   float *g, *lse2, *zt;
   float2* partial;
-  __nv_bfloat16 *WT, *HT, *D, *DT;
+  __nv_bfloat16* D;      // one vocabulary chunk of dZ, [N, ldD]
   float* dH_acc;
-  long long part_ld, ldWT, ldHT, ldD, ldDT;
+  long long part_ld, ldD;
   int n_tiles_fwd, vchunk, n_chunks;
   size_t bytes;
 };
@@ -717,14 +714,8 @@ LmheadWs carve_lmhead_ws(void* ws, long long N, int V, int H, int S) {
   w.partial = c.take<float2>((size_t)w.n_tiles_fwd * (size_t)w.part_ld);
   w.vchunk = V < kVChunk ? (int)pad_to(V, BN) : kVChunk;
   w.n_chunks = (V + w.vchunk - 1) / w.vchunk;
-  w.ldWT = pad_to(V, 8);
-  w.ldHT = pad_to(N, 8);
   w.ldD = w.vchunk;
-  w.ldDT = pad_to(N, 8);
-  w.WT = c.take<__nv_bfloat16>((size_t)H * (size_t)w.ldWT);
-  w.HT = c.take<__nv_bfloat16>((size_t)H * (size_t)w.ldHT);
   w.D = c.take<__nv_bfloat16>((size_t)N * (size_t)w.ldD);
-  w.DT = c.take<__nv_bfloat16>((size_t)w.vchunk * (size_t)w.ldDT);
   w.dH_acc = w.n_chunks > 1 ? c.take<float>((size_t)N * (size_t)H) : nullptr;
   w.bytes = c.off;
   return w;
@@ -737,11 +728,12 @@ size_t mrl_fused_lmhead_workspace_bytes(long long N, int V, int H, int S) {
   return carve_lmhead_ws(nullptr, N, V, H, S).bytes;
 }
 
-// C[M, N] = A[M, K] B[N, K]^T with a plain store (bf16 or fp32, optionally added to): the building block of the
-// two backward products, also reachable on its own for checks of the tensor-core mainloop.
-int mrl_lmhead_gemm_tn(const void* A, long long lda, const void* B, long long ldb, int M, int N, int K, void* C,
-                       long long ldc, int c_mode, float* Cacc, long long ldacc, int32_t* status, bool pair_tiles,
-                       cudaStream_t st) {
+// C[M, N] = A B^T with a plain store (bf16 or fp32, optionally added to): the building block of the two backward
+// products, also reachable on its own for checks of the tensor-core mainloop.  a_mn / b_mn: the operand is given
+// MN-major, i.e. as the row-major [K, M] (resp. [K, N]) matrix.
+int mrl_lmhead_gemm(const void* A, long long lda, bool a_mn, const void* B, long long ldb, bool b_mn, int M, int N, int K,
+                    void* C, long long ldc, int c_mode, float* Cacc, long long ldacc, int32_t* status, bool pair_tiles,
+                    cudaStream_t st) {
   GemmParams p = {};
   p.M = M;
   p.N = N;
@@ -752,7 +744,10 @@ int mrl_lmhead_gemm_tn(const void* A, long long lda, const void* B, long long ld
   p.Cacc = Cacc;
   p.ldacc = ldacc;
   p.status = status;
-  return launch_gemm<EPI_STORE>(A, lda, B, ldb, p, pair_tiles, st);
+  if (a_mn && b_mn) return launch_gemm<EPI_STORE, true, true>(A, lda, B, ldb, p, pair_tiles, st);
+  if (b_mn) return launch_gemm<EPI_STORE, false, true>(A, lda, B, ldb, p, pair_tiles, st);
+  if (a_mn) return MRL_ERR_INVALID_ARG;  // not needed by the pass: not instantiated
+  return launch_gemm<EPI_STORE, false, false>(A, lda, B, ldb, p, pair_tiles, st);
 }
 
 extern "C" int mrl_fused_lmhead_loss_fwd_bwd(const void* hidden, const void* W, int64_t N, int32_t H, int32_t V,
@@ -814,7 +809,7 @@ extern "C" int mrl_fused_lmhead_loss_fwd_bwd(const void* hidden, const void* W, 
     p.ids = ids;
     p.zt = w.zt;
     p.col0 = 0;
-    rc = launch_gemm<EPI_LSE>(hid, H, Wm, H, p, pair, st);
+    rc = launch_gemm<EPI_LSE, false, false>(hid, H, Wm, H, p, pair, st);
     if (rc != MRL_OK) return rc;
   }
   const bool seq_ratio = lp->ratio_level == MRL_RATIO_SEQUENCE;
@@ -832,15 +827,12 @@ extern "C" int mrl_fused_lmhead_loss_fwd_bwd(const void* hidden, const void* W, 
   if (rc != MRL_OK) return rc;
   if (dHidden == nullptr) return MRL_OK;
 
-  // ---- backward
-  rc = launch_transpose(Wm, V, H, H, w.WT, w.ldWT, st);
-  if (rc != MRL_OK) return rc;
-  rc = launch_transpose(hid, N, H, H, w.HT, w.ldHT, st);
-  if (rc != MRL_OK) return rc;
+  // ---- backward, per vocabulary chunk.  No operand is transposed in memory: W and hidden enter the two products
+  // MN-major, D enters dHidden's K-major and dW's MN-major.
   for (int ch = 0; ch < w.n_chunks; ++ch) {
     const int v0 = ch * w.vchunk;
     const int vc = V - v0 < w.vchunk ? V - v0 : w.vchunk;
-    {  // D = g (softmax - onehot) of the chunk's columns, both orientations
+    {  // D = g (softmax - onehot) of the chunk's columns
       GemmParams p = {};
       p.M = (int)N;
       p.N = vc;
@@ -852,23 +844,22 @@ extern "C" int mrl_fused_lmhead_loss_fwd_bwd(const void* hidden, const void* W, 
       p.lse2 = w.lse2;
       p.D = w.D;
       p.ldD = w.ldD;
-      p.DT = w.DT;
-      p.ldDT = w.ldDT;
-      rc = launch_gemm<EPI_DZ>(hid, H, Wm + (size_t)v0 * H, H, p, pair, st);
+      rc = launch_gemm<EPI_DZ, false, false>(hid, H, Wm + (size_t)v0 * H, H, p, pair, st);
       if (rc != MRL_OK) return rc;
     }
-    {  // dHidden (+)= D[N, vc] * (W^T[H, v0 : v0 + vc])^T
+    {  // dHidden[N, H] (+)= D[N, vc] * W[v0 : v0 + vc, :]   (A = D K-major; B = the chunk of W, [K = vc, N = H])
       int mode = C_BF16;
       if (w.n_chunks > 1) mode = ch == 0 ? C_F32 : (ch == w.n_chunks - 1 ? C_BF16_FROM_ACC : C_F32_ADD);
       void* C = (mode == C_BF16 || mode == C_BF16_FROM_ACC) ? dHidden : static_cast<void*>(w.dH_acc);
-      rc = mrl_lmhead_gemm_tn(w.D, w.ldD, w.WT + v0, w.ldWT, (int)N, H, vc, C, H, mode, w.dH_acc, H, status, pair, st);
+      rc = mrl_lmhead_gemm(w.D, w.ldD, false, Wm + (size_t)v0 * H, H, true, (int)N, H, vc, C, H, mode, w.dH_acc, H,
+                           status, pair, st);
       if (rc != MRL_OK) return rc;
     }
-    {  // dW[v0 : v0 + vc, :] = D^T[vc, N] * (hidden^T[H, N])^T
+    {  // dW[v0 : v0 + vc, :] = D^T hidden   (A = D as [K = N, M = vc]; B = hidden as [K = N, N = H])
       void* C = accum_dw ? static_cast<void*>(static_cast<float*>(dW) + (size_t)v0 * H)
                          : static_cast<void*>(static_cast<__nv_bfloat16*>(dW) + (size_t)v0 * H);
-      rc = mrl_lmhead_gemm_tn(w.DT, w.ldDT, w.HT, w.ldHT, vc, H, (int)N, C, H, accum_dw ? C_F32_ADD : C_BF16, nullptr,
-                              0, status, pair, st);
+      rc = mrl_lmhead_gemm(w.D, w.ldD, true, hid, H, true, vc, H, (int)N, C, H, accum_dw ? C_F32_ADD : C_BF16, nullptr, 0,
+                           status, pair, st);
       if (rc != MRL_OK) return rc;
     }
   }
