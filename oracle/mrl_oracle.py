@@ -23,6 +23,8 @@ Passages followed (by section / equation of the paper):
   * response-level ratio  w = exp(L_theta - L_behavior)                     (App. H, data-level coupling)
   * policy entropy diagnostic  H_t = - sum_v p_v log p_v                   (Sec. 6, App. B: entropy curves)
   * THL word-level trace alignment  Z_w, C_w, Z_w / C_w                    (Sec. 4.2; App. D, Alg. 3; Thm. 1)
+  * KL-style regulariser  beta R(theta): a per-token KL to a reference, its own loss term,
+    coefficient 1e-3                                                      (Eq. (1); App. A, hyperparameters)
 
 Readings taken where the paper is silent are listed in the repository's
 design notes; each is a parameter here with the default stated.
@@ -31,7 +33,9 @@ Pins (tests, CPU only): closed forms (uniform logits, V = 1, binary-reward
 advantages), brute force on tiny inputs, finite differences, the printed
 three-action example of Prop. 1, the rescue-gate probability of Def. 7, and
 library special cases (scipy logsumexp, torch cross_entropy), and for the word alignment the per-word mass
-conservation and the residual identity of Thm. 1 evaluated from its own set definitions.
+conservation and the residual identity of Thm. 1 evaluated from its own set definitions; for the KL penalty
+the exact expectation identities E_pi[k1] = E_pi[k3] = KL(pi || ref) against scipy's rel_entr, second-order
+agreement of k2, non-negativity, closed forms for a constant log-ratio, and finite differences.
 Functions without a pin: none.
 """
 from __future__ import annotations
@@ -62,6 +66,12 @@ RATIO_SEQUENCE = 1
 # token aggregation (Eq. (1) E_tok then 1/K; or one masked mean over all tokens)
 AGG_TOKEN_MEAN = 0
 AGG_SEQ_MEAN_TOKEN_MEAN = 1
+
+# per-token estimate of KL(pi_theta || pi_ref) from the sampled token's log-ratio d = logp - logp_ref.  The paper
+# says only "per-token KL between policy and reference" (App. A); the three usual sampled-token estimators are offered.
+KL_K1 = 0   # d
+KL_K2 = 1   # d^2 / 2
+KL_K3 = 2   # exp(-d) - 1 + d   (>= 0; like k1, its expectation under pi_theta is the KL exactly)
 
 _ROW_BLOCK = 128
 
@@ -226,6 +236,8 @@ class LossParams:
     seq_denominator: float = 0.0  # <= 0: number of sequences in this call
     nll_coeff: float = 0.0        # lambda_SGT / n_gated (Eq. (2); App. B)
     ratio_level: int = RATIO_TOKEN
+    kl_coeff: float = 0.0         # beta of Eq. (1); App. A: 1e-3.  Used only when a reference trace is given
+    kl_estimator: int = KL_K3
 
 
 def row_coefficients(valid, cu_seqlens, adv_seq, tok_weight, nll_weight, lp: LossParams):
@@ -294,14 +306,42 @@ def surrogate(logp, logp_old, A, cu, cn, lp: LossParams):
     return dict(pg_term=pg_term, nll_term=nll_term, g=g, rho=rho, clipped=clipped, margin=margin)
 
 
+def kl_penalty(logp, logp_ref, c, lp: LossParams):
+    """beta R(theta) of Eq. (1) as App. A describes it: a separate loss term, the per-token KL between the policy and
+    a reference, scaled by beta.  With only the sampled token's reference log-prob at hand, the per-token KL is one of
+    the sampled estimators k(d), d = logp_t - logp_ref_t (KL_K1 / KL_K2 / KL_K3 above), aggregated with the same
+    token coefficients c_t as the surrogate (without the stop-gradient weight u_t):
+
+        L_KL = beta * sum_t c_t k(d_t),      dL_KL/dlogp_t = beta c_t k'(d_t),
+        k1' = 1,  k2' = d,  k3' = 1 - exp(-d).
+
+    Returns dict: kl_term f64[N] (beta c_t k_t), g_kl f64[N] (the part of g_t: -dL_KL/dlogp_t), d.
+    """
+    logp = torch.as_tensor(logp).to(F64)
+    d = logp - torch.as_tensor(logp_ref).to(F64)
+    if lp.kl_estimator == KL_K1:
+        k, dk = d, torch.ones_like(d)
+    elif lp.kl_estimator == KL_K2:
+        k, dk = 0.5 * d * d, d
+    elif lp.kl_estimator == KL_K3:
+        k, dk = torch.expm1(-d) + d, -torch.expm1(-d)
+    else:
+        raise ValueError("unknown KL estimator")
+    w = lp.kl_coeff * c
+    on = w != 0
+    zero = torch.zeros_like(d)
+    return dict(kl_term=torch.where(on, w * k, zero), g_kl=torch.where(on, -w * dk, zero), d=d)
+
+
 def policy_loss(logits, ids, mask, cu_seqlens, adv_seq, logp_old, tok_weight=None, nll_weight=None,
-                lp: LossParams | None = None, want_dlogits: bool = True, rows=None):
+                lp: LossParams | None = None, want_dlogits: bool = True, rows=None, logp_ref=None):
     """The whole logits-in pass: log-probs, ratio, clipped surrogate, aggregation, dlogits.
 
     dlogits[t, v] = g_t * (softmax(z_t)[v] - 1[v == ids_t])  (score e_i - pi, App. H).
     `rows` (optional LongTensor) restricts the dlogits that are materialised to those rows;
     every scalar output still covers all N rows.
-    Returns dict: loss_pg, loss_nll (python floats), logp, lse, valid, g, rho, clipped, margin,
+    With `logp_ref` (f32/f64 [N]) the KL penalty of kl_penalty() is added: loss_kl, and its part of g.
+    Returns dict: loss_pg, loss_nll, loss_kl (python floats), logp, lse, valid, g, rho, clipped, margin,
     A, cu, cn, stats (active, clipped), dlogits f64[len(rows) or N, V] (if requested).
     """
     lp = lp or LossParams()
@@ -317,6 +357,13 @@ def policy_loss(logits, ids, mask, cu_seqlens, adv_seq, logp_old, tok_weight=Non
     out.update(logp=logp, lse=lse, valid=valid, A=A, cu=cu, cn=cn)
     out["loss_pg"] = float(sur["pg_term"].sum())
     out["loss_nll"] = float(sur["nll_term"].sum())
+    out["loss_kl"] = 0.0
+    if logp_ref is not None:
+        _, c, _ = row_coefficients(valid, cu_seqlens, adv_seq, None, None, lp)     # c_t alone (u_t = 1)
+        kl = kl_penalty(logp, logp_ref, c, lp)
+        out["g"] = sur["g"] = sur["g"] + kl["g_kl"]
+        out["kl_term"] = kl["kl_term"]
+        out["loss_kl"] = float(kl["kl_term"].sum())
     out["stats"] = (int(valid.sum()), int((valid & (A != 0) & sur["clipped"]).sum()))
     if want_dlogits:
         sel = torch.arange(N) if rows is None else torch.as_tensor(rows).long()
@@ -386,7 +433,7 @@ def sequence_ratio_surrogate(logp, logp_old, valid, cu_seqlens, adv_seq, nll_wei
 
 
 def policy_loss_sequence_ratio(logits, ids, mask, cu_seqlens, adv_seq, logp_old, nll_weight=None,
-                               lp: LossParams | None = None, want_dlogits: bool = True):
+                               lp: LossParams | None = None, want_dlogits: bool = True, logp_ref=None):
     """The logits-in pass with the response-level ratio: log-probs, sequence_ratio_surrogate, and
     dlogits[t, v] = g_t (softmax(z_t)[v] - 1[v == ids_t]) with the same g for every token of a response."""
     lp = lp or LossParams(ratio_level=RATIO_SEQUENCE)
@@ -401,6 +448,12 @@ def policy_loss_sequence_ratio(logits, ids, mask, cu_seqlens, adv_seq, logp_old,
     out.update(logp=logp, lse=lse, valid=valid)
     out["loss_pg"] = float(sur["seq_term"].sum())
     out["loss_nll"] = float(sur["nll_term"].sum())
+    out["loss_kl"] = 0.0
+    if logp_ref is not None:       # the penalty stays per token (App. A) whatever the ratio's level
+        _, c, _ = row_coefficients(valid, cu_seqlens, adv_seq, None, None, lp)
+        kl = kl_penalty(logp, logp_ref, c, lp)
+        out["g"] = sur["g"] = sur["g"] + kl["g_kl"]
+        out["loss_kl"] = float(kl["kl_term"].sum())
     cu = torch.as_tensor(cu_seqlens).long()
     lens = cu[1:] - cu[:-1]
     row_clipped = torch.repeat_interleave(sur["seq_clipped"], lens) & valid
@@ -419,12 +472,12 @@ def policy_loss_sequence_ratio(logits, ids, mask, cu_seqlens, adv_seq, logp_old,
 
 
 def fused_lmhead_loss(hidden, W, ids, mask, cu_seqlens, adv_seq, logp_old, tok_weight=None,
-                      nll_weight=None, lp: LossParams | None = None):
+                      nll_weight=None, lp: LossParams | None = None, logp_ref=None):
     """Hidden-in pass: z = hidden W^T (float64), then policy_loss; dHidden = dZ W, dW = dZ^T hidden."""
     h = torch.as_tensor(hidden).to(F64)
     w = torch.as_tensor(W).to(F64)
     z = h @ w.T
-    out = policy_loss(z, ids, mask, cu_seqlens, adv_seq, logp_old, tok_weight, nll_weight, lp)
+    out = policy_loss(z, ids, mask, cu_seqlens, adv_seq, logp_old, tok_weight, nll_weight, lp, logp_ref=logp_ref)
     dz = out["dlogits"]
     out["dHidden"] = dz @ w
     out["dW"] = dz.T @ h
