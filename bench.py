@@ -139,7 +139,8 @@ def barrier(world: int):
 class LogitsInWorkload:
     """Config 2: 8 prompts x G = 8, ragged lengths in [128, 1024] packed, V = 151,936, bf16 logits."""
 
-    def __init__(self, w: synth.Workload, seed: int, device, ratio_level: int = 0, with_entropy: bool = False):
+    def __init__(self, w: synth.Workload, seed: int, device, ratio_level: int = 0, with_entropy: bool = False,
+                 with_kl: bool = False):
         from paper_2605_07244_b200 import binding as B
         self.B = B
         self.w = w
@@ -181,6 +182,11 @@ class LogitsInWorkload:
             self.lp.entropy = self.entropy.data_ptr()
         scale = 1.0 if ratio_level == 0 else (self.S / max(self.N, 1)) ** 0.5
         self.logp_old = self.logp + b.noise.to(dev) * scale
+        if with_kl:          # Eq. (1)'s beta R(theta): k3 estimate against a reference trace, beta = 1e-3 (App. A)
+            self.logp_ref = self.logp + b.noise.to(dev).flip(0) * 2.0
+            self.kl_loss = torch.zeros(1, device=dev)
+            self.lp.logp_ref, self.lp.kl_loss = self.logp_ref.data_ptr(), self.kl_loss.data_ptr()
+            self.lp.kl_coeff, self.lp.kl_estimator = 1e-3, B.KL_K3
         torch.cuda.synchronize()
         # adv_prompt, seq_count, row_coef, row_stream, row_terms, finalize; the response-level ratio has a forward
         # launch, the per-response kernel and a backward launch instead of one fused row kernel
@@ -207,7 +213,7 @@ class LogitsInWorkload:
                             "GRPO group z-norm, eps 0.2",
                 "rows": self.N, "sequences": self.S, "V": self.V, "logits_dtype": "bf16",
                 "ratio_level": "token" if self.ratio_level == 0 else "response (App. H)",
-                "entropy_output": bool(self.lp.entropy),
+                "entropy_output": bool(self.lp.entropy), "kl_term": bool(self.lp.logp_ref),
                 "l2": "inputs (%.1f GB logits) exceed the 126 MB L2; no flush needed" % (self.z.numel() * 2 / 1e9)}
 
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region
@@ -569,7 +575,7 @@ def run_ours(args, rank, world, local_rank):
     cls = LmheadWorkload if lmhead_main else LogitsInWorkload
     wl = (cls(synth.CONFIGS[args.workload], args.seed + rank, device) if lmhead_main else
           cls(synth.CONFIGS[args.workload], args.seed + rank, device, 1 if args.ratio_level == "sequence" else 0,
-              args.with_entropy))
+              args.with_entropy, args.with_kl))
     res = measure(wl, args.steps, args.warmup, world, local_rank, rank, peaks, not args.no_e2e,
                   not args.no_cpu_baseline, args)
     del wl
@@ -616,6 +622,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="profiling runs only: skip the host-buffer leg")
     ap.add_argument("--ratio-level", default="token", choices=["token", "sequence"],
                     help="logits-in workloads: importance ratio per token (Eq. (1), default) or per response (App. H)")
+    ap.add_argument("--with-kl", action="store_true",
+                    help="logits-in workloads: add the KL penalty to a reference trace (k3 estimate, beta = 1e-3)")
     ap.add_argument("--with-entropy", action="store_true", help="logits-in workloads: also emit the per-row policy entropy")
     ap.add_argument("--no-lmhead", action="store_true", help="skip the short config-5 leg of the default run")
     args = ap.parse_args()

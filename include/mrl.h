@@ -38,7 +38,7 @@
 extern "C" {
 #endif
 
-#define MRL_VERSION 101
+#define MRL_VERSION 102
 
 /* return codes */
 #define MRL_OK 0
@@ -81,6 +81,13 @@ extern "C" {
 #define MRL_RATIO_SEQUENCE 1   /* w = exp(sum_t logp_t - sum_t logp_old_t) over a response, clipped per
                                   response; loss = - mean over responses of min(w A, clip(w) A)  (App. H) */
 
+/* mrl_loss_params.kl_estimator: per-token estimate of KL(pi_theta || pi_ref) from the sampled token alone,
+ * d = logp_t - logp_ref_t.  The paper states a per-token KL to a reference, as its own loss term (Eq. (1): beta R(theta);
+ * App. A: coefficient 1e-3) and not which estimator; these are the three usual ones. */
+#define MRL_KL_K1 0   /* d */
+#define MRL_KL_K2 1   /* d^2 / 2 */
+#define MRL_KL_K3 2   /* exp(-d) - 1 + d: non-negative, and like k1 its expectation under pi_theta is the KL exactly */
+
 /* mrl_loss_params.flags */
 #define MRL_FLAG_ACCUMULATE_LOSS 1u   /* loss[0..1] and stats += this call (micro-batch accumulation, App. A) */
 #define MRL_FLAG_SKIP_ZERO_ROWS 2u    /* rows whose gradient multiplier is known to be zero before reading the
@@ -121,6 +128,14 @@ typedef struct mrl_loss_params {
                                fused LM head): entropy - sum_v p_v log p_v of softmax(z_t) at every valid row, 0
                                elsewhere -- the policy-entropy diagnostic of Sec. 6 / App. B, taken from the same
                                pass over the logits (one more FMA per logit) */
+  const float* logp_ref;    /* [device] float32 [N], nullable: no KL term.  Reference policy's log-prob of ids[t] */
+  float kl_coeff;           /* beta of Eq. (1); App. A uses 1e-3 */
+  int32_t kl_estimator;     /* MRL_KL_* */
+  float* kl_loss;           /* [device] float32 [1]; required with logp_ref.  Receives beta * sum_t c_t k(d_t), c_t the
+                               aggregation coefficient of the token (agg_mode; without tok_weight); added to under
+                               MRL_FLAG_ACCUMULATE_LOSS.  The gradient outputs include this term's gradient,
+                               beta c_t k'(d_t) through logp_t.  Rows stay live under MRL_FLAG_SKIP_ZERO_ROWS while
+                               the term is on */
 } mrl_loss_params;
 
 /*
@@ -196,6 +211,11 @@ int mrl_token_logprobs(const void* logits, int32_t dtype, int64_t N, int32_t V, 
  * t is clipped iff (A_t > 0 and rho_t > 1+eps_hi) or (A_t < 0 and rho_t < 1-eps_lo); equality is
  * unclipped.  Rows with c_t u_t A_t = 0 add exactly 0 to loss[0].
  *
+ * With lp->logp_ref (Eq. (1)'s beta R(theta); App. A: a per-token KL to a reference, its own loss term):
+ *   d_t = logp_t - logp_ref_t,  k = the estimator lp->kl_estimator (MRL_KL_*)
+ *   lp->kl_loss[0] = kl_coeff * sum_t c_t k(d_t),   g_t -= kl_coeff * c_t k'(d_t)     (every valid row; both
+ *   ratio levels; the total loss is loss[0] + loss[1] + kl_loss[0])
+ *
  * With ratio_level = MRL_RATIO_SEQUENCE (App. H, data-level coupling) the ratio is taken per response:
  *   w_s = exp(sum over the valid rows of s of (logp_t - logp_old_t)),  S_d = seq_denominator (<= 0: S)
  *   loss[0] = - (1 / S_d) sum_s min(w_s A_s, clip(w_s) A_s)   over responses with a valid row
@@ -263,7 +283,7 @@ int mrl_policy_loss_fwd_bwd(const void* logits, int32_t dtype, int64_t N, int32_
  */
 #define MRL_STATIC_MAX_ROWS 65536
 #define MRL_STATIC_MAX_SEQS 65536
-#define MRL_STATIC_SCRATCH_BYTES (3u << 20)
+#define MRL_STATIC_SCRATCH_BYTES (4u << 20)
 int mrl_policy_loss_fwd_bwd_static(const void* logits, int32_t dtype, int64_t N, int32_t V, int64_t ld,
                                    const int32_t* ids, const uint8_t* mask, const int32_t* cu_seqlens,
                                    int32_t S, const float* adv_seq, const float* logp_old,

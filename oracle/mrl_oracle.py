@@ -453,6 +453,7 @@ def policy_loss_sequence_ratio(logits, ids, mask, cu_seqlens, adv_seq, logp_old,
         _, c, _ = row_coefficients(valid, cu_seqlens, adv_seq, None, None, lp)
         kl = kl_penalty(logp, logp_ref, c, lp)
         out["g"] = sur["g"] = sur["g"] + kl["g_kl"]
+        out["kl_term"] = kl["kl_term"]
         out["loss_kl"] = float(kl["kl_term"].sum())
     cu = torch.as_tensor(cu_seqlens).long()
     lens = cu[1:] - cu[:-1]

@@ -18,6 +18,7 @@ ADV_MEAN_ONLY, ADV_GROUP_ZNORM, ADV_BATCH_ZNORM = 0, 1, 2
 PICK_NONE, PICK_FIRST, PICK_SHORTEST, PICK_ALL, PICK_SEEDED = 0, 1, 2, 3, 4
 AGG_TOKEN_MEAN, AGG_SEQ_MEAN_TOKEN_MEAN = 0, 1
 RATIO_TOKEN, RATIO_SEQUENCE = 0, 1
+KL_K1, KL_K2, KL_K3 = 0, 1, 2
 FLAG_ACCUMULATE_LOSS, FLAG_SKIP_ZERO_ROWS, FLAG_ACCUMULATE_DW, FLAG_PAIR_TILES = 1, 2, 4, 8
 WS_TOKEN_LOGPROBS, WS_POLICY_LOSS, WS_FUSED_LMHEAD, WS_THL_WORD_ALIGN = 0, 1, 2, 3
 DEV_BAD_TOKEN_ID, DEV_TIMEOUT, DEV_BAD_WORD_MAP = 1, 2, 4
@@ -38,7 +39,9 @@ class AdvParams(C.Structure):
 class LossParams(C.Structure):
     _fields_ = [("eps_lo", C.c_float), ("eps_hi", C.c_float), ("agg_mode", C.c_int32),
                 ("flags", C.c_uint32), ("pg_denominator", C.c_double), ("seq_denominator", C.c_double),
-                ("nll_coeff", C.c_float), ("ratio_level", C.c_int32), ("entropy", C.c_void_p)]
+                ("nll_coeff", C.c_float), ("ratio_level", C.c_int32), ("entropy", C.c_void_p),
+                ("logp_ref", C.c_void_p), ("kl_coeff", C.c_float), ("kl_estimator", C.c_int32),
+                ("kl_loss", C.c_void_p)]
 
 
 class MrlError(RuntimeError):

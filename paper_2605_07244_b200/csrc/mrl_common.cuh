@@ -34,8 +34,9 @@ struct MrlCarver {
 // Per-row scratch of the loss passes (carved from the caller's workspace) and the host steps around the row kernels.
 struct MrlLossWs {
   float *rowA, *rowcu, *rowcn;        // A_t, c_t u_t, cn_t
+  float* rowck;                       // beta c_t of the KL term (0 when the term is off)
   float *row_m2, *row_s, *row_zt;     // base-2 running max, sum of 2^(x - max), target logit
-  double *pg_term, *nll_term;
+  double *pg_term, *nll_term, *kl_term;
   uint8_t* rowstat;                   // MRL_ROW_* bits
   int32_t* seq_cnt;
   unsigned long long* totals;
@@ -55,6 +56,13 @@ int mrl_rows_finish(const MrlLossWs& w, long long N, const float* logp_old, cons
 int mrl_rows_finish_sequence(const MrlLossWs& w, long long N, int S, const int32_t* cu_seqlens, const float* adv_seq,
                              const float* logp_old, const float* nll_weight, const mrl_loss_params* lp, float* logp,
                              float* loss, int64_t* stats, float* g_out, float* lse2_out, cudaStream_t st);
+
+// The KL term's arguments are consistent (Eq. (1), beta R(theta)).
+static inline bool mrl_kl_args_ok(const mrl_loss_params* lp) {
+  if (lp->logp_ref == nullptr) return true;
+  if (lp->kl_loss == nullptr) return false;
+  return lp->kl_estimator == MRL_KL_K1 || lp->kl_estimator == MRL_KL_K2 || lp->kl_estimator == MRL_KL_K3;
+}
 
 // Benchmark instrumentation (mrl_profile_dominant_kernel): event pairs recorded around dominant kernels.
 void mrl_profile_before(cudaStream_t st);
@@ -128,7 +136,18 @@ struct RowIn {
   float cn;        // NLL coefficient
   float logp_old;  // behaviour trace (ignored when has_old is false)
   bool has_old;
+  float ck;        // beta c_t of the KL term; 0: term off
+  float logp_ref;  // reference trace (read only when ck != 0)
+  int kl_est;      // MRL_KL_*
 };
+
+// k'(d) of the sampled-token KL estimators, d = logp - logp_ref
+__device__ __forceinline__ float kl_slope(float d, int est) {
+  return est == MRL_KL_K1 ? 1.0f : (est == MRL_KL_K2 ? d : -expm1f(-d));
+}
+__device__ __forceinline__ double kl_value(double d, int est) {
+  return est == MRL_KL_K1 ? d : (est == MRL_KL_K2 ? 0.5 * d * d : expm1(-d) + d);
+}
 
 struct RowOut {
   float logp;
@@ -138,7 +157,7 @@ struct RowOut {
   bool clipped;
 };
 
-// Ratio, clipped surrogate and gradient multiplier of one valid row (Eq. (1), Eq. (2)).
+// Ratio, clipped surrogate, KL slope and gradient multiplier of one valid row (Eq. (1), Eq. (2)).
 __device__ __forceinline__ RowOut mrl_row_loss(float logp, const RowIn& in, float eps_lo, float eps_hi) {
   RowOut o;
   o.logp = logp;
@@ -150,6 +169,7 @@ __device__ __forceinline__ RowOut mrl_row_loss(float logp, const RowIn& in, floa
   o.pg_term = live ? -in.cu * s : 0.f;
   o.nll_term = (in.cn != 0.f) ? -in.cn * logp : 0.f;
   o.g = ((live && !o.clipped) ? in.cu * in.A * rho : 0.f) + in.cn;
+  if (in.ck != 0.f) o.g -= in.ck * kl_slope(logp - in.logp_ref, in.kl_est);  // dL_KL/dlogp = beta c k'(d)
   return o;
 }
 

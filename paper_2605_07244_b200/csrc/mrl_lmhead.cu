@@ -535,6 +535,8 @@ __global__ void __launch_bounds__(256) lmhead_rows_kernel(long long N, int V, in
                                                            const float* __restrict__ rowA,
                                                            const float* __restrict__ rowcu,
                                                            const float* __restrict__ rowcn,
+                                                           const float* __restrict__ rowck,
+                                                           const float* __restrict__ logp_ref, int kl_est,
                                                            const float* __restrict__ logp_old, float eps_lo,
                                                            float eps_hi, float* __restrict__ row_m2,
                                                            float* __restrict__ row_s, float* __restrict__ row_zt,
@@ -561,6 +563,9 @@ __global__ void __launch_bounds__(256) lmhead_rows_kernel(long long N, int V, in
     in.cn = rowcn[t];
     in.has_old = logp_old != nullptr;
     in.logp_old = in.has_old ? logp_old[t] : 0.f;
+    in.ck = logp_ref != nullptr ? rowck[t] : 0.f;
+    in.logp_ref = logp_ref != nullptr ? logp_ref[t] : 0.f;
+    in.kl_est = kl_est;
     const mrl::RowOut ro = mrl::mrl_row_loss(logp, in, eps_lo, eps_hi);
     g = ro.g;
     st = MRL_ROW_VALID | MRL_ROW_READ;
@@ -765,6 +770,7 @@ extern "C" int mrl_fused_lmhead_loss_fwd_bwd(const void* hidden, const void* W, 
   if (lp->ratio_level != MRL_RATIO_TOKEN && lp->ratio_level != MRL_RATIO_SEQUENCE) return MRL_ERR_INVALID_ARG;
   if (lp->ratio_level == MRL_RATIO_SEQUENCE && tok_weight != nullptr) return MRL_ERR_INVALID_ARG;
   if (lp->entropy != nullptr) return MRL_ERR_INVALID_ARG;  // the entropy diagnostic is a logits-in output
+  if (!mrl_kl_args_ok(lp)) return MRL_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool accum_loss = lp->flags & MRL_FLAG_ACCUMULATE_LOSS;
   const bool accum_dw = lp->flags & MRL_FLAG_ACCUMULATE_DW;
@@ -773,6 +779,7 @@ extern "C" int mrl_fused_lmhead_loss_fwd_bwd(const void* hidden, const void* W, 
     if (N != 0) return MRL_ERR_INVALID_ARG;
     if (!accum_loss) {
       MRL_CUDA_OK(cudaMemsetAsync(loss, 0, 2 * sizeof(float), st));
+      if (lp->logp_ref != nullptr) MRL_CUDA_OK(cudaMemsetAsync(lp->kl_loss, 0, sizeof(float), st));
       if (stats != nullptr) MRL_CUDA_OK(cudaMemsetAsync(stats, 0, 4 * sizeof(int64_t), st));
     }
     if (dW != nullptr && !accum_dw) MRL_CUDA_OK(cudaMemsetAsync(dW, 0, (size_t)V * H * 2, st));
@@ -814,7 +821,8 @@ extern "C" int mrl_fused_lmhead_loss_fwd_bwd(const void* hidden, const void* W, 
   }
   const bool seq_ratio = lp->ratio_level == MRL_RATIO_SEQUENCE;
   lmhead_rows_kernel<<<(unsigned)((N + 255) / 256), 256, 0, st>>>(N, V, w.n_tiles_fwd, w.partial, w.part_ld, w.zt, ids,
-                                                                  mask, rw.rowA, rw.rowcu, rw.rowcn,
+                                                                  mask, rw.rowA, rw.rowcu, rw.rowcn, rw.rowck,
+                                                                  seq_ratio ? nullptr : lp->logp_ref, lp->kl_estimator,
                                                                   seq_ratio ? nullptr : logp_old, lp->eps_lo,
                                                                   lp->eps_hi, rw.row_m2, rw.row_s, rw.row_zt,
                                                                   rw.rowstat, w.g, w.lse2);

@@ -29,6 +29,9 @@ struct RowParams {
   const float* rowA;
   const float* rowcu;
   const float* rowcn;
+  const float* rowck;     // KL term: beta c_t; read only when logp_ref is given
+  const float* logp_ref;  // nullable
+  int kl_est;
   const float* logp_old;
   float eps_lo, eps_hi;
   uint32_t flags;
@@ -61,15 +64,23 @@ __device__ __forceinline__ RowCtx load_row_ctx(const RowParams& p, long long row
   c.in.cn = 0.f;
   c.in.logp_old = 0.f;
   c.in.has_old = false;
+  c.in.ck = 0.f;
+  c.in.logp_ref = 0.f;
+  c.in.kl_est = p.kl_est;
   if (p.loss_mode) {
     c.in.A = p.rowA[row];
     c.in.cu = p.rowcu[row];
     c.in.cn = p.rowcn[row];
     c.in.has_old = p.logp_old != nullptr;
     if (c.in.has_old) c.in.logp_old = p.logp_old[row];
+    if (p.logp_ref != nullptr) {
+      c.in.ck = p.rowck[row];
+      c.in.logp_ref = p.logp_ref[row];
+    }
   }
   c.dead = !c.valid;
-  if (p.loss_mode && (p.flags & MRL_FLAG_SKIP_ZERO_ROWS) && (c.in.cu == 0.f || c.in.A == 0.f) && c.in.cn == 0.f)
+  if (p.loss_mode && (p.flags & MRL_FLAG_SKIP_ZERO_ROWS) && (c.in.cu == 0.f || c.in.A == 0.f) && c.in.cn == 0.f &&
+      c.in.ck == 0.f)
     c.dead = true;
   return c;
 }
@@ -554,9 +565,11 @@ __global__ void __launch_bounds__(256) seq_ratio_kernel(const int32_t* __restric
                                                          const int32_t* __restrict__ seq_cnt,
                                                          const float* __restrict__ adv_seq,
                                                          const float* __restrict__ logp_old,
-                                                         const float* __restrict__ nll_weight, mrl_loss_params lp,
+                                                         const float* __restrict__ nll_weight,
+                                                         const float* __restrict__ rowck, mrl_loss_params lp,
                                                          double* __restrict__ pg_term, double* __restrict__ nll_term,
-                                                         float* __restrict__ logp, float* g_out, float* lse2_out) {
+                                                         double* __restrict__ kl_term, float* __restrict__ logp,
+                                                         float* g_out, float* lse2_out) {
   __shared__ double red[8];
   __shared__ double diff_sh;
   const int s = blockIdx.x, tid = threadIdx.x;
@@ -594,17 +607,23 @@ __global__ void __launch_bounds__(256) seq_ratio_kernel(const int32_t* __restric
     const bool valid = (st & kStatValid) && (st & kStatRead);
     double lpv = 0.0;
     float l2 = 0.f, g = 0.f;
-    double nl = 0.0;
+    double nl = 0.0, kl = 0.0;
     if (valid) {
       l2 = row_m2[t] + log2f(row_s[t]);
       lpv = (double)row_zt[t] - ((double)row_m2[t] + log2((double)row_s[t])) * kLn2;
       const float cn = nll_weight ? (float)cn_base * nll_weight[t] : 0.f;
       g = g_pg + cn;
       if (cn != 0.f) nl = -(double)cn * lpv;
+      if (lp.logp_ref != nullptr && rowck[t] != 0.f) {  // the KL term stays per token (App. A)
+        const double d = lpv - (double)lp.logp_ref[t];
+        kl = (double)rowck[t] * mrl::kl_value(d, lp.kl_estimator);
+        g -= rowck[t] * mrl::kl_slope((float)d, lp.kl_estimator);
+      }
       if (clipped) rowstat[t] = st | kStatClipped;
     }
     pg_term[t] = t == a ? term : 0.0;
     nll_term[t] = nl;
+    kl_term[t] = kl;
     if (logp != nullptr) logp[t] = (float)lpv;
     lse2_out[t] = l2;
     g_out[t] = g;
@@ -651,7 +670,7 @@ __global__ void __launch_bounds__(128) seq_count_kernel(const int32_t* __restric
   }
 }
 
-// A_t, c_t u_t and cn_t of every row (Eq. (1) aggregation, Eq. (2) per-token average)
+// A_t, c_t u_t, cn_t and beta c_t of every row (Eq. (1) aggregation and regulariser, Eq. (2) per-token average)
 __global__ void __launch_bounds__(128) row_coef_kernel(const int32_t* __restrict__ cu, int S, long long N, int V,
                                                         const int32_t* __restrict__ ids,
                                                         const uint8_t* __restrict__ mask,
@@ -660,7 +679,8 @@ __global__ void __launch_bounds__(128) row_coef_kernel(const int32_t* __restrict
                                                         const float* __restrict__ nll_weight,
                                                         const int32_t* __restrict__ seq_cnt,
                                                         const unsigned long long* __restrict__ totals,
-                                                        mrl_loss_params lp, float* rowA, float* rowcu, float* rowcn) {
+                                                        mrl_loss_params lp, float* rowA, float* rowcu, float* rowcn,
+                                                        float* rowck) {
   const int s = blockIdx.x;
   const long long a = max(0ll, min((long long)cu[s], N)), b = max(a, min((long long)cu[s + 1], N));
   const double len = (double)seq_cnt[s];
@@ -682,6 +702,7 @@ __global__ void __launch_bounds__(128) row_coef_kernel(const int32_t* __restrict
     rowA[t] = A;
     rowcu[t] = valid ? c * (tok_weight ? tok_weight[t] : 1.f) : 0.f;
     rowcn[t] = (valid && nll_weight) ? cn_base * nll_weight[t] : 0.f;
+    rowck[t] = (valid && lp.logp_ref != nullptr) ? lp.kl_coeff * c : 0.f;
   }
 }
 
@@ -696,13 +717,16 @@ __global__ void __launch_bounds__(256) row_terms_kernel(long long N, const float
                                                          const float* __restrict__ rowA,
                                                          const float* __restrict__ rowcu,
                                                          const float* __restrict__ rowcn,
+                                                         const float* __restrict__ rowck,
+                                                         const float* __restrict__ logp_ref, int kl_est,
                                                          const float* __restrict__ logp_old, float eps_lo,
                                                          float eps_hi, double* __restrict__ pg_term,
-                                                         double* __restrict__ nll_term, float* __restrict__ logp) {
+                                                         double* __restrict__ nll_term, double* __restrict__ kl_term,
+                                                         float* __restrict__ logp) {
   const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= N) return;
   const uint8_t st = rowstat[t];
-  double pg = 0.0, nl = 0.0, lp = 0.0;
+  double pg = 0.0, nl = 0.0, kl = 0.0, lp = 0.0;
   if ((st & kStatValid) && (st & kStatRead)) {
     const double lse = ((double)row_m2[t] + log2((double)row_s[t])) * 0.693147180559945309417232121458;
     lp = (double)row_zt[t] - lse;
@@ -713,18 +737,22 @@ __global__ void __launch_bounds__(256) row_terms_kernel(long long N, const float
       pg = -cu * fmin(rho * A, fmin(fmax(rho, lo), hi) * A);
     }
     if (cn != 0.0) nl = -cn * lp;
+    if (logp_ref != nullptr && rowck[t] != 0.f) kl = (double)rowck[t] * mrl::kl_value(lp - (double)logp_ref[t], kl_est);
   }
   pg_term[t] = pg;
   nll_term[t] = nl;
+  kl_term[t] = kl;
   if (logp != nullptr) logp[t] = (float)lp;
 }
 
 // fixed-order float64 sums of the per-row terms and the row statistics
 __global__ void __launch_bounds__(1024) finalize_kernel(const double* __restrict__ pg_term,
                                                          const double* __restrict__ nll_term,
+                                                         const double* __restrict__ kl_term,
                                                          const uint8_t* __restrict__ rowstat, long long N,
                                                          const unsigned long long* __restrict__ totals,
-                                                         uint32_t flags, float* loss, long long* stats) {
+                                                         uint32_t flags, float* loss, float* kl_loss,
+                                                         long long* stats) {
   __shared__ double red[6][32];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   double v[6] = {0, 0, 0, 0, 0, 0};
@@ -735,16 +763,17 @@ __global__ void __launch_bounds__(1024) finalize_kernel(const double* __restrict
     v[2] += (st & kStatValid) ? 1.0 : 0.0;
     v[3] += (st & kStatClipped) ? 1.0 : 0.0;
     v[4] += (st & kStatRead) ? 1.0 : 0.0;
+    v[5] += kl_term[t];
   }
 #pragma unroll
-  for (int k = 0; k < 5; ++k) {
+  for (int k = 0; k < 6; ++k) {
     for (int o = 16; o > 0; o >>= 1) v[k] += __shfl_xor_sync(0xffffffffu, v[k], o);
     if (lane == 0) red[k][warp] = v[k];
   }
   __syncthreads();
   if (warp == 0) {
 #pragma unroll
-    for (int k = 0; k < 5; ++k) {
+    for (int k = 0; k < 6; ++k) {
       double t = red[k][lane];
       for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
       v[k] = t;
@@ -753,6 +782,7 @@ __global__ void __launch_bounds__(1024) finalize_kernel(const double* __restrict
       const bool accum = flags & MRL_FLAG_ACCUMULATE_LOSS;
       loss[0] = (accum ? loss[0] : 0.f) + (float)v[0];
       loss[1] = (accum ? loss[1] : 0.f) + (float)v[1];
+      if (kl_loss != nullptr) kl_loss[0] = (accum ? kl_loss[0] : 0.f) + (float)v[5];
       if (stats != nullptr) {
         stats[0] = (accum ? stats[0] : 0) + (long long)v[2];
         stats[1] = (accum ? stats[1] : 0) + (long long)v[3];
@@ -770,11 +800,13 @@ MrlLossWs carve_loss_ws(void* ws, long long N, int S) {
   w.rowA = c.take<float>((size_t)N);
   w.rowcu = c.take<float>((size_t)N);
   w.rowcn = c.take<float>((size_t)N);
+  w.rowck = c.take<float>((size_t)N);
   w.row_m2 = c.take<float>((size_t)N);
   w.row_s = c.take<float>((size_t)N);
   w.row_zt = c.take<float>((size_t)N);
   w.pg_term = c.take<double>((size_t)N);
   w.nll_term = c.take<double>((size_t)N);
+  w.kl_term = c.take<double>((size_t)N);
   w.rowstat = c.take<uint8_t>((size_t)N);
   w.seq_cnt = c.take<int32_t>((size_t)S + 1);
   w.bytes = c.off;
@@ -857,7 +889,7 @@ int mrl_rows_prepare(void* workspace, long long N, int V, int S, const int32_t* 
   seq_count_kernel<<<S, 128, 0, st>>>(cu_seqlens, S, N, V, ids, mask, w.seq_cnt, w.totals, status);
   MRL_CUDA_OK(cudaGetLastError());
   row_coef_kernel<<<S, 128, 0, st>>>(cu_seqlens, S, N, V, ids, mask, adv_seq, tok_weight, nll_weight, w.seq_cnt,
-                                     w.totals, *lp, w.rowA, w.rowcu, w.rowcn);
+                                     w.totals, *lp, w.rowA, w.rowcu, w.rowcn, w.rowck);
   MRL_CUDA_OK(cudaGetLastError());
   *out = w;
   return MRL_OK;
@@ -867,10 +899,12 @@ int mrl_rows_prepare(void* workspace, long long N, int V, int S, const int32_t* 
 int mrl_rows_finish(const MrlLossWs& w, long long N, const float* logp_old, const mrl_loss_params* lp, float* logp,
                     float* loss, int64_t* stats, cudaStream_t st) {
   row_terms_kernel<<<(unsigned)((N + 255) / 256), 256, 0, st>>>(N, w.row_m2, w.row_s, w.row_zt, w.rowstat, w.rowA,
-                                                                w.rowcu, w.rowcn, logp_old, lp->eps_lo, lp->eps_hi,
-                                                                w.pg_term, w.nll_term, logp);
+                                                                w.rowcu, w.rowcn, w.rowck, lp->logp_ref,
+                                                                lp->kl_estimator, logp_old, lp->eps_lo, lp->eps_hi,
+                                                                w.pg_term, w.nll_term, w.kl_term, logp);
   MRL_CUDA_OK(cudaGetLastError());
-  finalize_kernel<<<1, 1024, 0, st>>>(w.pg_term, w.nll_term, w.rowstat, N, w.totals, lp->flags, loss,
+  finalize_kernel<<<1, 1024, 0, st>>>(w.pg_term, w.nll_term, w.kl_term, w.rowstat, N, w.totals, lp->flags, loss,
+                                      lp->logp_ref != nullptr ? lp->kl_loss : nullptr,
                                       reinterpret_cast<long long*>(stats));
   MRL_CUDA_OK(cudaGetLastError());
   return MRL_OK;
@@ -883,11 +917,14 @@ int mrl_rows_finish_sequence(const MrlLossWs& w, long long N, int S, const int32
                              float* loss, int64_t* stats, float* g_out, float* lse2_out, cudaStream_t st) {
   MRL_CUDA_OK(cudaMemsetAsync(w.pg_term, 0, (size_t)N * sizeof(double), st));
   MRL_CUDA_OK(cudaMemsetAsync(w.nll_term, 0, (size_t)N * sizeof(double), st));
+  MRL_CUDA_OK(cudaMemsetAsync(w.kl_term, 0, (size_t)N * sizeof(double), st));
   if (logp != nullptr) MRL_CUDA_OK(cudaMemsetAsync(logp, 0, (size_t)N * sizeof(float), st));
   seq_ratio_kernel<<<S, 256, 0, st>>>(cu_seqlens, S, N, w.row_m2, w.row_s, w.row_zt, w.rowstat, w.seq_cnt, adv_seq,
-                                      logp_old, nll_weight, *lp, w.pg_term, w.nll_term, logp, g_out, lse2_out);
+                                      logp_old, nll_weight, w.rowck, *lp, w.pg_term, w.nll_term, w.kl_term, logp, g_out,
+                                      lse2_out);
   MRL_CUDA_OK(cudaGetLastError());
-  finalize_kernel<<<1, 1024, 0, st>>>(w.pg_term, w.nll_term, w.rowstat, N, w.totals, lp->flags, loss,
+  finalize_kernel<<<1, 1024, 0, st>>>(w.pg_term, w.nll_term, w.kl_term, w.rowstat, N, w.totals, lp->flags, loss,
+                                      lp->logp_ref != nullptr ? lp->kl_loss : nullptr,
                                       reinterpret_cast<long long*>(stats));
   MRL_CUDA_OK(cudaGetLastError());
   return MRL_OK;
@@ -950,12 +987,14 @@ extern "C" int mrl_policy_loss_fwd_bwd(const void* logits, int32_t dtype, int64_
   if (!(lp->eps_lo >= 0.f) || !(lp->eps_hi >= 0.f)) return MRL_ERR_INVALID_ARG;
   if (lp->ratio_level != MRL_RATIO_TOKEN && lp->ratio_level != MRL_RATIO_SEQUENCE) return MRL_ERR_INVALID_ARG;
   if (lp->ratio_level == MRL_RATIO_SEQUENCE && tok_weight != nullptr) return MRL_ERR_INVALID_ARG;
+  if (!mrl_kl_args_ok(lp)) return MRL_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool accum = lp->flags & MRL_FLAG_ACCUMULATE_LOSS;
   if (N == 0 || S == 0) {
     if (N != 0) return MRL_ERR_INVALID_ARG;  // rows without a sequence
     if (!accum) {
       MRL_CUDA_OK(cudaMemsetAsync(loss, 0, 2 * sizeof(float), st));
+      if (lp->logp_ref != nullptr) MRL_CUDA_OK(cudaMemsetAsync(lp->kl_loss, 0, sizeof(float), st));
       if (stats != nullptr) MRL_CUDA_OK(cudaMemsetAsync(stats, 0, 4 * sizeof(int64_t), st));
     }
     return MRL_OK;
@@ -981,6 +1020,9 @@ extern "C" int mrl_policy_loss_fwd_bwd(const void* logits, int32_t dtype, int64_
   p.rowA = w.rowA;
   p.rowcu = w.rowcu;
   p.rowcn = w.rowcn;
+  p.rowck = w.rowck;
+  p.logp_ref = lp->logp_ref;
+  p.kl_est = lp->kl_estimator;
   p.logp_old = logp_old;
   p.eps_lo = lp->eps_lo;
   p.eps_hi = lp->eps_hi;

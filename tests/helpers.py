@@ -32,7 +32,22 @@ def oracle_lp(lp: B.LossParams) -> O.LossParams:
     # float32 parameters are upcast exactly, as the kernel sees them
     return O.LossParams(eps_lo=float(lp.eps_lo), eps_hi=float(lp.eps_hi), agg_mode=lp.agg_mode,
                         pg_denominator=lp.pg_denominator, seq_denominator=lp.seq_denominator,
-                        nll_coeff=float(lp.nll_coeff), ratio_level=lp.ratio_level)
+                        nll_coeff=float(lp.nll_coeff), ratio_level=lp.ratio_level,
+                        kl_coeff=float(lp.kl_coeff), kl_estimator=lp.kl_estimator)
+
+
+class KlTerm:
+    """Switches the KL penalty on in `lp`: uploads the reference trace, provides the device scalar the term is
+    written to, and keeps both alive for as long as `lp` is used."""
+
+    def __init__(self, lp, logp_ref, beta, estimator, init=float("nan")):
+        self.ref = dev(logp_ref, torch.float32)
+        self.out = torch.full((1,), init, dtype=torch.float32, device="cuda")
+        lp.logp_ref, lp.kl_loss = self.ref.data_ptr(), self.out.data_ptr()
+        lp.kl_coeff, lp.kl_estimator = beta, estimator
+
+    def value(self):
+        return float(self.out.cpu())
 
 
 def run_gpu_policy_loss(logits, ids, mask, cu, adv, logp_old, tok_weight, nll_weight, lp, V=None,

@@ -33,7 +33,7 @@ def test_header_declarations_are_all_exported(lib):
 
 
 def test_version_and_status_strings(lib):
-    assert B.version() == 101
+    assert B.version() == 102
     assert B.status_string(0) == "MRL_OK"
     assert B.status_string(4) == "MRL_ERR_WORKSPACE_TOO_SMALL"
     assert B.status_string(12345) == "MRL_ERR_UNKNOWN"
@@ -78,6 +78,9 @@ def test_policy_loss_rejects_bad_arguments(lib):
     assert call(ws=C.c_void_p(0x1010)) == 1    # workspace not 256-byte aligned
     assert call(lp_=B.LossParams(0.2, 0.2, 9, 0, 0.0, 0.0, 0.0, 0)) == 1
     assert call(lp_=B.LossParams(-0.1, 0.2, 0, 0, 0.0, 0.0, 0.0, 0)) == 1
+    # KL term: a reference trace needs somewhere to put the term and a known estimator
+    assert call(lp_=B.LossParams(0.2, 0.2, 0, 0, 0.0, 0.0, 0.0, 0, None, 0x1000, 1e-3, B.KL_K3, None)) == 1
+    assert call(lp_=B.LossParams(0.2, 0.2, 0, 0, 0.0, 0.0, 0.0, 0, None, 0x1000, 1e-3, 5, 0x1000)) == 1
 
 
 def test_group_advantages_rejects_bad_arguments(lib):
