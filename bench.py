@@ -204,6 +204,31 @@ class LogitsInWorkload:
                                   None, None, self.lp, self.dz if dz is None else dz, self.logp, self.loss,
                                   self.stats, self.status, self.ws)
 
+    def measure_skip_zero_rows(self, steps=10):
+        """The same step with MRL_FLAG_SKIP_ZERO_ROWS: rows of zero-advantage groups are not read (their gradient
+        rows are still written, as zeros).  Reported beside the headline, which streams every row."""
+        B = self.B
+        self.lp.flags |= B.FLAG_SKIP_ZERO_ROWS
+        try:
+            for _ in range(3):
+                self.step()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(steps):
+                self.step()
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / steps
+            st = self.stats.cpu()
+        finally:
+            self.lp.flags &= ~B.FLAG_SKIP_ZERO_ROWS
+        streamed = int(st[2])
+        V2 = self.V * self.z.element_size()
+        return {"value": self.N / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms, "steps": steps, "rows": self.N,
+                "streamed_rows": streamed, "algorithmic_bytes_per_step": streamed * 2 * V2 + (self.N - streamed) * V2,
+                "note": "tokens/s over all valid tokens; rows with A = 0 are not read, their dlogits rows are zero-filled"}
+
     def tokens(self):
         return self.N
 
@@ -323,8 +348,8 @@ class LmheadWorkload:
         torch.cuda.synchronize()
         chunks = -(-self.V // 16384)
         self.dominant_per_step = 1 + 3 * chunks          # forward GEMM, then (dZ, dHidden, dW) per vocabulary chunk
-        # adv, seq_count, row_coef, forward GEMM, rows, row_terms, finalize, two transposes, 3 GEMMs per chunk
-        self.kernels_per_step = 9 + 3 * chunks
+        # adv, seq_count, row_coef, forward GEMM, rows, row_terms, finalize, then 3 GEMMs per chunk
+        self.kernels_per_step = 7 + 3 * chunks
         self.flops_executed = 8.0 * self.N * self.H * self.V      # forward, recompute, dHidden, dW
         self.flops_algorithmic = 6.0 * self.N * self.H * self.V   # without the recompute
 
@@ -550,6 +575,8 @@ def measure(wl, steps, warmup, world, local_rank, rank, peaks, with_e2e, with_cp
            "gpu_launches": wl.kernels_per_step * steps, "roofline": wl.roofline(kernel_ms, peaks)}
     # end to end: pinned host buffers -> device -> kernels -> pinned host buffers
     out["e2e"] = run_e2e(args, wl, world) if with_e2e else None
+    if world == 1 and hasattr(wl, "measure_skip_zero_rows") and wl.ratio_level == 0 and not wl.lp.logp_ref:
+        out["skip_zero_rows"] = wl.measure_skip_zero_rows()
     out["cpu_baseline"] = None
     if with_cpu and rank == 0 and world == 1:
         n, dt, sample = wl.time_oracle()
@@ -603,6 +630,8 @@ def run_ours(args, rank, world, local_rank):
             "config": res["config"], "clocks": res["clocks"], "e2e": res["e2e"], "gpu_launches": res["gpu_launches"],
             "roofline": res["roofline"], "cpu_baseline": res["cpu_baseline"],
         }
+        if res.get("skip_zero_rows") is not None:
+            line["skip_zero_rows"] = res["skip_zero_rows"]
         if lmhead is not None:
             line["lmhead"] = lmhead
         if thl is not None:

@@ -374,7 +374,8 @@ __global__ void __launch_bounds__(kT, 1024 / kT) row_stream_kernel(const RowPara
   }
   const float neg_k = -(lse2 - log2f(fabsf(g)));  // 2^(z log2e - k) = |g| softmax(z)
   const uint32_t sign = g < 0.f ? 0x80008000u : 0u;
-  for (int base = 0; base < nvec; base += kT * kU) {
+  // (from the row's end backwards: what pass 1 loaded last is the most likely to be still in L1 / L2)
+  for (int base = ((nvec - 1) / (kT * kU)) * (kT * kU); base >= 0; base -= kT * kU) {
     const bool full = base + kT * kU <= nvec;
     Vec v[kU];
 #pragma unroll
