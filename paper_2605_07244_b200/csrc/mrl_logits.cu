@@ -114,7 +114,7 @@ __device__ __forceinline__ uint32_t hmax2_u32(uint32_t a, uint32_t b) {
 // ------------------------------------------------------------------------------------------------
 // Streaming kernel: bf16, one CTA per row, nothing resident in shared memory.
 // Pass 1 streams the row from HBM with 128- or 256-bit loads (running maximum and rescaled sum per thread);
-// pass 2 reads the same vectors again -- by then from L2: the rows in flight (two per SM) are a fraction of its
+// pass 2 reads the same vectors again (all but the group that is still in registers) -- by then from L2: the rows in flight (two per SM) are a fraction of its
 // capacity, and the first read asks L2 to keep the lines -- and writes g * (softmax - onehot) with streaming
 // stores.  HBM sees one read and one write of the row.  Many small CTAs with deep unrolling keep far more bytes
 // in flight per SM than a slice held in shared memory does, which is what this memory-bound pass needs.
@@ -236,9 +236,12 @@ __global__ void __launch_bounds__(kT, 1024 / kT) row_stream_kernel(const RowPara
   if (tid == 0 && owner) zt = __bfloat162float(grow[rel]);         // before anything is written in place
 
   // ---- pass 1: running (max, sum) in the base-2 domain
+  // The row is walked from its last group of kT * kU vectors (the ragged one) down to its first, so that the group
+  // read last is a full one: its vectors stay in registers over the reduction and pass 2 starts from them.
   float m_run = -INFINITY, s_run = 0.f, u_run = 0.f;  // u: sum of 2^(x - m) z, for the entropy (kEnt only)
-  for (int base = 0; base < nvec; base += kT * kU) {
-    Vec v[kU];
+  const int last_base = ((nvec - 1) / (kT * kU)) * (kT * kU);
+  Vec v[kU];
+  for (int base = last_base; base >= 0; base -= kT * kU) {
     if (base + kT * kU <= nvec) {
 #pragma unroll
       for (int u = 0; u < kU; ++u) v[u] = stream_ld<kWords, kHintKeep>(in + (size_t)(base + u * kT) * kVecBytes);
@@ -374,14 +377,16 @@ __global__ void __launch_bounds__(kT, 1024 / kT) row_stream_kernel(const RowPara
   }
   const float neg_k = -(lse2 - log2f(fabsf(g)));  // 2^(z log2e - k) = |g| softmax(z)
   const uint32_t sign = g < 0.f ? 0x80008000u : 0u;
-  // (from the row's end backwards: what pass 1 loaded last is the most likely to be still in L1 / L2)
-  for (int base = ((nvec - 1) / (kT * kU)) * (kT * kU); base >= 0; base -= kT * kU) {
+  // (the first group is still in registers; the others in the order pass 1 read them last-to-first, so the most
+  // recently loaded lines, the likeliest to be still in L2, come first)
+  for (int base = 0; base <= last_base; base += kT * kU) {
     const bool full = base + kT * kU <= nvec;
-    Vec v[kU];
+    if (base != 0) {
 #pragma unroll
-    for (int u = 0; u < kU; ++u)
-      v[u] = (full || base + u * kT + tid < nvec) ? stream_ld<kWords, kHintLast>(in + (size_t)(base + u * kT) * kVecBytes)
-                                                  : stream_fill<kWords>(0u);
+      for (int u = 0; u < kU; ++u)
+        v[u] = (full || base + u * kT + tid < nvec) ? stream_ld<kWords, kHintLast>(in + (size_t)(base + u * kT) * kVecBytes)
+                                                    : stream_fill<kWords>(0u);
+    }
 #pragma unroll
     for (int u = 0; u < kU; ++u) {
       Vec r;
