@@ -48,11 +48,15 @@ C3 = Workload("C3-prp-pool", P=16, M=2, G=8, V=128256, dtype=torch.bfloat16, own
 C4 = Workload("C4-xgrpo-sgt", P=64, M=2, G=16, V=151936, dtype=torch.bfloat16, own_len=(512, 512))
 C5 = Workload("C5-fused-lmhead", P=64, M=1, G=16, V=151936, dtype=torch.bfloat16, own_len=(64, 64),
               reward_beta=False, H=4096)
+# App. A's training setup as a shape: groups of 5, responses up to 3,072 tokens, a learner with the 128,256-token
+# vocabulary and one peer whose rollouts arrive re-tokenised (lengths a third to all of 3,072), spiked logits
+C6 = Workload("C6-appA-pool-3072", P=4, M=2, G=5, V=128256, dtype=torch.bfloat16, own_len=(1024, 3072),
+              peer_len_scale=(1.0 / 3.0, 1.0), spike=12.0, density_std=0.5)
 # config 2 with a quarter of the prompts: still far larger than L2, small enough for a profiler capture
 C2_SMALL = replace(C2, name="C2-qwen-vocab-2-prompts", P=2)
 # config 5 with an eighth of the rows and two vocabulary chunks: operands and scratch still exceed L2
 C5_SMALL = replace(C5, name="C5-fused-lmhead-8k-rows-32k-vocab", P=8, V=32768)
-CONFIGS = {"C1": C1, "C2": C2, "C3": C3, "C4": C4, "C5": C5, "C2s": C2_SMALL, "C5s": C5_SMALL}
+CONFIGS = {"C1": C1, "C2": C2, "C3": C3, "C4": C4, "C5": C5, "C6": C6, "C2s": C2_SMALL, "C5s": C5_SMALL}
 
 
 def scaled(w: Workload, **kw) -> Workload:

@@ -36,10 +36,12 @@ def slabs_of_whole_sequences(cu, target_rows):
 
 
 def stream_and_check(batch, V, adv_seq, tok_weight, nll_weight, nll_coeff, rows_per_slab_checked, seed, flags=0,
-                     all_rows_of=None):
+                     all_rows_of=None, slab_rows=SLAB_ROWS, kl=None):
     """Runs the whole batch slab by slab twice (behaviour trace = log-prob + noise; then ratio one), checks sampled
     rows against the oracle, returns the accumulated losses / stats and, for `all_rows_of` (bool [N]), the device
-    log-probs of those rows next to the oracle's."""
+    log-probs of those rows next to the oracle's.  `kl` = (beta, estimator, delta f32[N]) switches the KL penalty on
+    with the reference trace logp - delta (logp from the oracle on the sampled rows, from the library's forward pass
+    elsewhere), so that the accumulated term has the closed form beta / N * sum_t k(delta_t)."""
     N, cu = batch.N, batch.cu_seqlens
     g = torch.Generator().manual_seed(seed)
     lp = make_lp(pg_den=float(N), nll_coeff=nll_coeff, flags=flags | B.FLAG_ACCUMULATE_LOSS)
@@ -50,7 +52,11 @@ def stream_and_check(batch, V, adv_seq, tok_weight, nll_weight, nll_coeff, rows_
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     picked_logp_gpu, picked_logp_ref, picked_idx = [], [], []
     worst_logp, n_checked = 0.0, 0
-    for s0, s1 in slabs_of_whole_sequences(cu, SLAB_ROWS):
+    kl_loss = torch.zeros(1, device="cuda")
+    kl_loss_r1 = torch.zeros(1, device="cuda")
+    if kl is not None:
+        lp.kl_coeff, lp.kl_estimator = kl[0], kl[1]
+    for s0, s1 in slabs_of_whole_sequences(cu, slab_rows):
         a, b = int(cu[s0]), int(cu[s1])
         n = b - a
         z = batch.logits_rows(a, b, device="cuda")
@@ -69,10 +75,18 @@ def stream_and_check(batch, V, adv_seq, tok_weight, nll_weight, nll_coeff, rows_
         logp_s, lse_s, _ = O.token_logprobs(z_s, ids[rows])
         logp_old = fwd.cpu() + batch.noise[a:b]
         logp_old[rows] = (logp_s + batch.noise[a:b][rows].double()).float()
+        logp_ref = ref_d = None
+        if kl is not None:
+            logp_ref = fwd.cpu() - kl[2][a:b]
+            logp_ref[rows] = (logp_s - kl[2][a:b][rows].double()).float()
+            ref_d = dev(logp_ref)
+            lp.logp_ref = ref_d.data_ptr()
         dz = torch.empty_like(z)
         logp = torch.empty(n, device="cuda")
+        lp.kl_loss = kl_loss.data_ptr() if kl is not None else None
         B.mrl_policy_loss_fwd_bwd(z, dev(ids), None, cu_l, adv_l, dev(logp_old), dev(tw), dev(nw), lp, dz, logp, loss,
                                   stats, status, ws)
+        lp.kl_loss = kl_loss_r1.data_ptr() if kl is not None else None
         B.mrl_policy_loss_fwd_bwd(z, dev(ids), None, cu_l, adv_l, None, dev(tw), dev(nw), lp, None, logp, loss_r1,
                                   stats_r1, status, ws)
         torch.cuda.synchronize()
@@ -83,6 +97,9 @@ def stream_and_check(batch, V, adv_seq, tok_weight, nll_weight, nll_coeff, rows_
         u = torch.ones(rows.numel(), dtype=torch.float64) if tw is None else tw[rows].double()
         cn = torch.zeros(rows.numel(), dtype=torch.float64) if nw is None else nll_coeff * nw[rows].double() / len_rows
         sur = O.surrogate(logp_s, logp_old[rows], A_rows, u / N, cn, oracle_lp(lp))
+        if kl is not None:
+            pen = O.kl_penalty(logp_s, logp_ref[rows], torch.full_like(u, 1.0 / N), oracle_lp(lp))
+            sur["g"] = sur["g"] + pen["g_kl"]
         skipped = (flags & B.FLAG_SKIP_ZERO_ROWS) and True
         got_logp = logp.cpu()[rows].double()
         dead = ((A_rows == 0) | (u == 0)) & (cn == 0) if skipped else torch.zeros_like(A_rows, dtype=torch.bool)
@@ -110,7 +127,8 @@ def stream_and_check(batch, V, adv_seq, tok_weight, nll_weight, nll_coeff, rows_
         del z, dz, ws
     assert int(status.cpu()) == 0
     assert worst_logp <= LOGP_ATOL
-    out = dict(loss=loss.cpu(), loss_r1=loss_r1.cpu(), stats=stats.cpu(), n_checked=n_checked)
+    out = dict(loss=loss.cpu(), loss_r1=loss_r1.cpu(), stats=stats.cpu(), n_checked=n_checked,
+               kl_loss=float(kl_loss.cpu()), kl_loss_r1=float(kl_loss_r1.cpu()))
     if all_rows_of is not None:
         out.update(picked_gpu=torch.cat(picked_logp_gpu), picked_ref=torch.cat(picked_logp_ref), picked_idx=torch.cat(picked_idx))
     return out
@@ -162,3 +180,40 @@ def test_config4_full_size_xgrpo_baseline_with_sgt_rows_in_slabs():
     want = -float(A_rows.sum() / batch.N)
     terms = float(A_rows.abs().sum() / batch.N)
     assert abs(float(res["loss_r1"][0]) - want) <= 1e-5 * max(abs(want), 0.1 * terms)
+
+
+def test_app_a_setup_pool_of_two_policies_in_16k_token_micro_batches():
+    """The training setup of App. A as one step: groups of 5 rollouts from each of two policies, responses up to 3,072
+    tokens, group-centred advantages whitened over the batch, clip 0.2, KL penalty with coefficient 1e-3, log-prob
+    micro-batches of at most 16,384 tokens with the loss accumulated across them."""
+    w = synth.C6
+    meta = synth.make_meta(w, seed=6)
+    batch = synth.make_batch(meta, torch.ones(w.P, w.M, w.G, dtype=torch.bool))
+    assert batch.S == 40 and 60_000 < batch.N < 110_000
+    assert int((batch.cu_seqlens[1:] - batch.cu_seqlens[:-1]).max()) <= 3072
+    # advantages from the library (batch whitening), checked against the oracle before they are used
+    P, M, G = w.P, w.M, w.G
+    ap = B.AdvParams(B.ADV_BATCH_ZNORM, 0, 1e-6, 0.8, 0.2, B.PICK_NONE, 0)
+    adv_own = torch.empty(P, M, G, device="cuda")
+    adv_pool = torch.empty(P, M, G, device="cuda")
+    B.mrl_group_advantages(dev(meta.rewards), dev(meta.seq_len), 0, ap, adv_own, adv_pool, None, None, None, None)
+    own_ref, pool_ref = O.group_advantages(meta.rewards, mode=O.ADV_BATCH_ZNORM)
+    assert (adv_pool.cpu().double() - pool_ref).abs().max() <= 2e-6 and (adv_own.cpu().double() - own_ref).abs().max() <= 2e-6
+    adv_seq = adv_pool.cpu()[batch.seq_p.long(), batch.seq_m.long(), batch.seq_g.long()]
+    assert adv_seq.abs().max() > 0
+    g = torch.Generator().manual_seed(66)
+    delta = 0.2 * torch.randn(batch.N, generator=g)
+    beta = 1e-3
+    res = stream_and_check(batch, w.V, adv_seq, batch.tok_weight, None, 0.0, rows_per_slab_checked=8, seed=3,
+                           slab_rows=16384, kl=(beta, B.KL_K3, delta))
+    assert int(res["stats"][0]) == batch.N and res["n_checked"] >= 40
+    lens = (batch.cu_seqlens[1:] - batch.cu_seqlens[:-1]).long()
+    A_rows = torch.repeat_interleave(adv_seq.double(), lens)
+    want = -float((A_rows * batch.tok_weight.double()).sum() / batch.N)
+    terms = float((A_rows.abs() * batch.tok_weight.double()).sum() / batch.N)
+    assert abs(float(res["loss_r1"][0]) - want) <= 1e-5 * max(abs(want), 0.1 * terms)
+    # the accumulated penalty against its closed form (the reference trace is logp - delta by construction; the float32
+    # rounding of that difference moves k3 ~ delta^2 / 2 by a relative 2e-6 / |delta| per token, with random sign)
+    d = delta.double()
+    want_kl = beta * float((torch.expm1(-d) + d).sum()) / batch.N
+    assert abs(res["kl_loss"] - want_kl) <= 1e-5 * want_kl and abs(res["kl_loss_r1"] - want_kl) <= 1e-5 * want_kl
