@@ -304,9 +304,10 @@ class LmheadWorkload:
     """Config 5: N = 65,536 response tokens, H = 4,096, V = 151,936, bf16 hidden and LM-head weight; the logits
     are never stored; outputs logp, loss, dHidden, dW."""
 
-    def __init__(self, w: synth.Workload, seed: int, device):
+    def __init__(self, w: synth.Workload, seed: int, device, pair_tiles: bool = False):
         from paper_2605_07244_b200 import binding as B
         self.B = B
+        self.pair_tiles = pair_tiles
         self.w = w
         self.meta = synth.make_meta(w, seed)
         self.batch = synth.make_batch(self.meta)
@@ -338,7 +339,7 @@ class LmheadWorkload:
         self.ws = torch.empty(B.workspace_bytes(B.WS_FUSED_LMHEAD, self.N, self.V, self.H, B.BF16, self.S),
                               dtype=torch.uint8, device=dev)
         self.ap = B.AdvParams(B.ADV_GROUP_ZNORM, 0, 1e-6, 0.8, 0.2, B.PICK_SHORTEST, 0)
-        self.lp = B.LossParams(0.2, 0.2, B.AGG_TOKEN_MEAN, 0, 0.0, 0.0, 0.0, 0)
+        self.lp = B.LossParams(0.2, 0.2, B.AGG_TOKEN_MEAN, B.FLAG_PAIR_TILES if pair_tiles else 0, 0.0, 0.0, 0.0, 0)
         # behaviour trace: logp_old = logp + N(0, 0.1); logp from a forward-only call (input preparation)
         B.mrl_group_advantages(self.rewards, self.seq_len, 0, self.ap, self.adv_own, self.adv_pool, self.rescue,
                                self.pick, self.nllw_seq, self.n_gated)
@@ -368,7 +369,7 @@ class LmheadWorkload:
         return {"workload": f"{self.w.name}: fused LM-head, hidden-in: N={self.N} response tokens ({self.w.P} prompts x "
                             f"G=16 x T=64), H={self.H} bf16 hidden N(0,1), W[V={self.V},H] bf16 N(0,0.02^2), logits never "
                             "materialised, GRPO clipped surrogate, binary rewards, fwd+bwd -> dHidden, dW",
-                "rows": self.N, "sequences": self.S, "V": self.V, "H": self.H,
+                "rows": self.N, "sequences": self.S, "V": self.V, "H": self.H, "pair_tiles": self.pair_tiles,
                 "l2": "operands (1.8 GB) and scratch exceed the 126 MB L2; no flush needed"}
 
     def roofline(self, kernel_ms, peaks):
@@ -600,7 +601,7 @@ def run_ours(args, rank, world, local_rank):
     peaks = measured_peaks()
     lmhead_main = args.workload in ("C5", "C5s")
     cls = LmheadWorkload if lmhead_main else LogitsInWorkload
-    wl = (cls(synth.CONFIGS[args.workload], args.seed + rank, device) if lmhead_main else
+    wl = (cls(synth.CONFIGS[args.workload], args.seed + rank, device, args.pair_tiles) if lmhead_main else
           cls(synth.CONFIGS[args.workload], args.seed + rank, device, 1 if args.ratio_level == "sequence" else 0,
               args.with_entropy, args.with_kl))
     res = measure(wl, args.steps, args.warmup, world, local_rank, rank, peaks, not args.no_e2e,
@@ -654,6 +655,8 @@ def main():
     ap.add_argument("--with-kl", action="store_true",
                     help="logits-in workloads: add the KL penalty to a reference trace (k3 estimate, beta = 1e-3)")
     ap.add_argument("--with-entropy", action="store_true", help="logits-in workloads: also emit the per-row policy entropy")
+    ap.add_argument("--pair-tiles", action="store_true",
+                    help="fused LM-head workloads: 256-row tiles worked by CTA pairs (MRL_FLAG_PAIR_TILES)")
     ap.add_argument("--no-lmhead", action="store_true", help="skip the short config-5 leg of the default run")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
