@@ -243,25 +243,43 @@ class LogitsInWorkload:
 
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region
     def e2e_setup(self):
+        """Host buffers in, host buffers out through mrl_policy_loss_fwd_bwd_host: the batch goes through the device
+        in micro-batches of whole sequences with the copies of both directions overlapping the kernels."""
+        B = self.B
         self.h_z = torch.empty(self.z.shape, dtype=self.z.dtype, pin_memory=True)
         self.h_z.copy_(self.z)
         self.h_dz = torch.empty(self.z.shape, dtype=self.z.dtype, pin_memory=True)
-        self.h_small_in = [t.cpu().pin_memory() for t in (self.ids, self.cu, self.rewards, self.seq_len, self.logp_old)]
-        self.d_small_in = [self.ids, self.cu, self.rewards, self.seq_len, self.logp_old]
+        self.h_ids, self.h_cu, self.h_rewards, self.h_seq_len, self.h_logp_old = (
+            t.cpu().pin_memory() for t in (self.ids, self.cu, self.rewards, self.seq_len, self.logp_old))
+        self.h_adv = torch.empty(self.S, pin_memory=True)
         self.h_logp = torch.empty(self.N, pin_memory=True)
         self.h_loss = torch.empty(2, pin_memory=True)
-        h2d = self.h_z.numel() * 2 + sum(t.numel() * t.element_size() for t in self.h_small_in)
-        d2h = self.h_dz.numel() * 2 + self.N * 4 + 8
+        self.h_stats = torch.empty(4, dtype=torch.int64, pin_memory=True)
+        self.h_status = torch.empty(1, dtype=torch.int32, pin_memory=True)
+        self.slab_rows = max(getattr(self, "e2e_slab_rows", 1024), int((self.h_cu[1:] - self.h_cu[:-1]).max()))
+        self.host_ws = torch.empty(B.host_pipeline_workspace_bytes(self.N, self.V, B.BF16, self.S, self.slab_rows),
+                                   dtype=torch.uint8, device=self.z.device)
+        self.host_lp = B.LossParams(0.2, 0.2, B.AGG_TOKEN_MEAN, 0, 0.0, 0.0, 0.0, self.ratio_level)
+        self.e2e_note = ("mrl_policy_loss_fwd_bwd_host on pinned host buffers: every input (logits included) crosses "
+                         "to the device and dlogits, logp, loss come back inside the timed region, in micro-batches of "
+                         f"<= {self.slab_rows} rows over three staging buffers so that both copy directions overlap "
+                         "the kernels")
+        small = (self.h_ids, self.h_cu, self.h_rewards, self.h_seq_len, self.h_logp_old)
+        h2d = self.h_z.numel() * 2 + sum(t.numel() * t.element_size() for t in small) + self.S * 4
+        d2h = self.h_dz.numel() * 2 + self.N * 4 + 8 + 32 + 4 + self.S * 4
         return h2d, d2h
 
     def e2e_step(self):
-        for h, d in zip(self.h_small_in, self.d_small_in):
-            d.copy_(h, non_blocking=True)
-        self.z.copy_(self.h_z, non_blocking=True)
-        self.step()
-        self.h_dz.copy_(self.dz, non_blocking=True)
-        self.h_logp.copy_(self.logp, non_blocking=True)
-        self.h_loss.copy_(self.loss, non_blocking=True)
+        B = self.B
+        self.rewards.copy_(self.h_rewards, non_blocking=True)
+        self.seq_len.copy_(self.h_seq_len, non_blocking=True)
+        B.mrl_group_advantages(self.rewards, self.seq_len, 0, self.ap, self.adv_own, self.adv_pool, self.rescue,
+                               self.pick, self.nllw_seq, self.n_gated)
+        self.h_adv.copy_(self.adv_own.reshape(-1), non_blocking=True)
+        torch.cuda.current_stream().synchronize()     # S advantages are on the host; the pass takes host arrays
+        B.mrl_policy_loss_fwd_bwd_host(self.h_z, self.h_ids, None, self.h_cu, self.h_adv, self.h_logp_old, None, None,
+                                       self.host_lp, self.h_dz, self.h_logp, self.h_loss, self.h_stats, self.h_status,
+                                       self.slab_rows, self.host_ws)
 
     def roofline(self, kernel_ms, peaks):
         k_avg_ms = sum(kernel_ms) / (len(kernel_ms) / self.dominant_per_step)
@@ -530,6 +548,7 @@ def run_reference(args, rank, world):
 
 def run_e2e(args, wl, world):
     e2e_steps = max(1, min(args.steps, 3))
+    wl.e2e_slab_rows = args.e2e_slab_rows
     h2d, d2h = wl.e2e_setup()
     wl.e2e_step()
     torch.cuda.synchronize()
@@ -544,8 +563,9 @@ def run_e2e(args, wl, world):
     e2e_ms, e2e_tokens = aggregate_over_ranks(e0.elapsed_time(e1), wl.tokens() * e2e_steps, world)
     return {"value": e2e_tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
             "d2h_bytes_per_step": d2h, "steps": e2e_steps,
-            "note": "C-ABI calls on device buffers bracketed by pinned-host copies of every input (logits "
-                    "included) and of dlogits, logp and loss"}
+            "note": wl.e2e_note if hasattr(wl, "e2e_note") else
+            "C-ABI calls on device buffers bracketed by pinned-host copies of every input and of the gradients, "
+            "logp and loss"}
 
 
 def measure(wl, steps, warmup, world, local_rank, rank, peaks, with_e2e, with_cpu, args):
@@ -655,6 +675,8 @@ def main():
     ap.add_argument("--with-kl", action="store_true",
                     help="logits-in workloads: add the KL penalty to a reference trace (k3 estimate, beta = 1e-3)")
     ap.add_argument("--with-entropy", action="store_true", help="logits-in workloads: also emit the per-row policy entropy")
+    ap.add_argument("--e2e-slab-rows", type=int, default=1024,
+                    help="logits-in end-to-end leg: rows per micro-batch of the host pipeline")
     ap.add_argument("--pair-tiles", action="store_true",
                     help="fused LM-head workloads: 256-row tiles worked by CTA pairs (MRL_FLAG_PAIR_TILES)")
     ap.add_argument("--no-lmhead", action="store_true", help="skip the short config-5 leg of the default run")

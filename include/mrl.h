@@ -38,7 +38,7 @@
 extern "C" {
 #endif
 
-#define MRL_VERSION 102
+#define MRL_VERSION 103
 
 /* return codes */
 #define MRL_OK 0
@@ -256,6 +256,43 @@ int mrl_policy_loss_fwd_bwd(const void* logits, int32_t dtype, int64_t N, int32_
                             const mrl_loss_params* lp, void* dlogits, int64_t ld_out, float* logp,
                             float* loss, int64_t* stats, int32_t* status, void* workspace,
                             size_t workspace_bytes, void* stream);
+
+/*
+ * mrl_policy_loss_fwd_bwd_host -- mrl_policy_loss_fwd_bwd for a batch that lives in HOST memory.
+ *
+ * Defined by: the same passages as mrl_policy_loss_fwd_bwd; App. A (the step is fed in log-prob micro-batches
+ * and the loss is accumulated across them).  The batch is cut into micro-batches of whole sequences of at most
+ * `slab_rows` rows; for each one its logits are copied to a staging buffer, the pass runs in place there, and the
+ * gradient is copied back, the three legs on three streams over three staging buffers so that copies in both
+ * directions overlap the kernels.  Results are those of mrl_policy_loss_fwd_bwd called once on the whole batch
+ * (per-row outputs bit for bit; the loss up to the order of its float sums).
+ *
+ * Every `h_` argument, and lp->entropy, lp->logp_ref, lp->kl_loss, is a HOST pointer (page-locked memory is needed
+ * for the copies to overlap; pageable memory works and serialises).  Shapes and meaning are those of the device
+ * entry point.  h_cu_seqlens -- and h_ids / h_mask when agg_mode is TOKEN_MEAN and lp->pg_denominator <= 0 -- are
+ * read on the host before the call returns; everything else is read and written asynchronously and the outputs
+ * are valid once the caller has synchronised `stream`.  The host buffers must stay untouched until then.
+ *
+ *   slab_rows  capacity of one staging buffer in rows; no sequence may be longer (MRL_ERR_UNSUPPORTED_SHAPE)
+ *   h_dlogits  [host] dtype [N, ld_out]; nullable = forward only.  Must not overlap h_logits unless identical
+ *              with ld_out = ld (in place)
+ *   h_loss     [host] float32 [2]; h_stats [host] int64 [4], nullable; h_status [host] int32 [1], nullable
+ *   workspace  [device] >= mrl_host_pipeline_workspace_bytes(N, ld, dtype, S, slab_rows), 256-byte aligned:
+ *              three staging buffers of slab_rows * ld elements, the per-row arrays, the loss scratch
+ *   lp         [host] MRL_FLAG_ACCUMULATE_LOSS must be clear (the call returns the whole step's loss)
+ *
+ * ld * sizeof(element) must be a multiple of 32 bytes (MRL_ERR_UNSUPPORTED_SHAPE otherwise).  The library keeps
+ * two copy streams and a few events per device, created at the first call and never freed; calls on one device
+ * share them, so they must not overlap in time.  Errors: as mrl_policy_loss_fwd_bwd.
+ */
+int mrl_policy_loss_fwd_bwd_host(const void* h_logits, int32_t dtype, int64_t N, int32_t V, int64_t ld,
+                                 const int32_t* h_ids, const uint8_t* h_mask, const int32_t* h_cu_seqlens,
+                                 int32_t S, const float* h_adv_seq, const float* h_logp_old,
+                                 const float* h_tok_weight, const float* h_nll_weight, const mrl_loss_params* lp,
+                                 void* h_dlogits, int64_t ld_out, float* h_logp, float* h_loss, int64_t* h_stats,
+                                 int32_t* h_status, int64_t slab_rows, void* workspace, size_t workspace_bytes,
+                                 void* stream);
+size_t mrl_host_pipeline_workspace_bytes(int64_t N, int64_t ld, int32_t dtype, int32_t S, int64_t slab_rows);
 
 /*
  * mrl_policy_loss_fwd_bwd_static -- mrl_policy_loss_fwd_bwd for callers that cannot allocate.

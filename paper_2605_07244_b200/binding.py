@@ -25,7 +25,8 @@ DEV_BAD_TOKEN_ID, DEV_TIMEOUT, DEV_BAD_WORD_MAP = 1, 2, 4
 
 EXPORTS = ("mrl_group_advantages", "mrl_token_logprobs", "mrl_policy_loss_fwd_bwd",
            "mrl_fused_lmhead_loss_fwd_bwd", "mrl_workspace_bytes", "mrl_status_string", "mrl_version",
-           "mrl_profile_dominant_kernel", "mrl_policy_loss_fwd_bwd_static", "mrl_thl_word_align_logprobs")
+           "mrl_profile_dominant_kernel", "mrl_policy_loss_fwd_bwd_static", "mrl_thl_word_align_logprobs",
+           "mrl_policy_loss_fwd_bwd_host", "mrl_host_pipeline_workspace_bytes")
 STATIC_MAX_ROWS, STATIC_MAX_SEQS = 65536, 65536
 ERR_STATIC_SCRATCH_TOO_SMALL = 8
 
@@ -72,6 +73,11 @@ def lib() -> C.CDLL:
         L.mrl_policy_loss_fwd_bwd_static.argtypes = [vp, i32, i64, i32, i64, vp, vp, vp, i32, vp, vp, vp, vp,
                                                      C.POINTER(LossParams), vp, i64, vp, vp, vp, vp, vp]
         L.mrl_policy_loss_fwd_bwd_static.restype = C.c_int
+        L.mrl_policy_loss_fwd_bwd_host.argtypes = [vp, i32, i64, i32, i64, vp, vp, vp, i32, vp, vp, vp, vp,
+                                                   C.POINTER(LossParams), vp, i64, vp, vp, vp, vp, i64, vp, sz, vp]
+        L.mrl_policy_loss_fwd_bwd_host.restype = C.c_int
+        L.mrl_host_pipeline_workspace_bytes.argtypes = [i64, i64, i32, i32, i64]
+        L.mrl_host_pipeline_workspace_bytes.restype = sz
         L.mrl_fused_lmhead_loss_fwd_bwd.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, vp, vp, vp,
                                                     C.POINTER(LossParams), vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.mrl_fused_lmhead_loss_fwd_bwd.restype = C.c_int
@@ -173,6 +179,32 @@ def mrl_policy_loss_fwd_bwd_static(logits, ids, mask, cu_seqlens, adv_seq, logp_
                                                 _p(nll_weight), C.byref(lp), _p(dlogits), ld_out, _p(logp),
                                                 _p(loss), _p(stats), _p(status), _stream(stream)),
            "mrl_policy_loss_fwd_bwd_static")
+
+
+def host_pipeline_workspace_bytes(N: int, ld: int, dtype: int, S: int, slab_rows: int) -> int:
+    return int(lib().mrl_host_pipeline_workspace_bytes(N, ld, dtype, S, slab_rows))
+
+
+def mrl_policy_loss_fwd_bwd_host(h_logits, h_ids, h_mask, h_cu_seqlens, h_adv_seq, h_logp_old, h_tok_weight,
+                                 h_nll_weight, lp: LossParams, h_dlogits, h_logp, h_loss, h_stats, h_status,
+                                 slab_rows: int, workspace, V=None, stream=None):
+    """The logits-in pass on HOST tensors (pinned for overlap), pipelined in micro-batches of whole sequences over
+    three staging buffers in `workspace` (device).  Asynchronous: synchronise `stream` before reading the outputs."""
+    for t in (h_logits, h_ids, h_mask, h_cu_seqlens, h_adv_seq, h_logp_old, h_tok_weight, h_nll_weight, h_dlogits,
+              h_logp, h_loss, h_stats, h_status):
+        if t is not None and t.is_cuda:
+            raise MrlError(1, "mrl_policy_loss_fwd_bwd_host takes host tensors")
+    N = h_logits.shape[0]
+    V = h_logits.shape[1] if V is None else V
+    S = h_cu_seqlens.numel() - 1
+    ld = h_logits.stride(0) if N > 1 else max(h_logits.shape[1], V)
+    ld_out = ld if h_dlogits is None else (h_dlogits.stride(0) if N > 1 else max(h_dlogits.shape[1], V))
+    ws_bytes = workspace.numel() * workspace.element_size()
+    _check(lib().mrl_policy_loss_fwd_bwd_host(_p(h_logits), _dtype_code(h_logits), N, V, ld, _p(h_ids), _p(h_mask),
+                                              _p(h_cu_seqlens), S, _p(h_adv_seq), _p(h_logp_old), _p(h_tok_weight),
+                                              _p(h_nll_weight), C.byref(lp), _p(h_dlogits), ld_out, _p(h_logp),
+                                              _p(h_loss), _p(h_stats), _p(h_status), int(slab_rows), _p(workspace),
+                                              ws_bytes, _stream(stream)), "mrl_policy_loss_fwd_bwd_host")
 
 
 def mrl_fused_lmhead_loss_fwd_bwd(hidden, W, ids, mask, cu_seqlens, adv_seq, logp_old, tok_weight, nll_weight,

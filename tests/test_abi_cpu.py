@@ -33,7 +33,7 @@ def test_header_declarations_are_all_exported(lib):
 
 
 def test_version_and_status_strings(lib):
-    assert B.version() == 102
+    assert B.version() == 103
     assert B.status_string(0) == "MRL_OK"
     assert B.status_string(4) == "MRL_ERR_WORKSPACE_TOO_SMALL"
     assert B.status_string(12345) == "MRL_ERR_UNKNOWN"
@@ -98,3 +98,28 @@ def test_group_advantages_rejects_bad_arguments(lib):
     assert call(seq_len=None) == 1             # SHORTEST needs lengths
     assert call(ap_=B.AdvParams(7, 0, 1e-6, 0.8, 0.2, 0, 0)) == 1
     assert call(ap_=B.AdvParams(1, 2, 1e-6, 0.8, 0.2, 0, 0)) == 1
+
+
+def test_host_pipeline_rejects_bad_arguments(lib):
+    f = lib.mrl_policy_loss_fwd_bwd_host
+    lp = B.LossParams(0.2, 0.2, 0, 0, 0.0, 0.0, 0.0, 0)
+    cu = (C.c_int32 * 2)(0, 4)
+
+    def call(N=4, V=16, ld=16, S=1, lp_=lp, ws=FAKE, ws_bytes=1 << 30, slab=8, loss=FAKE, dtype=B.BF16, cu_=cu):
+        return f(FAKE, dtype, N, V, ld, FAKE, None, cu_, S, FAKE, None, None, None,
+                 C.byref(lp_) if lp_ is not None else None, None, ld, None, loss, None, None, slab, ws, ws_bytes, None)
+
+    assert call(lp_=None) == 1
+    assert call(loss=None) == 1
+    assert call(slab=0) == 1
+    assert call(ld=8) == 1
+    assert call(dtype=9) == 3
+    assert call(V=8, ld=8) == 7                 # rows of 16 bytes: not a multiple of 32
+    assert call(ws=None) == 4
+    assert call(ws_bytes=64) == 4
+    assert call(ws=C.c_void_p(0x1010)) == 1
+    assert call(lp_=B.LossParams(0.2, 0.2, 0, B.FLAG_ACCUMULATE_LOSS, 0.0, 0.0, 0.0, 0)) == 1
+    assert call(slab=3) == 7                    # the only sequence has 4 rows
+    assert call(cu_=(C.c_int32 * 2)(0, 5)) == 1  # cu[S] != N
+    assert lib.mrl_host_pipeline_workspace_bytes(1000, 4096, B.BF16, 8, 128) >= 3 * 128 * 4096 * 2
+    assert lib.mrl_host_pipeline_workspace_bytes(1000, 4096, 9, 8, 128) == 0
