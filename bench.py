@@ -54,7 +54,7 @@ def measured_peaks():
 # DRAM bytes per token (dram__bytes_read.sum + dram__bytes_write.sum over the rows of the capture) of the dominant
 # kernel as it stands, from the committed ncu summary profiles/row_stream_kernel_c2_logits_in.md; traffic grows in
 # proportion to the rows.  Set to None whenever that kernel changes, until the counters are taken again.
-ROW_STREAM_DRAM_BYTES_PER_TOKEN_V151936 = 662400
+ROW_STREAM_DRAM_BYTES_PER_TOKEN_V151936 = 655095
 
 
 class ClockSampler:
@@ -291,7 +291,8 @@ class LogitsInWorkload:
             live_rows = int(lens[(self.adv_own.reshape(-1) != 0).cpu()].sum()) - int(self.stats.cpu()[1])
             alg_bytes = (2 * self.tokens() + live_rows) * self.V * self.z.element_size()
         achieved = alg_bytes / (k_avg_ms * 1e-3) / 1e9
-        per_token = ROW_STREAM_DRAM_BYTES_PER_TOKEN_V151936 if self.V == 151936 and self.ratio_level == 0 else None
+        per_token = (ROW_STREAM_DRAM_BYTES_PER_TOKEN_V151936 if self.V == 151936 and self.ratio_level == 0
+                     and not self.lp.logp_ref and not self.lp.entropy else None)   # counters exist for the default pass only
         kernel = "row_stream_kernel" if self.ratio_level == 0 else "row_stream_kernel (forward) + row_backward_stream_kernel"
         return {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peaks["hbm_gbs"],
                 "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
