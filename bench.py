@@ -204,6 +204,29 @@ class LogitsInWorkload:
                                   None, None, self.lp, self.dz if dz is None else dz, self.logp, self.loss,
                                   self.stats, self.status, self.ws)
 
+    def measure_forward_only(self, peaks, steps=20):
+        """mrl_token_logprobs alone on the same logits: one read of every row, nothing written but N floats."""
+        B = self.B
+        f = lambda: B.mrl_token_logprobs(self.z, self.ids, None, self.logp)
+        for _ in range(3):
+            f()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(steps):
+            f()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / steps
+        alg = self.N * self.V * self.z.element_size()
+        gbs = alg / (ms * 1e-3) / 1e9
+        return {"metric": "token_logprobs_tokens_per_s", "value": self.N / (ms * 1e-3), "unit": UNIT, "ms_per_call": ms,
+                "steps": steps, "gpu_launches": steps,
+                "roofline": {"bound": "hbm", "kernel": "row_stream_kernel (forward only)", "achieved": gbs,
+                             "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+                             "peak_source": peaks["source"] + " (copy, burst)", "algorithmic_bytes_per_launch": alg,
+                             "traffic": None}}
+
     def measure_skip_zero_rows(self, steps=10):
         """The same step with MRL_FLAG_SKIP_ZERO_ROWS: rows of zero-advantage groups are not read (their gradient
         rows are still written, as zeros).  Reported beside the headline, which streams every row."""
@@ -599,6 +622,7 @@ def measure(wl, steps, warmup, world, local_rank, rank, peaks, with_e2e, with_cp
     out["e2e"] = run_e2e(args, wl, world) if with_e2e else None
     if world == 1 and hasattr(wl, "measure_skip_zero_rows") and wl.ratio_level == 0 and not wl.lp.logp_ref:
         out["skip_zero_rows"] = wl.measure_skip_zero_rows()
+        out["token_logprobs"] = wl.measure_forward_only(peaks)
     out["cpu_baseline"] = None
     if with_cpu and rank == 0 and world == 1:
         n, dt, sample = wl.time_oracle()
@@ -654,6 +678,7 @@ def run_ours(args, rank, world, local_rank):
         }
         if res.get("skip_zero_rows") is not None:
             line["skip_zero_rows"] = res["skip_zero_rows"]
+            line["token_logprobs"] = res["token_logprobs"]
         if lmhead is not None:
             line["lmhead"] = lmhead
         if thl is not None:
