@@ -346,10 +346,11 @@ class LmheadWorkload:
     """Config 5: N = 65,536 response tokens, H = 4,096, V = 151,936, bf16 hidden and LM-head weight; the logits
     are never stored; outputs logp, loss, dHidden, dW."""
 
-    def __init__(self, w: synth.Workload, seed: int, device, pair_tiles: bool = False):
+    def __init__(self, w: synth.Workload, seed: int, device, pair_tiles: bool = False, skip_zero_rows: bool = False):
         from paper_2605_07244_b200 import binding as B
         self.B = B
         self.pair_tiles = pair_tiles
+        self.skip_zero_rows = skip_zero_rows
         self.w = w
         self.meta = synth.make_meta(w, seed)
         self.batch = synth.make_batch(self.meta)
@@ -381,7 +382,8 @@ class LmheadWorkload:
         self.ws = torch.empty(B.workspace_bytes(B.WS_FUSED_LMHEAD, self.N, self.V, self.H, B.BF16, self.S),
                               dtype=torch.uint8, device=dev)
         self.ap = B.AdvParams(B.ADV_GROUP_ZNORM, 0, 1e-6, 0.8, 0.2, B.PICK_SHORTEST, 0)
-        self.lp = B.LossParams(0.2, 0.2, B.AGG_TOKEN_MEAN, B.FLAG_PAIR_TILES if pair_tiles else 0, 0.0, 0.0, 0.0, 0)
+        self.lp = B.LossParams(0.2, 0.2, B.AGG_TOKEN_MEAN, (B.FLAG_PAIR_TILES if pair_tiles else 0) |
+                               (B.FLAG_SKIP_ZERO_ROWS if skip_zero_rows else 0), 0.0, 0.0, 0.0, 0)
         # behaviour trace: logp_old = logp + N(0, 0.1); logp from a forward-only call (input preparation)
         B.mrl_group_advantages(self.rewards, self.seq_len, 0, self.ap, self.adv_own, self.adv_pool, self.rescue,
                                self.pick, self.nllw_seq, self.n_gated)
@@ -393,8 +395,19 @@ class LmheadWorkload:
         self.dominant_per_step = 1 + 3 * chunks          # forward GEMM, then (dZ, dHidden, dW) per vocabulary chunk
         # adv, seq_count, row_coef, forward GEMM, rows, row_terms, finalize, then 3 GEMMs per chunk
         self.kernels_per_step = 7 + 3 * chunks
-        self.flops_executed = 8.0 * self.N * self.H * self.V      # forward, recompute, dHidden, dW
-        self.flops_algorithmic = 6.0 * self.N * self.H * self.V   # without the recompute
+        # Blocks of 256 rows without any gradient are left out of the three backward products, and of the forward one
+        # too under MRL_FLAG_SKIP_ZERO_ROWS: count the rows of the blocks that are worked on (a block whose rows are
+        # all clipped is not expected and not counted as skipped).
+        lens = (self.cu[1:] - self.cu[:-1]).long()
+        row_live = torch.repeat_interleave(self.adv_own.reshape(-1) != 0, lens)
+        pad = (-self.N) % 256
+        blocks = torch.nn.functional.pad(row_live, (0, pad)).view(-1, 256).any(dim=1)
+        rows_bwd = min(int(blocks.sum()) * 256, self.N) if bool(blocks.any()) else min(256, self.N)
+        rows_fwd = rows_bwd if skip_zero_rows else self.N
+        self.rows_worked = {"forward": rows_fwd, "backward": rows_bwd}
+        hv = float(self.H) * self.V
+        self.flops_executed = 2.0 * hv * rows_fwd + 6.0 * hv * rows_bwd   # forward; recompute, dHidden, dW
+        self.flops_algorithmic = 2.0 * hv * rows_fwd + 4.0 * hv * rows_bwd   # without the recompute
 
     def step(self):
         B = self.B
@@ -412,6 +425,9 @@ class LmheadWorkload:
                             f"G=16 x T=64), H={self.H} bf16 hidden N(0,1), W[V={self.V},H] bf16 N(0,0.02^2), logits never "
                             "materialised, GRPO clipped surrogate, binary rewards, fwd+bwd -> dHidden, dW",
                 "rows": self.N, "sequences": self.S, "V": self.V, "H": self.H, "pair_tiles": self.pair_tiles,
+                "skip_zero_rows": self.skip_zero_rows,
+                "sequences_with_nonzero_advantage": int((self.adv_own != 0).sum()),
+                "rows_worked_on": self.rows_worked,
                 "l2": "operands (1.8 GB) and scratch exceed the 126 MB L2; no flush needed"}
 
     def roofline(self, kernel_ms, peaks):
@@ -640,13 +656,14 @@ def run_ours(args, rank, world, local_rank):
     from paper_2605_07244_b200 import build
     build.build()
     B.lib()
-    if args.workload not in ("C2", "C2s", "C5", "C5s"):
+    if args.workload not in ("C2", "C2s", "C5", "C5s", "C5b"):
         raise SystemExit("bench.py times config 2 (logits-in; C2s is its small profiling case) and config 5 "
                          "(fused LM head); the other configs are parity-test cases")
     peaks = measured_peaks()
-    lmhead_main = args.workload in ("C5", "C5s")
+    lmhead_main = args.workload in ("C5", "C5s", "C5b")
     cls = LmheadWorkload if lmhead_main else LogitsInWorkload
-    wl = (cls(synth.CONFIGS[args.workload], args.seed + rank, device, args.pair_tiles) if lmhead_main else
+    wl = (cls(synth.CONFIGS[args.workload], args.seed + rank, device, args.pair_tiles, args.skip_zero_rows)
+          if lmhead_main else
           cls(synth.CONFIGS[args.workload], args.seed + rank, device, 1 if args.ratio_level == "sequence" else 0,
               args.with_entropy, args.with_kl))
     res = measure(wl, args.steps, args.warmup, world, local_rank, rank, peaks, not args.no_e2e,
@@ -663,6 +680,11 @@ def run_ours(args, rank, world, local_rank):
         lmhead = {"metric": METRIC, "unit": UNIT, **{k: r5[k] for k in ("value", "ms_per_step", "steps", "config",
                                                                          "gpu_launches", "roofline", "cpu_baseline")}}
         del wl5
+        # the same shape with success rates drawn per prompt (many all-success / all-failure groups), zero rows skipped
+        wl5b = LmheadWorkload(synth.CONFIGS["C5b"], args.seed + rank, device, False, True)
+        r5b = measure(wl5b, min(args.steps, LMHEAD_SUB_STEPS), 3, world, local_rank, rank, peaks, False, False, args)
+        lmhead["skip_zero_rows"] = {k: r5b[k] for k in ("value", "ms_per_step", "steps", "config", "roofline")}
+        del wl5b
 
     thl = None
     if args.workload == "C2" and not args.no_lmhead and rank == 0 and world == 1:
@@ -703,6 +725,8 @@ def main():
     ap.add_argument("--with-entropy", action="store_true", help="logits-in workloads: also emit the per-row policy entropy")
     ap.add_argument("--e2e-slab-rows", type=int, default=1024,
                     help="logits-in end-to-end leg: rows per micro-batch of the host pipeline")
+    ap.add_argument("--skip-zero-rows", action="store_true",
+                    help="fused LM-head workloads: MRL_FLAG_SKIP_ZERO_ROWS (zero-multiplier rows are not produced)")
     ap.add_argument("--pair-tiles", action="store_true",
                     help="fused LM-head workloads: 256-row tiles worked by CTA pairs (MRL_FLAG_PAIR_TILES)")
     ap.add_argument("--no-lmhead", action="store_true", help="skip the short config-5 leg of the default run")

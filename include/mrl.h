@@ -91,8 +91,12 @@ extern "C" {
 /* mrl_loss_params.flags */
 #define MRL_FLAG_ACCUMULATE_LOSS 1u   /* loss[0..1] and stats += this call (micro-batch accumulation, App. A) */
 #define MRL_FLAG_SKIP_ZERO_ROWS 2u    /* rows whose gradient multiplier is known to be zero before reading the
-                                         logits (A = 0 or weight 0, and no NLL weight) are not read: logp = 0,
-                                         dlogits row = 0, they still count in the denominators */
+                                         logits (A = 0 or weight 0, and no NLL weight, no KL term) are not read:
+                                         logp = 0, dlogits row = 0, they still count in the denominators.  Fused
+                                         LM head: such rows report logp = 0 as well and blocks of 256 rows made of
+                                         them (or of masked rows) are left out of the forward product; blocks
+                                         without any gradient are left out of the backward products with or
+                                         without this flag (the results do not depend on it) */
 #define MRL_FLAG_ACCUMULATE_DW 4u     /* fused LM head: dW is float32 [V, H] and is added to, not overwritten */
 #define MRL_FLAG_PAIR_TILES 8u        /* fused LM head: 256-row tiles worked by pairs of CTAs (tcgen05 cta_group::2).
                                          Same results.  Faster for a product timed alone; inside a long

@@ -42,6 +42,11 @@ struct GemmParams {
   int M, N, K;
   int m_tiles, n_tiles, k_blocks;
   int group_m;            // row-tiles per raster group
+  // Optional compaction (device arrays; the counts are read by the kernel, so the host never waits for them):
+  const int* m_list;      // ascending indices of the row-tiles (of BM * kC rows) to work on; null = all of them
+  const int* m_count;     // [1] how many
+  const int* k_list;      // ascending indices of the K-blocks (of BK) to sum over; null = all of them
+  const int* k_count;     // [1]
   int32_t* status;
   // EPI_LSE
   float2* partial;        // [n_tiles][part_ld]: (running max, sum) of the tile's columns, base-2 domain
@@ -283,7 +288,9 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
   // a pair of CTAs (kC = 2) works on one tile of 256 rows: rank 0 leads (arms the barriers, issues the MMAs)
   const int rank = kC == 2 ? (int)(blockIdx.x & 1u) : 0;
   const int unit = (int)blockIdx.x / kC, n_units = (int)gridDim.x / kC;
-  const int total_tiles = p.m_tiles * p.n_tiles;
+  const int m_tiles = p.m_list != nullptr ? min(*p.m_count, p.m_tiles) : p.m_tiles;
+  const int k_blocks = p.k_list != nullptr ? min(*p.k_count, p.k_blocks) : p.k_blocks;
+  const int total_tiles = m_tiles * p.n_tiles;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
@@ -325,31 +332,49 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
       bool ok = true;
       for (int t = unit; t < total_tiles && ok; t += n_units) {
         int m, n;
-        tile_coords(t, p.m_tiles, p.n_tiles, p.group_m, m, n);
+        tile_coords(t, m_tiles, p.n_tiles, p.group_m, m, n);
+        if (p.m_list != nullptr) m = p.m_list[m];
         const int a_row = (m * kC + rank) * BM, b_row = n * BN + rank * Cfg::kBRows;
-        for (int kb = 0; kb < p.k_blocks; ++kb) {
-          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
-          const uint32_t a_dst = tiles + (uint32_t)stage * kStageBytes;
-          // the leader's barrier counts the bytes of both CTAs of a pair; only the leader arms it
-          const uint32_t bar = kC == 2 ? mapa_u32(full_bar(stage), 0u) : full_bar(stage);
-          if (rank == 0) mbar_expect_tx(full_bar(stage), (uint32_t)kC * kStageBytes);
-          auto load = [&](uint32_t dst, const CUtensorMap* map, int x, int y) {
-            if (kC == 2) tma_load_2d_pair(dst, map, x, y, bar); else tma_load_2d(dst, map, x, y, bar);
-          };
-          if (kAMn) {  // boxes of 64 rows-of-the-tile x BK
+        // K-block indices come from the list (when there is one) eight at a time and one group ahead, so that their
+        // loads never sit between two copies
+        auto k_index = [&](int kb) { return (p.k_list != nullptr && kb < k_blocks) ? __ldg(p.k_list + kb) : kb; };
+        int k_next[8];
 #pragma unroll
-            for (int j = 0; j < BM / 64; ++j) load(a_dst + (uint32_t)j * (BK * 128), &tmapA, a_row + 64 * j, kb * BK);
-          } else {
-            load(a_dst, &tmapA, kb * BK, a_row);
-          }
-          if (kBMn) {
+        for (int j = 0; j < 8; ++j) k_next[j] = k_index(j);
+        for (int kb0 = 0; kb0 < k_blocks && ok; kb0 += 8) {
+          int k_cur[8];
 #pragma unroll
-            for (int j = 0; j < Cfg::kBRows / 64; ++j)
-              load(a_dst + kABytes + (uint32_t)j * (BK * 128), &tmapB, b_row + 64 * j, kb * BK);
-          } else {
-            load(a_dst + kABytes, &tmapB, kb * BK, b_row);
+          for (int j = 0; j < 8; ++j) {
+            k_cur[j] = k_next[j];
+            k_next[j] = k_index(kb0 + 8 + j);
           }
-          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            if (kb0 + j >= k_blocks) break;
+            const int kx = k_cur[j] * BK;
+            if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+            const uint32_t a_dst = tiles + (uint32_t)stage * kStageBytes;
+            // the leader's barrier counts the bytes of both CTAs of a pair; only the leader arms it
+            const uint32_t bar = kC == 2 ? mapa_u32(full_bar(stage), 0u) : full_bar(stage);
+            if (rank == 0) mbar_expect_tx(full_bar(stage), (uint32_t)kC * kStageBytes);
+            auto load = [&](uint32_t dst, const CUtensorMap* map, int x, int y) {
+              if (kC == 2) tma_load_2d_pair(dst, map, x, y, bar); else tma_load_2d(dst, map, x, y, bar);
+            };
+            if (kAMn) {  // boxes of 64 rows-of-the-tile x BK
+#pragma unroll
+              for (int q = 0; q < BM / 64; ++q) load(a_dst + (uint32_t)q * (BK * 128), &tmapA, a_row + 64 * q, kx);
+            } else {
+              load(a_dst, &tmapA, kx, a_row);
+            }
+            if (kBMn) {
+#pragma unroll
+              for (int q = 0; q < Cfg::kBRows / 64; ++q)
+                load(a_dst + kABytes + (uint32_t)q * (BK * 128), &tmapB, b_row + 64 * q, kx);
+            } else {
+              load(a_dst + kABytes, &tmapB, kx, b_row);
+            }
+            if (++stage == kStages) { stage = 0; phase ^= 1u; }
+          }
         }
       }
     }
@@ -363,7 +388,7 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)acc * BN;
-        for (int kb = 0; kb < p.k_blocks; ++kb) {
+        for (int kb = 0; kb < k_blocks; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
           tc_fence_after();
           const uint32_t a_src = tiles + (uint32_t)stage * kStageBytes;
@@ -396,7 +421,8 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
     bool ok = true;
     for (int t = unit; t < total_tiles && ok; t += n_units) {
       int m, n;
-      tile_coords(t, p.m_tiles, p.n_tiles, p.group_m, m, n);
+      tile_coords(t, m_tiles, p.n_tiles, p.group_m, m, n);
+      if (p.m_list != nullptr) m = p.m_list[m];
       const int row = (m * kC + rank) * BM + row_in_tile;
       const bool row_ok = row < p.M;
       const int ncols_valid = min(BN, p.N - n * BN);
@@ -527,6 +553,91 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
 }
 
 // ------------------------------------------------------------------------------------------ small kernels
+// Does the forward product have to produce this (unmasked, in-range) row?
+__device__ __forceinline__ bool row_needs_forward(long long t, const float* rowA, const float* rowcu, const float* rowcn,
+                                                  const float* rowck, bool has_ref, uint32_t flags) {
+  if (!(flags & MRL_FLAG_SKIP_ZERO_ROWS)) return true;
+  const bool zero = (rowcu[t] == 0.f || rowA[t] == 0.f) && rowcn[t] == 0.f && (!has_ref || rowck[t] == 0.f);
+  return !zero;
+}
+
+// Liveness of every block of 256 rows.  mode 0 (backward): some row has g != 0.  mode 1 (forward): some row is
+// unmasked with an id in range and needs the forward product.  One warp per block of rows.
+__global__ void __launch_bounds__(256) tile_live_kernel(long long N, int n256, int mode, const float* __restrict__ g,
+                                                         const int32_t* __restrict__ ids,
+                                                         const uint8_t* __restrict__ mask, int V,
+                                                         const float* __restrict__ rowA,
+                                                         const float* __restrict__ rowcu,
+                                                         const float* __restrict__ rowcn,
+                                                         const float* __restrict__ rowck, bool has_ref, uint32_t flags,
+                                                         uint8_t* __restrict__ live) {
+  const int tile = (int)((blockIdx.x * 256u + threadIdx.x) >> 5), lane = threadIdx.x & 31;
+  if (tile >= n256) return;
+  bool any = false;
+  for (int r = lane; r < 256; r += 32) {
+    const long long t = (long long)tile * 256 + r;
+    if (t >= N) break;
+    if (mode == 0) {
+      any |= g[t] != 0.f;
+    } else {
+      const int id = ids[t];
+      const bool in_batch = (mask == nullptr || mask[t] != 0) && id >= 0 && id < V;
+      any |= in_batch && row_needs_forward(t, rowA, rowcu, rowcn, rowck, has_ref, flags);
+    }
+  }
+  any = __any_sync(0xffffffffu, any);
+  if (lane == 0) live[tile] = any ? 1 : 0;
+}
+
+// Ascending lists of the live blocks at the three granularities the products use: 256-row tiles (CTA pairs),
+// 128-row tiles, 64-row K-blocks; counts[0..2] = their lengths.  A batch without any live block lists block 0, so
+// that no product runs empty (its rows then contribute zeros).  One block; ordered, hence reproducible.
+__global__ void __launch_bounds__(1024) tile_lists_kernel(int n256, int n128, int n64, const uint8_t* __restrict__ live,
+                                                           int* __restrict__ m256, int* __restrict__ m128,
+                                                           int* __restrict__ k64, int* __restrict__ counts) {
+  __shared__ int warp_tot[32];
+  __shared__ int base_sh;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) base_sh = 0;
+  __syncthreads();
+  for (int c0 = 0; c0 < n256; c0 += 1024) {
+    const int t = c0 + tid;
+    const bool f = t < n256 && live[t] != 0;
+    const unsigned bal = __ballot_sync(0xffffffffu, f);
+    if (lane == 0) warp_tot[warp] = __popc(bal);
+    __syncthreads();
+    int off = base_sh;
+    for (int wi = 0; wi < warp; ++wi) off += warp_tot[wi];
+    if (f) {
+      const int pos = off + __popc(bal & ((1u << lane) - 1u));
+      m256[pos] = t;
+      for (int j = 0; j < 2; ++j) if (2 * t + j < n128) m128[2 * pos + j] = 2 * t + j;
+      for (int j = 0; j < 4; ++j) if (4 * t + j < n64) k64[4 * pos + j] = 4 * t + j;
+    }
+    __syncthreads();
+    if (tid == 0) {
+      int tot = 0;
+      for (int wi = 0; wi < 32; ++wi) tot += warp_tot[wi];
+      base_sh += tot;
+    }
+    __syncthreads();
+  }
+  if (tid == 0) {
+    int cnt = base_sh;
+    if (cnt == 0) {
+      m256[0] = 0;
+      for (int j = 0; j < 2 && j < n128; ++j) m128[j] = j;
+      for (int j = 0; j < 4 && j < n64; ++j) k64[j] = j;
+      cnt = 1;
+    }
+    // only the batch's last block of 256 rows can be short of 128- or 64-row blocks
+    const bool has_last = m256[cnt - 1] == n256 - 1;
+    counts[0] = cnt;
+    counts[1] = 2 * cnt - (has_last ? 2 * n256 - n128 : 0);
+    counts[2] = 4 * cnt - (has_last ? 4 * n256 - n64 : 0);
+  }
+}
+
 // Merges the per-tile partials of every row in tile order, then the row's ratio / clip / gradient multiplier.
 __global__ void __launch_bounds__(256) lmhead_rows_kernel(long long N, int V, int n_tiles, const float2* __restrict__ partial,
                                                            long long part_ld, const float* __restrict__ zt,
@@ -541,11 +652,14 @@ __global__ void __launch_bounds__(256) lmhead_rows_kernel(long long N, int V, in
                                                            float eps_hi, float* __restrict__ row_m2,
                                                            float* __restrict__ row_s, float* __restrict__ row_zt,
                                                            uint8_t* __restrict__ rowstat, float* __restrict__ g_out,
-                                                           float* __restrict__ lse2_out) {
+                                                           float* __restrict__ lse2_out, uint32_t flags) {
   const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= N) return;
   const int id = ids[t];
-  const bool valid = (mask == nullptr || mask[t] != 0) && id >= 0 && id < V;
+  const bool in_batch = (mask == nullptr || mask[t] != 0) && id >= 0 && id < V;
+  // under MRL_FLAG_SKIP_ZERO_ROWS a row whose multiplier is known to be zero is not read (its tile may not even
+  // have been computed): it reports logp = 0 and still counts in the denominators
+  const bool valid = in_batch && row_needs_forward(t, rowA, rowcu, rowcn, rowck, logp_ref != nullptr, flags);
   mrl::Lse2 acc = mrl::lse2_empty();
   if (valid)
     for (int n = 0; n < n_tiles; ++n) {
@@ -574,7 +688,7 @@ __global__ void __launch_bounds__(256) lmhead_rows_kernel(long long N, int V, in
   row_m2[t] = acc.m;
   row_s[t] = acc.s;
   row_zt[t] = valid ? zt[t] : 0.f;
-  rowstat[t] = st;
+  rowstat[t] = in_batch ? (st | MRL_ROW_VALID) : st;
   g_out[t] = g;
   lse2_out[t] = l2;
 }
@@ -642,9 +756,15 @@ int resident_pairs(cudaLaunchConfig_t* cfg) {
 
 // C[M, N] = A B^T.  A K-major operand is a row-major [rows = M or N, K] matrix; an MN-major one is a row-major
 // [K, rows] matrix (what the other one would be transposed), `ld` elements between its rows either way.
+// Compact lists of the blocks of rows that carry work (device arrays, see tile_lists_kernel).
+struct TileLists {
+  int *m256, *m128, *k64, *counts;
+};
+
+// `m_rows` / `k_rows`: the M (resp. K) dimension of the product is the batch's rows and only the listed blocks count.
 template <int EPI, bool kAMn, bool kBMn>
 int launch_gemm(const void* A, long long lda, const void* B, long long ldb, GemmParams p, bool pair_tiles,
-                cudaStream_t st) {
+                cudaStream_t st, const TileLists* m_rows = nullptr, const TileLists* k_rows = nullptr) {
   if (p.M <= 0 || p.N <= 0 || p.K <= 0) return MRL_OK;
   p.n_tiles = (p.N + BN - 1) / BN;
   p.k_blocks = (p.K + BK - 1) / BK;
@@ -671,6 +791,14 @@ int launch_gemm(const void* A, long long lda, const void* B, long long ldb, Gemm
   rc = kBMn ? make_tmap(&tb, B, p.K, p.N, ldb, BK) : make_tmap(&tb, B, p.N, p.K, ldb, BN / kC);
   if (rc != MRL_OK) return rc;
   p.m_tiles = (p.M + BM * kC - 1) / (BM * kC);
+  if (m_rows != nullptr) {
+    p.m_list = kC == 2 ? m_rows->m256 : m_rows->m128;
+    p.m_count = m_rows->counts + (kC == 2 ? 0 : 1);
+  }
+  if (k_rows != nullptr) {
+    p.k_list = k_rows->k64;
+    p.k_count = k_rows->counts + 2;
+  }
   // rows of A per raster group: a wave's operands should share L2; with a short K a taller group re-uses A
   // across the next waves as well (measured: 4,096 rows at K = 4,096, 2,048 rows at K >= 16,384)
   p.group_m = (kC == 2 && p.K <= 8192 ? 4096 : 2048) / (BM * kC);
@@ -702,6 +830,9 @@ struct LmheadWs {
   float2* partial;
   __nv_bfloat16* D;      // one vocabulary chunk of dZ, [N, ldD]
   float* dH_acc;
+  uint8_t* live;         // per block of 256 rows
+  TileLists fwd, bwd;    // rows the forward product has to produce / rows with a gradient
+  int n256, n128, n64;
   long long part_ld, ldD;
   int n_tiles_fwd, vchunk, n_chunks;
   size_t bytes;
@@ -722,6 +853,16 @@ LmheadWs carve_lmhead_ws(void* ws, long long N, int V, int H, int S) {
   w.ldD = w.vchunk;
   w.D = c.take<__nv_bfloat16>((size_t)N * (size_t)w.ldD);
   w.dH_acc = w.n_chunks > 1 ? c.take<float>((size_t)N * (size_t)H) : nullptr;
+  w.n256 = (int)((N + 255) / 256);
+  w.n128 = (int)((N + 127) / 128);
+  w.n64 = (int)((N + 63) / 64);
+  w.live = c.take<uint8_t>((size_t)w.n256);
+  for (TileLists* l : {&w.fwd, &w.bwd}) {
+    l->m256 = c.take<int>((size_t)w.n256);
+    l->m128 = c.take<int>((size_t)2 * w.n256);
+    l->k64 = c.take<int>((size_t)4 * w.n256);
+    l->counts = c.take<int>(4);
+  }
   w.bytes = c.off;
   return w;
 }
@@ -736,9 +877,10 @@ size_t mrl_fused_lmhead_workspace_bytes(long long N, int V, int H, int S) {
 // C[M, N] = A B^T with a plain store (bf16 or fp32, optionally added to): the building block of the two backward
 // products, also reachable on its own for checks of the tensor-core mainloop.  a_mn / b_mn: the operand is given
 // MN-major, i.e. as the row-major [K, M] (resp. [K, N]) matrix.
-int mrl_lmhead_gemm(const void* A, long long lda, bool a_mn, const void* B, long long ldb, bool b_mn, int M, int N, int K,
-                    void* C, long long ldc, int c_mode, float* Cacc, long long ldacc, int32_t* status, bool pair_tiles,
-                    cudaStream_t st) {
+static int lmhead_gemm_rows(const void* A, long long lda, bool a_mn, const void* B, long long ldb, bool b_mn, int M,
+                            int N, int K, void* C, long long ldc, int c_mode, float* Cacc, long long ldacc,
+                            int32_t* status, bool pair_tiles, cudaStream_t st, const TileLists* m_rows,
+                            const TileLists* k_rows) {
   GemmParams p = {};
   p.M = M;
   p.N = N;
@@ -749,10 +891,17 @@ int mrl_lmhead_gemm(const void* A, long long lda, bool a_mn, const void* B, long
   p.Cacc = Cacc;
   p.ldacc = ldacc;
   p.status = status;
-  if (a_mn && b_mn) return launch_gemm<EPI_STORE, true, true>(A, lda, B, ldb, p, pair_tiles, st);
-  if (b_mn) return launch_gemm<EPI_STORE, false, true>(A, lda, B, ldb, p, pair_tiles, st);
+  if (a_mn && b_mn) return launch_gemm<EPI_STORE, true, true>(A, lda, B, ldb, p, pair_tiles, st, m_rows, k_rows);
+  if (b_mn) return launch_gemm<EPI_STORE, false, true>(A, lda, B, ldb, p, pair_tiles, st, m_rows, k_rows);
   if (a_mn) return MRL_ERR_INVALID_ARG;  // not needed by the pass: not instantiated
-  return launch_gemm<EPI_STORE, false, false>(A, lda, B, ldb, p, pair_tiles, st);
+  return launch_gemm<EPI_STORE, false, false>(A, lda, B, ldb, p, pair_tiles, st, m_rows, k_rows);
+}
+
+int mrl_lmhead_gemm(const void* A, long long lda, bool a_mn, const void* B, long long ldb, bool b_mn, int M, int N, int K,
+                    void* C, long long ldc, int c_mode, float* Cacc, long long ldacc, int32_t* status, bool pair_tiles,
+                    cudaStream_t st) {
+  return lmhead_gemm_rows(A, lda, a_mn, B, ldb, b_mn, M, N, K, C, ldc, c_mode, Cacc, ldacc, status, pair_tiles, st,
+                          nullptr, nullptr);
 }
 
 extern "C" int mrl_fused_lmhead_loss_fwd_bwd(const void* hidden, const void* W, int64_t N, int32_t H, int32_t V,
@@ -803,6 +952,19 @@ extern "C" int mrl_fused_lmhead_loss_fwd_bwd(const void* hidden, const void* W, 
                             &rw);
   if (rc != MRL_OK) return rc;
   MRL_CUDA_OK(cudaMemsetAsync(w.zt, 0, (size_t)N * sizeof(float), st));
+  const bool seq_ratio = lp->ratio_level == MRL_RATIO_SEQUENCE;
+  // a response-level ratio needs every valid row of a response for its sum: nothing is skipped on the way forward
+  const uint32_t row_flags = seq_ratio ? (lp->flags & ~MRL_FLAG_SKIP_ZERO_ROWS) : lp->flags;
+  const bool has_ref = !seq_ratio && lp->logp_ref != nullptr;
+  const unsigned live_grid = (unsigned)((w.n256 + 7) / 8);
+
+  // ---- which blocks of rows the forward product has to produce (all-masked blocks never; zero-multiplier blocks
+  // not under MRL_FLAG_SKIP_ZERO_ROWS)
+  tile_live_kernel<<<live_grid, 256, 0, st>>>(N, w.n256, 1, nullptr, ids, mask, V, rw.rowA, rw.rowcu, rw.rowcn, rw.rowck,
+                                              has_ref, row_flags, w.live);
+  MRL_CUDA_OK(cudaGetLastError());
+  tile_lists_kernel<<<1, 1024, 0, st>>>(w.n256, w.n128, w.n64, w.live, w.fwd.m256, w.fwd.m128, w.fwd.k64, w.fwd.counts);
+  MRL_CUDA_OK(cudaGetLastError());
 
   // ---- forward: per-tile log-sum-exp partials and the target logit, logits never stored
   {
@@ -816,16 +978,15 @@ extern "C" int mrl_fused_lmhead_loss_fwd_bwd(const void* hidden, const void* W, 
     p.ids = ids;
     p.zt = w.zt;
     p.col0 = 0;
-    rc = launch_gemm<EPI_LSE, false, false>(hid, H, Wm, H, p, pair, st);
+    rc = launch_gemm<EPI_LSE, false, false>(hid, H, Wm, H, p, pair, st, &w.fwd);
     if (rc != MRL_OK) return rc;
   }
-  const bool seq_ratio = lp->ratio_level == MRL_RATIO_SEQUENCE;
   lmhead_rows_kernel<<<(unsigned)((N + 255) / 256), 256, 0, st>>>(N, V, w.n_tiles_fwd, w.partial, w.part_ld, w.zt, ids,
                                                                   mask, rw.rowA, rw.rowcu, rw.rowcn, rw.rowck,
                                                                   seq_ratio ? nullptr : lp->logp_ref, lp->kl_estimator,
                                                                   seq_ratio ? nullptr : logp_old, lp->eps_lo,
                                                                   lp->eps_hi, rw.row_m2, rw.row_s, rw.row_zt,
-                                                                  rw.rowstat, w.g, w.lse2);
+                                                                  rw.rowstat, w.g, w.lse2, row_flags);
   MRL_CUDA_OK(cudaGetLastError());
   if (seq_ratio)  // response-level ratio: g_t comes from the whole response (App. H)
     rc = mrl_rows_finish_sequence(rw, N, S, cu_seqlens, adv_seq, logp_old, nll_weight, lp, logp, loss, stats, w.g,
@@ -834,6 +995,15 @@ extern "C" int mrl_fused_lmhead_loss_fwd_bwd(const void* hidden, const void* W, 
     rc = mrl_rows_finish(rw, N, logp_old, lp, logp, loss, stats, st);
   if (rc != MRL_OK) return rc;
   if (dHidden == nullptr) return MRL_OK;
+
+  // ---- blocks of rows with a gradient: the rest (zero advantage, clipped, masked) is left out of all three backward
+  // products -- their dHidden rows are zero, and they add nothing to dW
+  tile_live_kernel<<<live_grid, 256, 0, st>>>(N, w.n256, 0, w.g, nullptr, nullptr, V, nullptr, nullptr, nullptr, nullptr,
+                                              false, 0u, w.live);
+  MRL_CUDA_OK(cudaGetLastError());
+  tile_lists_kernel<<<1, 1024, 0, st>>>(w.n256, w.n128, w.n64, w.live, w.bwd.m256, w.bwd.m128, w.bwd.k64, w.bwd.counts);
+  MRL_CUDA_OK(cudaGetLastError());
+  MRL_CUDA_OK(cudaMemsetAsync(dHidden, 0, (size_t)N * H * 2, st));
 
   // ---- backward, per vocabulary chunk.  No operand is transposed in memory: W and hidden enter the two products
   // MN-major, D enters dHidden's K-major and dW's MN-major.
@@ -852,22 +1022,22 @@ extern "C" int mrl_fused_lmhead_loss_fwd_bwd(const void* hidden, const void* W, 
       p.lse2 = w.lse2;
       p.D = w.D;
       p.ldD = w.ldD;
-      rc = launch_gemm<EPI_DZ, false, false>(hid, H, Wm + (size_t)v0 * H, H, p, pair, st);
+      rc = launch_gemm<EPI_DZ, false, false>(hid, H, Wm + (size_t)v0 * H, H, p, pair, st, &w.bwd);
       if (rc != MRL_OK) return rc;
     }
     {  // dHidden[N, H] (+)= D[N, vc] * W[v0 : v0 + vc, :]   (A = D K-major; B = the chunk of W, [K = vc, N = H])
       int mode = C_BF16;
       if (w.n_chunks > 1) mode = ch == 0 ? C_F32 : (ch == w.n_chunks - 1 ? C_BF16_FROM_ACC : C_F32_ADD);
       void* C = (mode == C_BF16 || mode == C_BF16_FROM_ACC) ? dHidden : static_cast<void*>(w.dH_acc);
-      rc = mrl_lmhead_gemm(w.D, w.ldD, false, Wm + (size_t)v0 * H, H, true, (int)N, H, vc, C, H, mode, w.dH_acc, H,
-                           status, pair, st);
+      rc = lmhead_gemm_rows(w.D, w.ldD, false, Wm + (size_t)v0 * H, H, true, (int)N, H, vc, C, H, mode, w.dH_acc, H,
+                            status, pair, st, &w.bwd, nullptr);
       if (rc != MRL_OK) return rc;
     }
     {  // dW[v0 : v0 + vc, :] = D^T hidden   (A = D as [K = N, M = vc]; B = hidden as [K = N, N = H])
       void* C = accum_dw ? static_cast<void*>(static_cast<float*>(dW) + (size_t)v0 * H)
                          : static_cast<void*>(static_cast<__nv_bfloat16*>(dW) + (size_t)v0 * H);
-      rc = mrl_lmhead_gemm(w.D, w.ldD, true, hid, H, true, vc, H, (int)N, C, H, accum_dw ? C_F32_ADD : C_BF16, nullptr, 0,
-                           status, pair, st);
+      rc = lmhead_gemm_rows(w.D, w.ldD, true, hid, H, true, vc, H, (int)N, C, H, accum_dw ? C_F32_ADD : C_BF16, nullptr,
+                            0, status, pair, st, nullptr, &w.bwd);
       if (rc != MRL_OK) return rc;
     }
   }

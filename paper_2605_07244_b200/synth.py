@@ -56,7 +56,9 @@ C6 = Workload("C6-appA-pool-3072", P=4, M=2, G=5, V=128256, dtype=torch.bfloat16
 C2_SMALL = replace(C2, name="C2-qwen-vocab-2-prompts", P=2)
 # config 5 with an eighth of the rows and two vocabulary chunks: operands and scratch still exceed L2
 C5_SMALL = replace(C5, name="C5-fused-lmhead-8k-rows-32k-vocab", P=8, V=32768)
-CONFIGS = {"C1": C1, "C2": C2, "C3": C3, "C4": C4, "C5": C5, "C6": C6, "C2s": C2_SMALL, "C5s": C5_SMALL}
+# config 5 with per-prompt success rates drawn like the logits-in configs: many groups are all-success or all-failure
+C5_BETA = replace(C5, name="C5-fused-lmhead-beta-success-rates", reward_beta=True)
+CONFIGS = {"C1": C1, "C2": C2, "C3": C3, "C4": C4, "C5": C5, "C6": C6, "C2s": C2_SMALL, "C5s": C5_SMALL, "C5b": C5_BETA}
 
 
 def scaled(w: Workload, **kw) -> Workload:
