@@ -1,12 +1,12 @@
 #!/usr/bin/env python
 """Benchmark of the policy-loss hot path on B200 (one process per GPU).
 
-    python bench.py --gpus N --steps K --warmup W [--impl reference] [--workload C2|C2s|C5]
+    python bench.py --gpus N --steps K --warmup W [--impl reference] [--workload C2|C2s|C5|C5s|C5b]
 
 A step is one pass of the whole hot path over one batch of synthetic input: group advantages and
 SGT gate (mrl_group_advantages), then log-probs, ratio, clipped surrogate, aggregation and dlogits
-(mrl_policy_loss_fwd_bwd).  The workload at N = 1 is config 2 of the baseline (Qwen-size vocabulary,
-logits in, bf16, packed ragged sequences); each rank of an N-GPU run processes its own batch of the
+(mrl_policy_loss_fwd_bwd).  The workload at N = 1 is the Qwen-size-vocabulary configuration (151,936 columns,
+logits in, bf16, packed ragged sequences; `C2` in synth.py); each rank of an N-GPU run processes its own batch of the
 same shape (independent replicas, no data-path collective), so scaling is weak.
 
 Rank 0 prints ONE JSON line.  `--impl reference` times the CPU float64 oracle on a bounded sample
