@@ -14,6 +14,11 @@ namespace {
 constexpr int kThreads = 256;        // general kernel
 constexpr int kStreamThreads = 512;  // streaming kernel: two CTAs per SM
 constexpr long long kSplitRowBytes = 512 * 1024;  // rows at least this long are split over a cluster of two CTAs
+// Shared memory per CTA that holds the oldest vectors of its row between the passes.  More is not better: the
+// carve-out comes out of L1, and L1 is what keeps this kernel's loads in flight (measured on B200, ms per step on
+// 34 k rows of 304 KB, half / all of them with a gradient: 0 KB 3.40 / 3.88, 32 KB 3.35 / 3.82, 48 KB 3.35 / 3.79,
+// 64 KB 3.37 / 3.81, 80 KB 3.38 / 3.79, 96 KB 4.09 / 4.37).
+constexpr int kParkBytes = 48 * 1024;
 
 // rowstat bits
 constexpr uint8_t kStatValid = MRL_ROW_VALID, kStatClipped = MRL_ROW_CLIPPED, kStatRead = MRL_ROW_READ;
@@ -44,6 +49,7 @@ struct RowParams {
   float* row_zt;
   uint8_t* rowstat;
   int32_t* status;
+  int keep_q;  // streaming kernel: how many groups of blockDim vectors, the first ones pass 1 reads, are parked
 };
 
 // Everything the loss needs from one row besides the logits.
@@ -112,7 +118,7 @@ __device__ __forceinline__ uint32_t hmax2_u32(uint32_t a, uint32_t b) {
 }
 
 // ------------------------------------------------------------------------------------------------
-// Streaming kernel: bf16, one CTA per row, nothing resident in shared memory.
+// Streaming kernel: bf16, one CTA per row; shared memory holds only the few vectors parked between the passes.
 // Pass 1 streams the row from HBM with 128- or 256-bit loads (running maximum and rescaled sum per thread);
 // pass 2 reads the same vectors again (all but the group that is still in registers) -- by then from L2: the rows in flight (two per SM) are a fraction of its
 // capacity, and the first read asks L2 to keep the lines -- and writes g * (softmax - onehot) with streaming
@@ -179,6 +185,31 @@ __device__ __forceinline__ void stream_st(void* p, const StreamVec<kWords>& v) {
                  : "memory");
   }
 }
+// A thread's own vectors parked in shared memory between the passes (only the thread that wrote one reads it back,
+// so no barrier is needed).  256-bit vectors are kept as two planes of 16-byte halves: every 16-byte access of a
+// warp is then contiguous.
+template <int kWords>
+__device__ __forceinline__ void park_st(uint32_t base, uint32_t plane_bytes, uint32_t slot, const StreamVec<kWords>& v) {
+  const uint32_t a = base + slot * 16u;
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(v.w[0]), "r"(v.w[1]), "r"(v.w[2]), "r"(v.w[3])
+               : "memory");
+  if constexpr (kWords == 8)
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a + plane_bytes), "r"(v.w[4]), "r"(v.w[5]), "r"(v.w[6]),
+                 "r"(v.w[7])
+                 : "memory");
+}
+template <int kWords>
+__device__ __forceinline__ StreamVec<kWords> park_ld(uint32_t base, uint32_t plane_bytes, uint32_t slot) {
+  StreamVec<kWords> v;
+  const uint32_t a = base + slot * 16u;
+  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.w[0]), "=r"(v.w[1]), "=r"(v.w[2]), "=r"(v.w[3]) : "r"(a));
+  if constexpr (kWords == 8)
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.w[4]), "=r"(v.w[5]), "=r"(v.w[6]), "=r"(v.w[7])
+                 : "r"(a + plane_bytes));
+  return v;
+}
+
 template <int kWords>
 __device__ __forceinline__ StreamVec<kWords> stream_fill(uint32_t x) {
   StreamVec<kWords> v;
@@ -198,7 +229,10 @@ __global__ void __launch_bounds__(kT, 1024 / kT) row_stream_kernel(const RowPara
   __shared__ float fin[4];
   __shared__ __align__(16) float4 xchg[2];
   __shared__ __align__(8) uint64_t xbar;
+  extern __shared__ __align__(16) unsigned char parked[];  // keep_q * kT vectors
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int keep_q = p.keep_q;
+  const uint32_t park_base = smem_u32(parked), park_plane = (uint32_t)keep_q * kT * 16u;
   const long long row = blockIdx.x / kC;
   const int rank = blockIdx.x % kC;  // rank in the 1-D cluster
   const int row_nvec = p.V / kVecElems;
@@ -250,6 +284,14 @@ __global__ void __launch_bounds__(kT, 1024 / kT) row_stream_kernel(const RowPara
       for (int u = 0; u < kU; ++u)
         v[u] = (base + u * kT + tid < nvec) ? stream_ld<kWords, kHintKeep>(in + (size_t)(base + u * kT) * kVecBytes)
                                             : stream_fill<kWords>(0xff80ff80u);  // (-inf, -inf)
+    }
+    // the first vectors read are the ones L2 is likeliest to have dropped by pass 2: park them
+    const int q0 = ((last_base - base) / (kT * kU)) * kU;
+    if (q0 < keep_q) {
+#pragma unroll
+      for (int u = 0; u < kU; ++u)
+        if (q0 + u < keep_q && base + u * kT + tid < nvec)
+          park_st<kWords>(park_base, park_plane, (uint32_t)((q0 + u) * kT + tid), v[u]);
     }
     uint32_t mx = 0xff80ff80u;
 #pragma unroll
@@ -378,14 +420,16 @@ __global__ void __launch_bounds__(kT, 1024 / kT) row_stream_kernel(const RowPara
   const float neg_k = -(lse2 - log2f(fabsf(g)));  // 2^(z log2e - k) = |g| softmax(z)
   const uint32_t sign = g < 0.f ? 0x80008000u : 0u;
   // (the first group is still in registers; the others in the order pass 1 read them last-to-first, so the most
-  // recently loaded lines, the likeliest to be still in L2, come first)
+  // recently loaded lines, the likeliest to be still in L2, come first; the oldest come back from shared memory)
   for (int base = 0; base <= last_base; base += kT * kU) {
     const bool full = base + kT * kU <= nvec;
     if (base != 0) {
+      const int q0 = ((last_base - base) / (kT * kU)) * kU;
 #pragma unroll
       for (int u = 0; u < kU; ++u)
-        v[u] = (full || base + u * kT + tid < nvec) ? stream_ld<kWords, kHintLast>(in + (size_t)(base + u * kT) * kVecBytes)
-                                                    : stream_fill<kWords>(0u);
+        v[u] = !(full || base + u * kT + tid < nvec) ? stream_fill<kWords>(0u)
+               : (q0 + u < keep_q)                   ? park_ld<kWords>(park_base, park_plane, (uint32_t)((q0 + u) * kT + tid))
+                                                     : stream_ld<kWords, kHintLast>(in + (size_t)(base + u * kT) * kVecBytes);
     }
 #pragma unroll
     for (int u = 0; u < kU; ++u) {
@@ -851,10 +895,13 @@ int launch_rows(RowParams p, int dtype, cudaStream_t st) {
   const bool split = (long long)p.V * 2 >= kSplitRowBytes && p.N <= 0x3fffffffll && p.entropy == nullptr;
   const bool ent = p.entropy != nullptr;
   const int C = split ? 2 : 1;
+  // gradient launches of whole rows park the vectors read first (whole groups of blockDim vectors)
+  p.keep_q = (p.dlogits != nullptr && !split) ? kParkBytes / (kStreamThreads * words * 4) : 0;
+  const size_t park_bytes = (size_t)p.keep_q * kStreamThreads * words * 4;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(n * (unsigned)C);
   cfg.blockDim = dim3(kStreamThreads);
-  cfg.dynamicSmemBytes = 0;
+  cfg.dynamicSmemBytes = park_bytes;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -863,16 +910,22 @@ int launch_rows(RowParams p, int dtype, cudaStream_t st) {
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  using Kernel = void (*)(const RowParams);
+  const Kernel k = words == 8 ? (split ? row_stream_kernel<kStreamThreads, 4, 8, 2, false>
+                                 : ent ? row_stream_kernel<kStreamThreads, 4, 8, 1, true>
+                                       : row_stream_kernel<kStreamThreads, 4, 8, 1, false>)
+                              : (split ? row_stream_kernel<kStreamThreads, 8, 4, 2, false>
+                                 : ent ? row_stream_kernel<kStreamThreads, 8, 4, 1, true>
+                                       : row_stream_kernel<kStreamThreads, 8, 4, 1, false>);
+  if (park_bytes > 0) {
+    // exactly the carve-out two CTAs per SM need, as a percentage of the 228 KB an SM can give: the rest stays L1
+    const int carve = (int)((2 * (park_bytes + 2048) * 100 + 228 * 1024 - 1) / (228 * 1024));
+    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)park_bytes) != cudaSuccess ||
+        cudaFuncSetAttribute(k, cudaFuncAttributePreferredSharedMemoryCarveout, carve < 100 ? carve : 100) != cudaSuccess)
+      return MRL_ERR_CUDA;
+  }
   mrl_profile_before(st);
-  cudaError_t e;
-  if (words == 8)
-    e = split ? cudaLaunchKernelEx(&cfg, row_stream_kernel<kStreamThreads, 4, 8, 2, false>, p)
-        : ent ? cudaLaunchKernelEx(&cfg, row_stream_kernel<kStreamThreads, 4, 8, 1, true>, p)
-              : cudaLaunchKernelEx(&cfg, row_stream_kernel<kStreamThreads, 4, 8, 1, false>, p);
-  else
-    e = split ? cudaLaunchKernelEx(&cfg, row_stream_kernel<kStreamThreads, 8, 4, 2, false>, p)
-        : ent ? cudaLaunchKernelEx(&cfg, row_stream_kernel<kStreamThreads, 8, 4, 1, true>, p)
-              : cudaLaunchKernelEx(&cfg, row_stream_kernel<kStreamThreads, 8, 4, 1, false>, p);
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, k, p);
   mrl_profile_after(st);
   return e == cudaSuccess ? MRL_OK : MRL_ERR_CUDA;
 }
