@@ -120,10 +120,12 @@ __device__ __forceinline__ uint32_t hmax2_u32(uint32_t a, uint32_t b) {
 // ------------------------------------------------------------------------------------------------
 // Streaming kernel: bf16, one CTA per row; shared memory holds only the few vectors parked between the passes.
 // Pass 1 streams the row from HBM with 128- or 256-bit loads (running maximum and rescaled sum per thread);
-// pass 2 reads the same vectors again (all but the group that is still in registers) -- by then from L2: the rows in flight (two per SM) are a fraction of its
-// capacity, and the first read asks L2 to keep the lines -- and writes g * (softmax - onehot) with streaming
-// stores.  HBM sees one read and one write of the row.  Many small CTAs with deep unrolling keep far more bytes
-// in flight per SM than a slice held in shared memory does, which is what this memory-bound pass needs.
+// pass 2 needs the same vectors again: the last group read is still in registers, the first 48 KB read were
+// parked in shared memory, the rest comes from L2 -- the rows in flight (two per SM) are a fraction of its
+// capacity, and the first read asks L2 to keep the lines -- and g * (softmax - onehot) leaves with streaming
+// stores.  HBM sees one read and one write of the row (plus the second reads L2 misses).  Many small CTAs with
+// deep unrolling keep far more bytes in flight per SM than a slice fetched into shared memory does, which is what
+// this memory-bound pass needs.
 // ------------------------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ uint32_t mapa_u32(uint32_t addr, uint32_t rank) {
