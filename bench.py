@@ -481,6 +481,42 @@ class LmheadWorkload:
         return n, dt, f"first {n} rows of the same batch, full V and H, fwd+bwd incl. dW, float64, {dt:.1f} s"
 
 
+def measure_tiny_latency(seed):
+    """Config 1 (P = 4, G = 4, T = 64: 1,024 rows of 1,024 float32 logits, 4 MiB, L2-resident): a step is launch-bound,
+    so it is reported as time per step, launched call by call and replayed from a CUDA graph."""
+    wl = LogitsInWorkload(synth.CONFIGS["C1"], seed, torch.device("cuda", torch.cuda.current_device()))
+    reps = 200
+    side = torch.cuda.Stream()
+    B = wl.B
+
+    def step(stream):
+        B.mrl_group_advantages(wl.rewards, wl.seq_len, 0, wl.ap, wl.adv_own, wl.adv_pool, wl.rescue, wl.pick,
+                               wl.nllw_seq, wl.n_gated, stream=stream)
+        B.mrl_policy_loss_fwd_bwd(wl.z, wl.ids, None, wl.cu, wl.adv_own, wl.logp_old, None, None, wl.lp, wl.dz, wl.logp,
+                                  wl.loss, wl.stats, wl.status, wl.ws, stream=stream)
+
+    def timed(f):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(side):
+            for _ in range(10):
+                f()
+            side.synchronize()
+            e0.record(side)
+            for _ in range(reps):
+                f()
+            e1.record(side)
+        side.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / reps
+
+    direct = timed(lambda: step(side))
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        step(side)
+    replay = timed(graph.replay)
+    return {"workload": wl.w.name, "rows": wl.N, "V": wl.V, "us_per_step_direct": direct, "us_per_step_graph": replay,
+            "kernels_per_step": wl.kernels_per_step, "steps": reps, "status": int(wl.status.cpu())}
+
+
 def measure_thl_align(seed, with_cpu):
     """THL word alignment on a batch shaped like one PRP step of App. G.1: 256 prompts x 5 peer rollouts of
     ~630 response tokens, words cut into 1..4 tokens by each tokenizer.  It is tiny next to the loss pass (a few
@@ -686,9 +722,10 @@ def run_ours(args, rank, world, local_rank):
         lmhead["skip_zero_rows"] = {k: r5b[k] for k in ("value", "ms_per_step", "steps", "config", "roofline")}
         del wl5b
 
-    thl = None
+    thl = tiny = None
     if args.workload == "C2" and not args.no_lmhead and rank == 0 and world == 1:
         thl = measure_thl_align(args.seed, not args.no_cpu_baseline)
+        tiny = measure_tiny_latency(args.seed)
 
     if rank == 0:
         line = {
@@ -705,6 +742,8 @@ def run_ours(args, rank, world, local_rank):
             line["lmhead"] = lmhead
         if thl is not None:
             line["thl_align"] = thl
+        if tiny is not None:
+            line["tiny_step_latency"] = tiny
         print(json.dumps(line))
 
 
