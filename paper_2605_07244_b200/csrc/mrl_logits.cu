@@ -157,7 +157,7 @@ __device__ __forceinline__ StreamVec<kWords> stream_ld(const void* p) {
   StreamVec<kWords> v;
   if constexpr (kWords == 8) {
     if constexpr (kHint == kHintKeep)
-      asm volatile("ld.global.L2::evict_last.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+      asm volatile("ld.global.L1::no_allocate.L2::evict_last.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
                    : "=r"(v.w[0]), "=r"(v.w[1]), "=r"(v.w[2]), "=r"(v.w[3]), "=r"(v.w[4]), "=r"(v.w[5]), "=r"(v.w[6]),
                      "=r"(v.w[7])
                    : "l"(p));
