@@ -128,10 +128,10 @@ typedef struct mrl_loss_params {
   double seq_denominator;   /* SEQ_MEAN_TOKEN_MEAN: number of sequences of the whole step; <= 0: S */
   float nll_coeff;          /* lambda_SGT / n_gated (Eq. (2), App. B); 0 disables the NLL term */
   int32_t ratio_level;      /* MRL_RATIO_*; 0 (token level) is the default */
-  float* entropy;           /* [device] float32 [N], nullable.  mrl_policy_loss_fwd_bwd only (must be NULL for the
-                               fused LM head): entropy - sum_v p_v log p_v of softmax(z_t) at every valid row, 0
-                               elsewhere -- the policy-entropy diagnostic of Sec. 6 / App. B, taken from the same
-                               pass over the logits (one more FMA per logit) */
+  float* entropy;           /* [device] float32 [N], nullable: entropy - sum_v p_v log p_v of softmax(z_t) at every valid
+                               row that is read, 0 elsewhere -- the policy-entropy diagnostic of Sec. 6 / App. B,
+                               taken from the same pass (one more FMA per logit; on the fused LM head one more
+                               float per row and column tile of scratch traffic) */
   const float* logp_ref;    /* [device] float32 [N], nullable: no KL term.  Reference policy's log-prob of ids[t] */
   float kl_coeff;           /* beta of Eq. (1); App. A uses 1e-3 */
   int32_t kl_estimator;     /* MRL_KL_* */

@@ -35,7 +35,7 @@ struct GemmCfg {
 constexpr uint32_t kWaitLimit = 1u << 24;   // mbarrier polls before a wait gives up (of the order of a second)
 constexpr int kVChunk = 16384;              // vocabulary columns per backward chunk (multiple of BN)
 
-enum { EPI_LSE = 0, EPI_DZ = 1, EPI_STORE = 2 };
+enum { EPI_LSE = 0, EPI_DZ = 1, EPI_STORE = 2, EPI_LSE_ENT = 3 };  // _ENT: also sum_v 2^(x_v - m) z_v, for the entropy
 enum { C_BF16 = 0, C_F32 = 1, C_F32_ADD = 2, C_BF16_FROM_ACC = 3 };
 
 struct GemmParams {
@@ -50,6 +50,7 @@ struct GemmParams {
   int32_t* status;
   // EPI_LSE
   float2* partial;        // [n_tiles][part_ld]: (running max, sum) of the tile's columns, base-2 domain
+  float* partial_u;       // EPI_LSE_ENT: [n_tiles][part_ld] sum of 2^(x - max) z over the tile's columns
   long long part_ld;
   const int32_t* ids;     // [M]
   float* zt;              // [M] target logit
@@ -217,8 +218,10 @@ __device__ __forceinline__ void tile_coords(int t, int m_tiles, int n_tiles, int
 struct LseRow {
   float m, s, zt;
   bool has;
+  float u;  // sum of 2^(x - m) z (kEnt only)
 };
 
+template <bool kEnt>
 __device__ __forceinline__ void epi_lse_batch(const float* v, int c, int ncols_valid, int rel_id, LseRow& st) {
   float bm = -INFINITY;
 #pragma unroll
@@ -226,15 +229,26 @@ __device__ __forceinline__ void epi_lse_batch(const float* v, int c, int ncols_v
     if (c + j < ncols_valid) bm = fmaxf(bm, v[j]);
   if (bm == -INFINITY) return;  // no valid column in this batch
   const float m_new = fmaxf(st.m, bm * MRL_LOG2E);
-  st.s *= mrl::ex2_approx(st.m - m_new);  // first batch: 0 * 2^-inf = 0
+  const float f = mrl::ex2_approx(st.m - m_new);  // first batch: 0 * 2^-inf = 0
+  st.s *= f;
+  if (kEnt) st.u *= f;
   st.m = m_new;
-  float s0 = 0.f, s1 = 0.f;
+  float s0 = 0.f, s1 = 0.f, u0 = 0.f, u1 = 0.f;
 #pragma unroll
   for (int j = 0; j < 32; j += 2) {
-    if (c + j < ncols_valid) s0 += mrl::ex2_approx(fmaf(v[j], MRL_LOG2E, -m_new));
-    if (c + j + 1 < ncols_valid) s1 += mrl::ex2_approx(fmaf(v[j + 1], MRL_LOG2E, -m_new));
+    if (c + j < ncols_valid) {
+      const float e = mrl::ex2_approx(fmaf(v[j], MRL_LOG2E, -m_new));
+      s0 += e;
+      if (kEnt) u0 = e != 0.f ? fmaf(e, v[j], u0) : u0;  // e = 0 exactly where z = -inf: keep 0 * inf out
+    }
+    if (c + j + 1 < ncols_valid) {
+      const float e = mrl::ex2_approx(fmaf(v[j + 1], MRL_LOG2E, -m_new));
+      s1 += e;
+      if (kEnt) u1 = e != 0.f ? fmaf(e, v[j + 1], u1) : u1;
+    }
   }
   st.s += s0 + s1;
+  if (kEnt) st.u += u0 + u1;
   if (rel_id >= c && rel_id < c + 32) {
 #pragma unroll
     for (int j = 0; j < 32; ++j)
@@ -270,6 +284,7 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
   using Cfg = GemmCfg<kC>;
   constexpr int kStages = Cfg::kStages;
   constexpr uint32_t kStageBytes = Cfg::kStageBytes;
+  constexpr bool kLse = EPI == EPI_LSE || EPI == EPI_LSE_ENT;
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_addr(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;  // swizzled tiles need 1024-byte alignment
@@ -427,10 +442,10 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
       const bool row_ok = row < p.M;
       const int ncols_valid = min(BN, p.N - n * BN);
       // per-row inputs before the accumulator is ready
-      LseRow st = {-INFINITY, 0.f, 0.f, false};
+      LseRow st = {-INFINITY, 0.f, 0.f, false, 0.f};
       int rel_id = -1;
       float g = 0.f, neg_k = 0.f, l2 = 0.f, sgn = 1.f;
-      if (EPI == EPI_LSE) {
+      if (kLse) {
         if (row_ok) rel_id = p.ids[row] - (p.col0 + n * BN);
       } else if (EPI == EPI_DZ) {
         if (row_ok) {
@@ -449,8 +464,8 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
         if (c >= ncols_valid) break;  // uniform across the CTA
         float v[32];
         tc_ld32(t_row + (uint32_t)c, v);
-        if (EPI == EPI_LSE) {
-          epi_lse_batch(v, c, ncols_valid, rel_id, st);
+        if (kLse) {
+          epi_lse_batch<EPI == EPI_LSE_ENT>(v, c, ncols_valid, rel_id, st);
         } else if (EPI == EPI_DZ) {
           float d[32];
           if (g == 0.f) {
@@ -523,8 +538,9 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
       if (lane == 0) {  // the leader's barrier collects the epilogue warps of both CTAs
         if (kC == 2 && rank != 0) mbar_arrive_remote(mapa_u32(tempty_bar(acc), 0u)); else mbar_arrive(tempty_bar(acc));
       }
-      if (EPI == EPI_LSE && row_ok) {
+      if (kLse && row_ok) {
         p.partial[(long long)n * p.part_ld + row] = make_float2(st.m, st.s);
+        if (EPI == EPI_LSE_ENT) p.partial_u[(long long)n * p.part_ld + row] = st.u;
         if (st.has) p.zt[row] = st.zt;
       }
       if (++acc == kAccStages) { acc = 0; acc_phase ^= 1u; }
@@ -640,6 +656,7 @@ __global__ void __launch_bounds__(1024) tile_lists_kernel(int n256, int n128, in
 
 // Merges the per-tile partials of every row in tile order, then the row's ratio / clip / gradient multiplier.
 __global__ void __launch_bounds__(256) lmhead_rows_kernel(long long N, int V, int n_tiles, const float2* __restrict__ partial,
+                                                           const float* __restrict__ partial_u, float* __restrict__ entropy,
                                                            long long part_ld, const float* __restrict__ zt,
                                                            const int32_t* __restrict__ ids,
                                                            const uint8_t* __restrict__ mask,
@@ -661,9 +678,15 @@ __global__ void __launch_bounds__(256) lmhead_rows_kernel(long long N, int V, in
   // have been computed): it reports logp = 0 and still counts in the denominators
   const bool valid = in_batch && row_needs_forward(t, rowA, rowcu, rowcn, rowck, logp_ref != nullptr, flags);
   mrl::Lse2 acc = mrl::lse2_empty();
+  float usum = 0.f;  // sum_v 2^(x_v - acc.m) z_v, carried along when the entropy is asked for
   if (valid)
     for (int n = 0; n < n_tiles; ++n) {
       const float2 q = partial[(long long)n * part_ld + t];
+      if (entropy != nullptr) {
+        const float m = fmaxf(acc.m, q.x);
+        if (m != -INFINITY)
+          usum = usum * mrl::ex2_approx(acc.m - m) + partial_u[(long long)n * part_ld + t] * mrl::ex2_approx(q.x - m);
+      }
       acc = mrl::lse2_merge(acc, mrl::Lse2{q.x, q.y});
     }
   float g = 0.f, l2 = 0.f;
@@ -685,6 +708,7 @@ __global__ void __launch_bounds__(256) lmhead_rows_kernel(long long N, int V, in
     st = MRL_ROW_VALID | MRL_ROW_READ;
     if (ro.clipped && in.A != 0.f) st |= MRL_ROW_CLIPPED;
   }
+  if (entropy != nullptr) entropy[t] = valid ? l2 * MRL_LN2 - usum / acc.s : 0.f;  // H = lse - sum_v p_v z_v
   row_m2[t] = acc.m;
   row_s[t] = acc.s;
   row_zt[t] = valid ? zt[t] : 0.f;
@@ -828,6 +852,7 @@ struct LmheadWs {
   void* rows;            // per-row scratch of the loss (MrlLossWs)
   float *g, *lse2, *zt;
   float2* partial;
+  float* partial_u;      // the entropy's third partial
   __nv_bfloat16* D;      // one vocabulary chunk of dZ, [N, ldD]
   float* dH_acc;
   uint8_t* live;         // per block of 256 rows
@@ -848,6 +873,7 @@ LmheadWs carve_lmhead_ws(void* ws, long long N, int V, int H, int S) {
   w.n_tiles_fwd = (V + BN - 1) / BN;
   w.part_ld = pad_to(N, BM);
   w.partial = c.take<float2>((size_t)w.n_tiles_fwd * (size_t)w.part_ld);
+  w.partial_u = c.take<float>((size_t)w.n_tiles_fwd * (size_t)w.part_ld);
   w.vchunk = V < kVChunk ? (int)pad_to(V, BN) : kVChunk;
   w.n_chunks = (V + w.vchunk - 1) / w.vchunk;
   w.ldD = w.vchunk;
@@ -918,7 +944,6 @@ extern "C" int mrl_fused_lmhead_loss_fwd_bwd(const void* hidden, const void* W, 
   if (!(lp->eps_lo >= 0.f) || !(lp->eps_hi >= 0.f)) return MRL_ERR_INVALID_ARG;
   if (lp->ratio_level != MRL_RATIO_TOKEN && lp->ratio_level != MRL_RATIO_SEQUENCE) return MRL_ERR_INVALID_ARG;
   if (lp->ratio_level == MRL_RATIO_SEQUENCE && tok_weight != nullptr) return MRL_ERR_INVALID_ARG;
-  if (lp->entropy != nullptr) return MRL_ERR_INVALID_ARG;  // the entropy diagnostic is a logits-in output
   if (!mrl_kl_args_ok(lp)) return MRL_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool accum_loss = lp->flags & MRL_FLAG_ACCUMULATE_LOSS;
@@ -974,14 +999,17 @@ extern "C" int mrl_fused_lmhead_loss_fwd_bwd(const void* hidden, const void* W, 
     p.K = H;
     p.status = status;
     p.partial = w.partial;
+    p.partial_u = w.partial_u;
     p.part_ld = w.part_ld;
     p.ids = ids;
     p.zt = w.zt;
     p.col0 = 0;
-    rc = launch_gemm<EPI_LSE, false, false>(hid, H, Wm, H, p, pair, st, &w.fwd);
+    rc = lp->entropy != nullptr ? launch_gemm<EPI_LSE_ENT, false, false>(hid, H, Wm, H, p, pair, st, &w.fwd)
+                                : launch_gemm<EPI_LSE, false, false>(hid, H, Wm, H, p, pair, st, &w.fwd);
     if (rc != MRL_OK) return rc;
   }
-  lmhead_rows_kernel<<<(unsigned)((N + 255) / 256), 256, 0, st>>>(N, V, w.n_tiles_fwd, w.partial, w.part_ld, w.zt, ids,
+  lmhead_rows_kernel<<<(unsigned)((N + 255) / 256), 256, 0, st>>>(N, V, w.n_tiles_fwd, w.partial, w.partial_u, lp->entropy,
+                                                                  w.part_ld, w.zt, ids,
                                                                   mask, rw.rowA, rw.rowcu, rw.rowcn, rw.rowck,
                                                                   seq_ratio ? nullptr : lp->logp_ref, lp->kl_estimator,
                                                                   seq_ratio ? nullptr : logp_old, lp->eps_lo,

@@ -60,15 +60,23 @@ def test_entropy_matches_oracle(N, V, dtype, pad, mask_p, ratio_level):
     assert (logp.double() - ref_logp).abs().max() <= 1e-4      # the log-probs are unchanged by asking for the entropy
 
 
-def test_entropy_is_refused_on_the_hidden_in_path():
-    h = torch.zeros(4, 64, dtype=torch.bfloat16, device="cuda")
-    W = torch.zeros(8, 64, dtype=torch.bfloat16, device="cuda")
-    ent = torch.zeros(4, device="cuda")
-    lp = make_lp()
+@pytest.mark.parametrize("pair", [False, True])
+@pytest.mark.parametrize("N,H,V,S,mask_p", [
+    (300, 128, 1000, 5, None),       # ragged tiles, one chunk
+    (260, 192, 40000, 7, 0.8),       # many column tiles to merge, masked rows
+    (1, 64, 37, 1, None),
+])
+def test_entropy_on_the_hidden_in_path(N, H, V, S, mask_p, pair):
+    import test_lmhead_gpu as LM
+    hidden, W, ids, mask, cu, adv, old, g = LM.toy(N, H, V, S, seed=N + V, mask_p=mask_p)
+    lp = make_lp(flags=B.FLAG_PAIR_TILES if pair else 0)
+    ent = torch.full((N,), float("nan"), device="cuda")
     lp.entropy = ent.data_ptr()
-    with pytest.raises(B.MrlError):
-        B.mrl_fused_lmhead_loss_fwd_bwd(h, W, torch.zeros(4, dtype=torch.int32, device="cuda"), None,
-                                        torch.tensor([0, 4], dtype=torch.int32, device="cuda"),
-                                        torch.ones(1, device="cuda"), None, None, None, lp, None, None,
-                                        torch.zeros(4, device="cuda"), torch.zeros(2, device="cuda"), None, None,
-                                        torch.zeros(1 << 20, dtype=torch.uint8, device="cuda"))
+    got = LM.run_gpu_lmhead(hidden, W, ids, mask, cu, adv, old, None, None, lp)
+    z = hidden.double() @ W.double().T
+    ref = O.token_entropy(z, ids, mask)
+    assert torch.isfinite(ent).all()
+    assert (ent.cpu().double() - ref).abs().max() <= ENT_ATOL
+    lp0 = make_lp(flags=B.FLAG_PAIR_TILES if pair else 0)
+    plain = LM.run_gpu_lmhead(hidden, W, ids, mask, cu, adv, old, None, None, lp0)
+    assert torch.equal(plain["logp"], got["logp"]) and torch.equal(plain["dW"], got["dW"])   # nothing else changes
