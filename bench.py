@@ -54,7 +54,7 @@ def measured_peaks():
 # DRAM bytes per token (dram__bytes_read.sum + dram__bytes_write.sum over the rows of the capture) of the dominant
 # kernel as it stands, from the committed ncu summary profiles/row_stream_kernel_c2_logits_in.md; traffic grows in
 # proportion to the rows.  Set to None whenever that kernel changes, until the counters are taken again.
-ROW_STREAM_DRAM_BYTES_PER_TOKEN_V151936 = 642025
+ROW_STREAM_DRAM_BYTES_PER_TOKEN_V151936 = 642153
 
 
 class ClockSampler:
