@@ -317,3 +317,17 @@ def test_config5_full_size_unmasked_sampled_rows_and_invariants():
     assert torch.isfinite(dW).all()
     col, mag = dW.sum(dim=0), dW.abs().sum(dim=0)
     assert (col.abs() <= 2e-2 * mag + 1e-12).all()
+
+
+@pytest.mark.parametrize("pair", [False, True])
+def test_two_runs_give_the_same_bits(pair):
+    # every sum has a fixed order (tile partials merged in tile order, chunks accumulated in sequence, float64 loss sums
+    # in one block): the pass is reproducible bit for bit
+    N, H, V, S = 700, 256, 40000, 6
+    hidden, W, ids, mask, cu, adv, old, g = toy(N, H, V, S, seed=77, mask_p=0.9)
+    lp = make_lp(flags=B.FLAG_PAIR_TILES if pair else 0)
+    a = run_gpu_lmhead(hidden, W, ids, mask, cu, adv, old, None, None, lp)
+    b = run_gpu_lmhead(hidden, W, ids, mask, cu, adv, old, None, None, lp)
+    for k in ("logp", "loss", "stats", "dH", "dW"):
+        assert torch.equal(a[k].view(torch.int16) if a[k].dtype == torch.bfloat16 else a[k],
+                           b[k].view(torch.int16) if b[k].dtype == torch.bfloat16 else b[k]), k
