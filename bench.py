@@ -393,8 +393,9 @@ class LmheadWorkload:
         torch.cuda.synchronize()
         chunks = -(-self.V // 16384)
         self.dominant_per_step = 1 + 3 * chunks          # forward GEMM, then (dZ, dHidden, dW) per vocabulary chunk
-        # adv, seq_count, row_coef, forward GEMM, rows, row_terms, finalize, then 3 GEMMs per chunk
-        self.kernels_per_step = 7 + 3 * chunks
+        # adv, seq_count, row_coef, forward GEMM, rows, row_terms, finalize, two live-block list builds of two kernels
+        # each (forward, backward), then 3 GEMMs per chunk
+        self.kernels_per_step = 11 + 3 * chunks
         # Blocks of 256 rows without any gradient are left out of the three backward products, and of the forward one
         # too under MRL_FLAG_SKIP_ZERO_ROWS: count the rows of the blocks that are worked on (a block whose rows are
         # all clipped is not expected and not counted as skipped).
