@@ -123,3 +123,31 @@ def test_host_pipeline_rejects_bad_arguments(lib):
     assert call(cu_=(C.c_int32 * 2)(0, 5)) == 1  # cu[S] != N
     assert lib.mrl_host_pipeline_workspace_bytes(1000, 4096, B.BF16, 8, 128) >= 3 * 128 * 4096 * 2
     assert lib.mrl_host_pipeline_workspace_bytes(1000, 4096, 9, 8, 128) == 0
+
+
+def test_header_is_plain_c_and_links_from_c(tmp_path):
+    """include/mrl.h compiles as C99 with pedantic warnings as errors, and a C program linked against the library
+    can call the host-only entry points (no CUDA call is made)."""
+    import shutil
+    import subprocess
+    if shutil.which("gcc") is None:
+        pytest.skip("no C compiler")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    src = tmp_path / "abi.c"
+    src.write_text('#include <stdio.h>\n#include <string.h>\n#include "mrl.h"\n'
+                   "int main(void) {\n"
+                   "  mrl_loss_params lp; mrl_adv_params ap; memset(&lp, 0, sizeof lp); memset(&ap, 0, sizeof ap);\n"
+                   "  if (mrl_version() != MRL_VERSION) return 2;\n"
+                   '  if (strcmp(mrl_status_string(MRL_OK), "MRL_OK") != 0) return 3;\n'
+                   "  if (mrl_workspace_bytes(MRL_WS_POLICY_LOSS, 1000, 4096, 0, MRL_BF16, 8) == 0) return 4;\n"
+                   "  if (mrl_policy_loss_fwd_bwd(0, MRL_BF16, 4, 16, 16, 0, 0, 0, 1, 0, 0, 0, 0, 0, 0, 16, 0, 0, 0, 0, 0, 0, 0)\n"
+                   "      != MRL_ERR_INVALID_ARG) return 5;\n"
+                   '  printf("%d %u\\n", mrl_version(), (unsigned)sizeof(mrl_loss_params));\n  return 0;\n}\n')
+    exe = tmp_path / "abi"
+    lib_dir = os.path.join(root, "paper_2605_07244_b200")
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-I", os.path.join(root, "include"),
+                    str(src), "-o", str(exe), "-L", lib_dir, "-l:libmrl.so", "-Wl,-rpath," + lib_dir], check=True)
+    out = subprocess.run([str(exe)], capture_output=True, text=True)
+    assert out.returncode == 0, out
+    version, size = out.stdout.split()
+    assert int(version) == B.version() and int(size) == C.sizeof(B.LossParams)   # the binding mirrors the C struct
