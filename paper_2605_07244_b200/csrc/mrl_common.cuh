@@ -36,7 +36,8 @@ struct MrlLossWs {
   float *rowA, *rowcu, *rowcn;        // A_t, c_t u_t, cn_t
   float* rowck;                       // beta c_t of the KL term (0 when the term is off)
   float *row_m2, *row_s, *row_zt;     // base-2 running max, sum of 2^(x - max), target logit
-  double *pg_term, *nll_term, *kl_term;
+  double *pg_term, *nll_term, *kl_term;  // per-row terms (response-level ratio only)
+  double* partials;                      // [ceil(N / 256)][6] block sums of the terms and the row statistics
   uint8_t* rowstat;                   // MRL_ROW_* bits
   int32_t* seq_cnt;
   unsigned long long* totals;

@@ -758,6 +758,26 @@ __global__ void __launch_bounds__(128) row_coef_kernel(const int32_t* __restrict
   }
 }
 
+// Sum of six per-thread float64 values over a block of 256 threads in a fixed order (shuffle tree inside a warp, then
+// the warps in turn); the result is in thread 0.
+__device__ __forceinline__ void block_sum6(double (&v)[6], double (*red)[8]) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int k = 0; k < 6; ++k) {
+    for (int o = 16; o > 0; o >>= 1) v[k] += __shfl_xor_sync(0xffffffffu, v[k], o);
+    if (lane == 0) red[k][warp] = v[k];
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+#pragma unroll
+    for (int k = 0; k < 6; ++k) {
+      double t = 0.0;
+      for (int w = 0; w < 8; ++w) t += red[k][w];
+      v[k] = t;
+    }
+  }
+}
+
 // Ratio, clipped surrogate and NLL term of every row in float64, from the row kernel's reduction triple:
 // lse = (m2 + log2 s) ln 2, logp = z_target - lse, rho = exp(logp - logp_old)  (Sec. 3; Eq. (1); Eq. (2)).
 // The surrogate is continuous across the clip bound, so the float32 decision the gradient used and the
@@ -772,12 +792,11 @@ __global__ void __launch_bounds__(256) row_terms_kernel(long long N, const float
                                                          const float* __restrict__ rowck,
                                                          const float* __restrict__ logp_ref, int kl_est,
                                                          const float* __restrict__ logp_old, float eps_lo,
-                                                         float eps_hi, double* __restrict__ pg_term,
-                                                         double* __restrict__ nll_term, double* __restrict__ kl_term,
+                                                         float eps_hi, double* __restrict__ partials,
                                                          float* __restrict__ logp) {
+  __shared__ double red[6][8];
   const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (t >= N) return;
-  const uint8_t st = rowstat[t];
+  const uint8_t st = t < N ? rowstat[t] : 0;
   double pg = 0.0, nl = 0.0, kl = 0.0, lp = 0.0;
   if ((st & kStatValid) && (st & kStatRead)) {
     const double lse = ((double)row_m2[t] + log2((double)row_s[t])) * 0.693147180559945309417232121458;
@@ -791,56 +810,50 @@ __global__ void __launch_bounds__(256) row_terms_kernel(long long N, const float
     if (cn != 0.0) nl = -cn * lp;
     if (logp_ref != nullptr && rowck[t] != 0.f) kl = (double)rowck[t] * mrl::kl_value(lp - (double)logp_ref[t], kl_est);
   }
-  pg_term[t] = pg;
-  nll_term[t] = nl;
-  kl_term[t] = kl;
-  if (logp != nullptr) logp[t] = (float)lp;
+  if (t < N && logp != nullptr) logp[t] = (float)lp;
+  double v[6] = {pg, nl, (st & kStatValid) ? 1.0 : 0.0, (st & kStatClipped) ? 1.0 : 0.0, (st & kStatRead) ? 1.0 : 0.0, kl};
+  block_sum6(v, red);
+  if (threadIdx.x == 0)
+    for (int k = 0; k < 6; ++k) partials[(long long)blockIdx.x * 6 + k] = v[k];
 }
 
-// fixed-order float64 sums of the per-row terms and the row statistics
-__global__ void __launch_bounds__(1024) finalize_kernel(const double* __restrict__ pg_term,
-                                                         const double* __restrict__ nll_term,
-                                                         const double* __restrict__ kl_term,
-                                                         const uint8_t* __restrict__ rowstat, long long N,
-                                                         const unsigned long long* __restrict__ totals,
-                                                         uint32_t flags, float* loss, float* kl_loss,
-                                                         long long* stats) {
-  __shared__ double red[6][32];
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+// The same block partials from per-row term arrays (the response-level ratio writes those).
+__global__ void __launch_bounds__(256) rows_partial_kernel(long long N, const double* __restrict__ pg_term,
+                                                            const double* __restrict__ nll_term,
+                                                            const double* __restrict__ kl_term,
+                                                            const uint8_t* __restrict__ rowstat,
+                                                            double* __restrict__ partials) {
+  __shared__ double red[6][8];
+  const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const uint8_t st = t < N ? rowstat[t] : 0;
+  double v[6] = {t < N ? pg_term[t] : 0.0, t < N ? nll_term[t] : 0.0, (st & kStatValid) ? 1.0 : 0.0,
+                 (st & kStatClipped) ? 1.0 : 0.0, (st & kStatRead) ? 1.0 : 0.0, t < N ? kl_term[t] : 0.0};
+  block_sum6(v, red);
+  if (threadIdx.x == 0)
+    for (int k = 0; k < 6; ++k) partials[(long long)blockIdx.x * 6 + k] = v[k];
+}
+
+// fixed-order float64 sums of the blocks' partial sums (terms and row statistics) into loss / stats
+__global__ void __launch_bounds__(256) finalize_kernel(const double* __restrict__ partials, long long n_blocks,
+                                                        const unsigned long long* __restrict__ totals, uint32_t flags,
+                                                        float* loss, float* kl_loss, long long* stats) {
+  __shared__ double red[6][8];
   double v[6] = {0, 0, 0, 0, 0, 0};
-  for (long long t = tid; t < N; t += 1024) {
-    v[0] += pg_term[t];
-    v[1] += nll_term[t];
-    const uint8_t st = rowstat[t];
-    v[2] += (st & kStatValid) ? 1.0 : 0.0;
-    v[3] += (st & kStatClipped) ? 1.0 : 0.0;
-    v[4] += (st & kStatRead) ? 1.0 : 0.0;
-    v[5] += kl_term[t];
-  }
+  for (long long b = threadIdx.x; b < n_blocks; b += 256) {
 #pragma unroll
-  for (int k = 0; k < 6; ++k) {
-    for (int o = 16; o > 0; o >>= 1) v[k] += __shfl_xor_sync(0xffffffffu, v[k], o);
-    if (lane == 0) red[k][warp] = v[k];
+    for (int k = 0; k < 6; ++k) v[k] += partials[b * 6 + k];
   }
-  __syncthreads();
-  if (warp == 0) {
-#pragma unroll
-    for (int k = 0; k < 6; ++k) {
-      double t = red[k][lane];
-      for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
-      v[k] = t;
-    }
-    if (lane == 0) {
-      const bool accum = flags & MRL_FLAG_ACCUMULATE_LOSS;
-      loss[0] = (accum ? loss[0] : 0.f) + (float)v[0];
-      loss[1] = (accum ? loss[1] : 0.f) + (float)v[1];
-      if (kl_loss != nullptr) kl_loss[0] = (accum ? kl_loss[0] : 0.f) + (float)v[5];
-      if (stats != nullptr) {
-        stats[0] = (accum ? stats[0] : 0) + (long long)v[2];
-        stats[1] = (accum ? stats[1] : 0) + (long long)v[3];
-        stats[2] = (accum ? stats[2] : 0) + (long long)v[4];
-        stats[3] = (accum ? stats[3] : 0) + (long long)totals[1];
-      }
+  block_sum6(v, red);
+  if (threadIdx.x == 0) {
+    const bool accum = flags & MRL_FLAG_ACCUMULATE_LOSS;
+    loss[0] = (accum ? loss[0] : 0.f) + (float)v[0];
+    loss[1] = (accum ? loss[1] : 0.f) + (float)v[1];
+    if (kl_loss != nullptr) kl_loss[0] = (accum ? kl_loss[0] : 0.f) + (float)v[5];
+    if (stats != nullptr) {
+      stats[0] = (accum ? stats[0] : 0) + (long long)v[2];
+      stats[1] = (accum ? stats[1] : 0) + (long long)v[3];
+      stats[2] = (accum ? stats[2] : 0) + (long long)v[4];
+      stats[3] = (accum ? stats[3] : 0) + (long long)totals[1];
     }
   }
 }
@@ -859,6 +872,7 @@ MrlLossWs carve_loss_ws(void* ws, long long N, int S) {
   w.pg_term = c.take<double>((size_t)N);
   w.nll_term = c.take<double>((size_t)N);
   w.kl_term = c.take<double>((size_t)N);
+  w.partials = c.take<double>((size_t)((N + 255) / 256) * 6);
   w.rowstat = c.take<uint8_t>((size_t)N);
   w.seq_cnt = c.take<int32_t>((size_t)S + 1);
   w.bytes = c.off;
@@ -962,11 +976,10 @@ int mrl_rows_finish(const MrlLossWs& w, long long N, const float* logp_old, cons
   row_terms_kernel<<<(unsigned)((N + 255) / 256), 256, 0, st>>>(N, w.row_m2, w.row_s, w.row_zt, w.rowstat, w.rowA,
                                                                 w.rowcu, w.rowcn, w.rowck, lp->logp_ref,
                                                                 lp->kl_estimator, logp_old, lp->eps_lo, lp->eps_hi,
-                                                                w.pg_term, w.nll_term, w.kl_term, logp);
+                                                                w.partials, logp);
   MRL_CUDA_OK(cudaGetLastError());
-  finalize_kernel<<<1, 1024, 0, st>>>(w.pg_term, w.nll_term, w.kl_term, w.rowstat, N, w.totals, lp->flags, loss,
-                                      lp->logp_ref != nullptr ? lp->kl_loss : nullptr,
-                                      reinterpret_cast<long long*>(stats));
+  finalize_kernel<<<1, 256, 0, st>>>(w.partials, (N + 255) / 256, w.totals, lp->flags, loss,
+                                     lp->logp_ref != nullptr ? lp->kl_loss : nullptr, reinterpret_cast<long long*>(stats));
   MRL_CUDA_OK(cudaGetLastError());
   return MRL_OK;
 }
@@ -984,9 +997,11 @@ int mrl_rows_finish_sequence(const MrlLossWs& w, long long N, int S, const int32
                                       logp_old, nll_weight, w.rowck, *lp, w.pg_term, w.nll_term, w.kl_term, logp, g_out,
                                       lse2_out);
   MRL_CUDA_OK(cudaGetLastError());
-  finalize_kernel<<<1, 1024, 0, st>>>(w.pg_term, w.nll_term, w.kl_term, w.rowstat, N, w.totals, lp->flags, loss,
-                                      lp->logp_ref != nullptr ? lp->kl_loss : nullptr,
-                                      reinterpret_cast<long long*>(stats));
+  rows_partial_kernel<<<(unsigned)((N + 255) / 256), 256, 0, st>>>(N, w.pg_term, w.nll_term, w.kl_term, w.rowstat,
+                                                                   w.partials);
+  MRL_CUDA_OK(cudaGetLastError());
+  finalize_kernel<<<1, 256, 0, st>>>(w.partials, (N + 255) / 256, w.totals, lp->flags, loss,
+                                     lp->logp_ref != nullptr ? lp->kl_loss : nullptr, reinterpret_cast<long long*>(stats));
   MRL_CUDA_OK(cudaGetLastError());
   return MRL_OK;
 }
