@@ -453,3 +453,43 @@ def test_config2_full_size_sampled_rows():
     want_loss = -float((adv.double() * lens).sum() / N)
     assert abs(float(loss.cpu()[0]) - want_loss) <= 1e-5 * abs(want_loss)
     assert abs(want_loss) > 1e-4     # the property is not vacuous for this seed
+
+
+@pytest.mark.parametrize("V,dtype", [(1000, torch.float32), (4096, torch.bfloat16), (40008, torch.bfloat16),
+                                     (262144 + 16, torch.bfloat16)])
+def test_extreme_logits(V, dtype):
+    """Vocabulary masking with -inf, a logit that dominates the row, large magnitudes, an exactly uniform row: the
+    running maximum / rescaled sum must neither overflow nor produce NaN, and must match the oracle."""
+    N, S = 12, 3
+    g = torch.Generator().manual_seed(V)
+    z = (torch.randn(N, V, generator=g) * 2.0)
+    ids = torch.randint(V // 2, V, (N,), generator=g, dtype=torch.int32)
+    z[0, :V // 2] = float("-inf")                       # half of the vocabulary masked out (targets are in the other half)
+    z[1, torch.randperm(V, generator=g)[:V - 40]] = float("-inf")
+    z[1, ids[1]] = 0.5                                  # ... all but 40 columns masked, the target kept
+    # (float32: magnitudes stay moderate -- float32 holds a log-sum-exp near 300 to 2e-5 only, which is already
+    # above the 1e-5 asked of float32 gradients; the bf16 cases, judged at 1e-2, take the large ones)
+    big = dtype == torch.bfloat16
+    z[2, 7] = 80.0 if big else 40.0                     # one column carries all the mass: logp of the target ~ -80
+    z[3, ids[3]] = 60.0 if big else 40.0                # the target carries all the mass: logp ~ 0, dz ~ 0
+    z[4] = 0.0                                          # uniform: logp = -log V
+    z[5] = z[5] * (30.0 if big else 6.0)                # large magnitudes
+    z[6] = -200.0 if big else -30.0                     # uniform far from zero
+    z[7, :] = float("-inf")
+    z[7, ids[7]] = -3.0                                 # only the target survives: logp = 0
+    z = z.to(dtype)
+    cu = torch.tensor([0, 4, 8, 12], dtype=torch.int32)
+    adv = torch.tensor([0.9, -1.2, 0.6])
+    logp, _, _ = O.token_logprobs(z, ids)
+    assert torch.isfinite(logp).all()
+    old = (logp + 0.05 * torch.randn(N, generator=g, dtype=torch.float64)).float()
+    nllw = torch.zeros(N)
+    nllw[8:] = 1.0
+    lp = make_lp(nll_coeff=0.1)
+    got = run_gpu_policy_loss(z, ids, None, cu, adv, old, None, nllw, lp)
+    ref = O.policy_loss(z, ids, None, cu, adv, old, None, nllw, oracle_lp(lp))
+    assert got["status"] == 0 and torch.isfinite(got["dlogits"].float()).all() and torch.isfinite(got["loss"]).all()
+    assert abs(float(got["logp"][4]) + math.log(V)) <= 1e-5 and abs(float(got["logp"][7])) <= 1e-6
+    compare_policy_loss(got, ref, V, dtype, loss_floor=0.1 * float(ref["pg_term"].abs().sum()))
+    # masked-out columns get exactly zero gradient
+    assert got["dlogits"][0, :V // 2].abs().max() == 0
