@@ -823,9 +823,10 @@ int launch_gemm(const void* A, long long lda, const void* B, long long ldb, Gemm
     p.k_list = k_rows->k64;
     p.k_count = k_rows->counts + 2;
   }
-  // rows of A per raster group: a wave's operands should share L2; with a short K a taller group re-uses A
-  // across the next waves as well (measured: 4,096 rows at K = 4,096, 2,048 rows at K >= 16,384)
-  p.group_m = (kC == 2 && p.K <= 8192 ? 4096 : 2048) / (BM * kC);
+  // rows of A per raster group: the group's rows of A stay in L2 while B streams past them, so B is fetched from
+  // DRAM once per group -- the taller the group the better, as long as its A panel (rows x K) fits L2 beside the
+  // stream (measured: 4,096 rows at K = 4,096, 2,048 rows at K >= 16,384; DRAM traffic costs clock under the power cap)
+  p.group_m = (p.K <= 8192 ? 4096 : 2048) / (BM * kC);
   const long long tiles = (long long)p.m_tiles * p.n_tiles;
   if (tiles > 0x7fffffffll) return MRL_ERR_UNSUPPORTED_SHAPE;
   if (kC == 2) {
