@@ -72,3 +72,51 @@ def test_advantages_and_loss_pass_replay_from_a_cuda_graph(V, dtype):
     got = dict(logp=logp.cpu(), loss=loss.cpu(), stats=stats.cpu(), status=int(status.cpu()), dlogits=dz.cpu())
     assert got["status"] == 0
     compare_policy_loss(got, ref, V, dtype, loss_floor=0.1 * float(ref["pg_term"].abs().sum()))
+
+
+def test_fused_lm_head_replays_from_a_cuda_graph():
+    """The hidden-in pass too: tensor maps are built on the host at capture time from the same pointers, the live-block
+    counts are read on the device, so a replay on new values gives what a direct call gives, bit for bit."""
+    import test_lmhead_gpu as LM
+    N, H, V, S = 700, 128, 20000, 6
+    hidden, W, ids, mask, cu, adv, old, g = LM.toy(N, H, V, S, seed=5, mask_p=0.9)
+    d = dict(h=dev(hidden), W=dev(W), ids=dev(ids), mask=dev(mask), cu=dev(cu), adv=dev(adv), old=dev(old))
+    dH = torch.empty(N, H, dtype=torch.bfloat16, device="cuda")
+    dW = torch.empty(V, H, dtype=torch.bfloat16, device="cuda")
+    logp = torch.empty(N, device="cuda")
+    loss = torch.zeros(2, device="cuda")
+    stats = torch.zeros(4, dtype=torch.int64, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ws = torch.empty(B.workspace_bytes(B.WS_FUSED_LMHEAD, N, V, H, B.BF16, S), dtype=torch.uint8, device="cuda")
+    lp = make_lp()
+
+    def step(stream):
+        B.mrl_fused_lmhead_loss_fwd_bwd(d["h"], d["W"], d["ids"], d["mask"], d["cu"], d["adv"], d["old"], None, None, lp,
+                                        dH, dW, logp, loss, stats, status, ws, stream=stream)
+
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        step(side)
+    side.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        step(side)
+    # new values (another batch with a block of zero-advantage sequences), same buffers
+    hidden2, W2, ids2, mask2, _, adv2, old2, _ = LM.toy(N, H, V, S, seed=6, mask_p=0.8)
+    adv2 = adv2.clone()
+    adv2[:2] = 0.0
+    for k, t in (("h", hidden2), ("W", W2), ("ids", ids2), ("mask", mask2), ("adv", adv2), ("old", old2)):
+        d[k].copy_(t)
+    dH.fill_(float("nan"))
+    dW.fill_(float("nan"))
+    graph.replay()
+    torch.cuda.synchronize()
+    replayed = dict(logp=logp.cpu(), loss=loss.cpu(), stats=stats.cpu(), dH=dH.cpu(), dW=dW.cpu(), status=int(status.cpu()))
+    direct = LM.run_gpu_lmhead(hidden2, W2, ids2, mask2, cu, adv2, old2, None, None, make_lp())
+    assert replayed["status"] == 0
+    for k in ("logp", "loss", "stats"):
+        assert torch.equal(replayed[k], direct[k]), k
+    for k in ("dH", "dW"):
+        assert torch.equal(replayed[k].view(torch.int16), direct[k].view(torch.int16)), k
+    ref = O.fused_lmhead_loss(hidden2, W2, ids2, mask2, cu, adv2, old2, None, None, oracle_lp(lp))
+    LM.compare(replayed, ref)
