@@ -1,12 +1,15 @@
 // Logits-in path: mrl_token_logprobs and mrl_policy_loss_fwd_bwd.
 //
-// Streaming kernel (bf16, 16- or 32-byte aligned rows): one CTA per logits row, two CTAs per SM.  Pass 1
+// Streaming kernel (bf16 or float32, 16- or 32-byte aligned rows of at least 4,096 columns): one CTA per logits row,
+// two CTAs per SM.  Pass 1
 // streams the row from HBM with wide loads while keeping a running (max, sum of exponentials) per thread;
 // after the block reduction and the ratio / clip / loss scalars, pass 2 re-reads the row -- from L2, which
 // holds every row in flight several times over -- and writes g * (softmax - onehot) with streaming stores.
 // The row crosses the HBM interface once in each direction; nothing is shared between CTAs.
 // General kernel (any dtype, any V, any alignment): one CTA per row, three passes over global
-// memory; used for small or unaligned problems.
+// memory; used for short or unaligned rows.
+#include <type_traits>
+
 #include "mrl_common.cuh"
 
 namespace {
@@ -110,6 +113,20 @@ __device__ __forceinline__ void write_row_scalars(const RowParams& p, long long 
   }
 }
 
+// scalar element access in either logits type
+template <typename T>
+__device__ __forceinline__ float ld_as_f32(const T* p);
+template <>
+__device__ __forceinline__ float ld_as_f32<float>(const float* p) { return *p; }
+template <>
+__device__ __forceinline__ float ld_as_f32<__nv_bfloat16>(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+template <typename T>
+__device__ __forceinline__ void st_from_f32(T* p, float v);
+template <>
+__device__ __forceinline__ void st_from_f32<float>(float* p, float v) { *p = v; }
+template <>
+__device__ __forceinline__ void st_from_f32<__nv_bfloat16>(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
+
 // packed maximum of two bf16 pairs
 __device__ __forceinline__ uint32_t hmax2_u32(uint32_t a, uint32_t b) {
   uint32_t r;
@@ -118,7 +135,7 @@ __device__ __forceinline__ uint32_t hmax2_u32(uint32_t a, uint32_t b) {
 }
 
 // ------------------------------------------------------------------------------------------------
-// Streaming kernel: bf16, one CTA per row; shared memory holds only the few vectors parked between the passes.
+// Streaming kernel: one CTA per row; shared memory holds only the few vectors parked between the passes.
 // Pass 1 streams the row from HBM with 128- or 256-bit loads (running maximum and rescaled sum per thread);
 // pass 2 needs the same vectors again: the last group read is still in registers, the first 48 KB read were
 // parked in shared memory, the rest comes from L2 -- the rows in flight (two per SM) are a fraction of its
@@ -222,10 +239,13 @@ __device__ __forceinline__ StreamVec<kWords> stream_fill(uint32_t x) {
 
 // kC = 1: the CTA takes the whole row.  kC = 2: a cluster of two CTAs takes the row, half each, and the halves'
 // (max, sum, target logit) cross through distributed shared memory: a remote store plus a remote mbarrier arrive.
-template <int kT, int kU, int kWords, int kC, bool kEnt>
+// kF32: float32 logits (one element per 32-bit word) instead of bf16 (two).
+template <int kT, int kU, int kWords, int kC, bool kEnt, bool kF32>
 __global__ void __launch_bounds__(kT, 1024 / kT) row_stream_kernel(const RowParams p) {
   constexpr int kWarpsT = kT / 32;
-  constexpr int kVecBytes = kWords * 4, kVecElems = kWords * 2;
+  constexpr int kVecBytes = kWords * 4, kVecElems = kF32 ? kWords : kWords * 2;
+  constexpr uint32_t kNegInf = kF32 ? 0xff800000u : 0xff80ff80u;  // -inf, or a pair of them
+  using Elem = typename std::conditional<kF32, float, __nv_bfloat16>::type;
   using Vec = StreamVec<kWords>;
   __shared__ float red[3 * 32];
   __shared__ float fin[4];
@@ -242,8 +262,8 @@ __global__ void __launch_bounds__(kT, 1024 / kT) row_stream_kernel(const RowPara
   const int part_off = rank * part_nvec * kVecElems;               // first element of this CTA's part
   const int nvec = max(0, min(row_nvec - rank * part_nvec, part_nvec));
   const bool want_grad = p.dlogits != nullptr;
-  const __nv_bfloat16* grow = static_cast<const __nv_bfloat16*>(p.logits) + row * p.ld + part_off;
-  __nv_bfloat16* orow = want_grad ? static_cast<__nv_bfloat16*>(p.dlogits) + row * p.ld_out + part_off : nullptr;
+  const Elem* grow = static_cast<const Elem*>(p.logits) + row * p.ld + part_off;
+  Elem* orow = want_grad ? static_cast<Elem*>(p.dlogits) + row * p.ld_out + part_off : nullptr;
   const char* in = reinterpret_cast<const char*>(grow) + (size_t)tid * kVecBytes;
   char* out = reinterpret_cast<char*>(orow) + (size_t)tid * kVecBytes;
 
@@ -269,7 +289,7 @@ __global__ void __launch_bounds__(kT, 1024 / kT) row_stream_kernel(const RowPara
   const int rel = ctx.id - part_off;                               // target column relative to this part
   const bool owner = ctx.valid && rel >= 0 && rel < nvec * kVecElems;
   float zt = 0.f;
-  if (tid == 0 && owner) zt = __bfloat162float(grow[rel]);         // before anything is written in place
+  if (tid == 0 && owner) zt = ld_as_f32<Elem>(grow + rel);         // before anything is written in place
 
   // ---- pass 1: running (max, sum) in the base-2 domain
   // The row is walked from its last group of kT * kU vectors (the ragged one) down to its first, so that the group
@@ -285,7 +305,7 @@ __global__ void __launch_bounds__(kT, 1024 / kT) row_stream_kernel(const RowPara
 #pragma unroll
       for (int u = 0; u < kU; ++u)
         v[u] = (base + u * kT + tid < nvec) ? stream_ld<kWords, kHintKeep>(in + (size_t)(base + u * kT) * kVecBytes)
-                                            : stream_fill<kWords>(0xff80ff80u);  // (-inf, -inf)
+                                            : stream_fill<kWords>(kNegInf);
     }
     // the first vectors read are the ones L2 is likeliest to have dropped by pass 2: park them
     const int q0 = ((last_base - base) / (kT * kU)) * kU;
@@ -295,13 +315,23 @@ __global__ void __launch_bounds__(kT, 1024 / kT) row_stream_kernel(const RowPara
         if (q0 + u < keep_q && base + u * kT + tid < nvec)
           park_st<kWords>(park_base, park_plane, (uint32_t)((q0 + u) * kT + tid), v[u]);
     }
-    uint32_t mx = 0xff80ff80u;
+    float vmax;
+    if constexpr (kF32) {
+      vmax = -INFINITY;
 #pragma unroll
-    for (int u = 0; u < kU; ++u) {
+      for (int u = 0; u < kU; ++u) {
 #pragma unroll
-      for (int j = 0; j < kWords; ++j) mx = hmax2_u32(mx, v[u].w[j]);
+        for (int j = 0; j < kWords; ++j) vmax = fmaxf(vmax, __uint_as_float(v[u].w[j]));
+      }
+    } else {
+      uint32_t mx = kNegInf;
+#pragma unroll
+      for (int u = 0; u < kU; ++u) {
+#pragma unroll
+        for (int j = 0; j < kWords; ++j) mx = hmax2_u32(mx, v[u].w[j]);
+      }
+      vmax = fmaxf(mrl::bf16lo_to_f32(mx), mrl::bf16hi_to_f32(mx));
     }
-    const float vmax = fmaxf(mrl::bf16lo_to_f32(mx), mrl::bf16hi_to_f32(mx));
     const float m_new = fmaxf(m_run, vmax * MRL_LOG2E);
     if (m_new > m_run) {  // also the first group (m_run = -inf, s_run = 0)
       const float f = mrl::ex2_approx(m_run - m_new);
@@ -316,13 +346,22 @@ __global__ void __launch_bounds__(kT, 1024 / kT) row_stream_kernel(const RowPara
       for (int u = 0; u < kU; ++u) {
 #pragma unroll
         for (int j = 0; j < kWords; ++j) {
-          const float zlo = mrl::bf16lo_to_f32(v[u].w[j]), zhi = mrl::bf16hi_to_f32(v[u].w[j]);
-          const float a = mrl::ex2_approx(fmaf(zlo, MRL_LOG2E, neg_m)), b = mrl::ex2_approx(fmaf(zhi, MRL_LOG2E, neg_m));
-          s0 += a;
-          s1 += b;
-          if (kEnt) {  // a = 0 exactly where z = -inf: keep 0 * inf out of the sum
-            u0 = a != 0.f ? fmaf(a, zlo, u0) : u0;
-            u1 = b != 0.f ? fmaf(b, zhi, u1) : u1;
+          if constexpr (kF32) {
+            const float z = __uint_as_float(v[u].w[j]);
+            const float a = mrl::ex2_approx(fmaf(z, MRL_LOG2E, neg_m));
+            if (j & 1) s1 += a; else s0 += a;
+            if (kEnt) {  // a = 0 exactly where z = -inf: keep 0 * inf out of the sum
+              if (j & 1) u1 = a != 0.f ? fmaf(a, z, u1) : u1; else u0 = a != 0.f ? fmaf(a, z, u0) : u0;
+            }
+          } else {
+            const float zlo = mrl::bf16lo_to_f32(v[u].w[j]), zhi = mrl::bf16hi_to_f32(v[u].w[j]);
+            const float a = mrl::ex2_approx(fmaf(zlo, MRL_LOG2E, neg_m)), b = mrl::ex2_approx(fmaf(zhi, MRL_LOG2E, neg_m));
+            s0 += a;
+            s1 += b;
+            if (kEnt) {
+              u0 = a != 0.f ? fmaf(a, zlo, u0) : u0;
+              u1 = b != 0.f ? fmaf(b, zhi, u1) : u1;
+            }
           }
         }
       }
@@ -420,7 +459,7 @@ __global__ void __launch_bounds__(kT, 1024 / kT) row_stream_kernel(const RowPara
     return;
   }
   const float neg_k = -(lse2 - log2f(fabsf(g)));  // 2^(z log2e - k) = |g| softmax(z)
-  const uint32_t sign = g < 0.f ? 0x80008000u : 0u;
+  const uint32_t sign = g < 0.f ? (kF32 ? 0x80000000u : 0x80008000u) : 0u;
   // (the first group is still in registers; the others in the order pass 1 read them last-to-first, so the most
   // recently loaded lines, the likeliest to be still in L2, come first; the oldest come back from shared memory)
   for (int base = 0; base <= last_base; base += kT * kU) {
@@ -438,32 +477,24 @@ __global__ void __launch_bounds__(kT, 1024 / kT) row_stream_kernel(const RowPara
       Vec r;
 #pragma unroll
       for (int j = 0; j < kWords; ++j) {
-        const float a = mrl::ex2_approx(fmaf(mrl::bf16lo_to_f32(v[u].w[j]), MRL_LOG2E, neg_k));
-        const float b = mrl::ex2_approx(fmaf(mrl::bf16hi_to_f32(v[u].w[j]), MRL_LOG2E, neg_k));
-        r.w[j] = mrl::pack_bf16x2(a, b) ^ sign;
+        if constexpr (kF32) {
+          r.w[j] = __float_as_uint(mrl::ex2_approx(fmaf(__uint_as_float(v[u].w[j]), MRL_LOG2E, neg_k))) ^ sign;
+        } else {
+          const float a = mrl::ex2_approx(fmaf(mrl::bf16lo_to_f32(v[u].w[j]), MRL_LOG2E, neg_k));
+          const float b = mrl::ex2_approx(fmaf(mrl::bf16hi_to_f32(v[u].w[j]), MRL_LOG2E, neg_k));
+          r.w[j] = mrl::pack_bf16x2(a, b) ^ sign;
+        }
       }
       if (full || base + u * kT + tid < nvec) stream_st<kWords>(out + (size_t)(base + u * kT) * kVecBytes, r);
     }
   }
   // the thread whose vector store covered the target column patches it (program order on one address)
-  if (owner && tid == (rel / kVecElems) % kT) orow[rel] = __float2bfloat16_rn(tfix);
+  if (owner && tid == (rel / kVecElems) % kT) st_from_f32<Elem>(orow + rel, tfix);
 }
 
 // ------------------------------------------------------------------------------------------------
 // General kernel: one CTA per row, any dtype / V / alignment.
 // ------------------------------------------------------------------------------------------------
-template <typename T>
-__device__ __forceinline__ float ld_as_f32(const T* p);
-template <>
-__device__ __forceinline__ float ld_as_f32<float>(const float* p) { return *p; }
-template <>
-__device__ __forceinline__ float ld_as_f32<__nv_bfloat16>(const __nv_bfloat16* p) { return __bfloat162float(*p); }
-template <typename T>
-__device__ __forceinline__ void st_from_f32(T* p, float v);
-template <>
-__device__ __forceinline__ void st_from_f32<float>(float* p, float v) { *p = v; }
-template <>
-__device__ __forceinline__ void st_from_f32<__nv_bfloat16>(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
 
 template <typename T>
 __global__ void __launch_bounds__(kThreads) row_general_kernel(const RowParams p) {
@@ -540,18 +571,19 @@ __global__ void __launch_bounds__(kThreads) row_general_kernel(const RowParams p
 // Backward-only row kernels (response-level ratio): g_t is known only once the whole response has been scored, so
 // the gradient is a launch of its own that reads the row again.
 // ------------------------------------------------------------------------------------------------
-template <int kT, int kU, int kWords>
+template <int kT, int kU, int kWords, bool kF32>
 __global__ void __launch_bounds__(kT, 1024 / kT) row_backward_stream_kernel(const RowParams p, const float* __restrict__ row_g,
                                                                             const float* __restrict__ row_lse2,
                                                                             const float* __restrict__ row_zt) {
-  constexpr int kVecBytes = kWords * 4, kVecElems = kWords * 2;
+  constexpr int kVecBytes = kWords * 4, kVecElems = kF32 ? kWords : kWords * 2;
+  using Elem = typename std::conditional<kF32, float, __nv_bfloat16>::type;
   using Vec = StreamVec<kWords>;
   const int tid = threadIdx.x;
   const long long row = blockIdx.x;
   const int nvec = p.V / kVecElems;
-  const char* in = reinterpret_cast<const char*>(static_cast<const __nv_bfloat16*>(p.logits) + row * p.ld) +
+  const char* in = reinterpret_cast<const char*>(static_cast<const Elem*>(p.logits) + row * p.ld) +
                    (size_t)tid * kVecBytes;
-  __nv_bfloat16* orow = static_cast<__nv_bfloat16*>(p.dlogits) + row * p.ld_out;
+  Elem* orow = static_cast<Elem*>(p.dlogits) + row * p.ld_out;
   char* out = reinterpret_cast<char*>(orow) + (size_t)tid * kVecBytes;
   const float g = row_g[row];
   if (g == 0.f) {
@@ -560,7 +592,7 @@ __global__ void __launch_bounds__(kT, 1024 / kT) row_backward_stream_kernel(cons
   }
   const float lse2 = row_lse2[row];
   const float neg_k = -(lse2 - log2f(fabsf(g)));  // 2^(z log2e - k) = |g| softmax(z)
-  const uint32_t sign = g < 0.f ? 0x80008000u : 0u;
+  const uint32_t sign = g < 0.f ? (kF32 ? 0x80000000u : 0x80008000u) : 0u;
   for (int base = 0; base < nvec; base += kT * kU) {
     const bool full = base + kT * kU <= nvec;
     Vec v[kU];
@@ -573,16 +605,20 @@ __global__ void __launch_bounds__(kT, 1024 / kT) row_backward_stream_kernel(cons
       Vec r;
 #pragma unroll
       for (int j = 0; j < kWords; ++j) {
-        const float a = mrl::ex2_approx(fmaf(mrl::bf16lo_to_f32(v[u].w[j]), MRL_LOG2E, neg_k));
-        const float b = mrl::ex2_approx(fmaf(mrl::bf16hi_to_f32(v[u].w[j]), MRL_LOG2E, neg_k));
-        r.w[j] = mrl::pack_bf16x2(a, b) ^ sign;
+        if constexpr (kF32) {
+          r.w[j] = __float_as_uint(mrl::ex2_approx(fmaf(__uint_as_float(v[u].w[j]), MRL_LOG2E, neg_k))) ^ sign;
+        } else {
+          const float a = mrl::ex2_approx(fmaf(mrl::bf16lo_to_f32(v[u].w[j]), MRL_LOG2E, neg_k));
+          const float b = mrl::ex2_approx(fmaf(mrl::bf16hi_to_f32(v[u].w[j]), MRL_LOG2E, neg_k));
+          r.w[j] = mrl::pack_bf16x2(a, b) ^ sign;
+        }
       }
       if (full || base + u * kT + tid < nvec) stream_st<kWords>(out + (size_t)(base + u * kT) * kVecBytes, r);
     }
   }
   const int id = p.ids[row];  // g != 0 only on valid rows: the id is in range
   if (tid == (id / kVecElems) % kT)
-    orow[id] = __float2bfloat16_rn(g * (mrl::ex2_approx(fmaf(row_zt[row], MRL_LOG2E, -lse2)) - 1.0f));
+    st_from_f32<Elem>(orow + id, g * (mrl::ex2_approx(fmaf(row_zt[row], MRL_LOG2E, -lse2)) - 1.0f));
 }
 
 template <typename T>
@@ -881,12 +917,12 @@ MrlLossWs carve_loss_ws(void* ws, long long N, int S) {
 
 // Which kernel takes the rows: 0 = general, 4 = streaming with 128-bit accesses, 8 = with 256-bit accesses.
 int pick_stream_words(const RowParams& p, int dtype) {
-  if (dtype != MRL_BF16) return 0;
   if (p.V < 4096) return 0;  // short rows: the general kernel's three passes stay in cache
   const uintptr_t in = reinterpret_cast<uintptr_t>(p.logits), out = reinterpret_cast<uintptr_t>(p.dlogits);
   const bool grad = p.dlogits != nullptr;
-  if (p.V % 16 == 0 && p.ld % 16 == 0 && (in & 31) == 0 && (!grad || (p.ld_out % 16 == 0 && (out & 31) == 0))) return 8;
-  if (p.V % 8 == 0 && p.ld % 8 == 0 && (in & 15) == 0 && (!grad || (p.ld_out % 8 == 0 && (out & 15) == 0))) return 4;
+  const int e32 = dtype == MRL_BF16 ? 16 : 8, e16 = e32 / 2;  // elements per 32- and 16-byte vector
+  if (p.V % e32 == 0 && p.ld % e32 == 0 && (in & 31) == 0 && (!grad || (p.ld_out % e32 == 0 && (out & 31) == 0))) return 8;
+  if (p.V % e16 == 0 && p.ld % e16 == 0 && (in & 15) == 0 && (!grad || (p.ld_out % e16 == 0 && (out & 15) == 0))) return 4;
   return 0;
 }
 
@@ -908,7 +944,8 @@ int launch_rows(RowParams p, int dtype, cudaStream_t st) {
   // before the second pass reads them back -- the two halves of one row as a cluster of two.  (At 300 KB rows the
   // split reads HBM 1.01x instead of 1.34x but is 4 % slower: its per-CTA fixed work is spread over half the bytes.)
   // (the entropy diagnostic is carried by the whole-row variant only)
-  const bool split = (long long)p.V * 2 >= kSplitRowBytes && p.N <= 0x3fffffffll && p.entropy == nullptr;
+  const bool f32 = dtype == MRL_F32;
+  const bool split = (long long)p.V * (f32 ? 4 : 2) >= kSplitRowBytes && p.N <= 0x3fffffffll && p.entropy == nullptr;
   const bool ent = p.entropy != nullptr;
   const int C = split ? 2 : 1;
   // gradient launches of whole rows park the vectors read first (whole groups of blockDim vectors)
@@ -927,12 +964,18 @@ int launch_rows(RowParams p, int dtype, cudaStream_t st) {
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   using Kernel = void (*)(const RowParams);
-  const Kernel k = words == 8 ? (split ? row_stream_kernel<kStreamThreads, 4, 8, 2, false>
-                                 : ent ? row_stream_kernel<kStreamThreads, 4, 8, 1, true>
-                                       : row_stream_kernel<kStreamThreads, 4, 8, 1, false>)
-                              : (split ? row_stream_kernel<kStreamThreads, 8, 4, 2, false>
-                                 : ent ? row_stream_kernel<kStreamThreads, 8, 4, 1, true>
-                                       : row_stream_kernel<kStreamThreads, 8, 4, 1, false>);
+  const Kernel k = f32 ? (words == 8 ? (split ? row_stream_kernel<kStreamThreads, 4, 8, 2, false, true>
+                                        : ent ? row_stream_kernel<kStreamThreads, 4, 8, 1, true, true>
+                                              : row_stream_kernel<kStreamThreads, 4, 8, 1, false, true>)
+                                     : (split ? row_stream_kernel<kStreamThreads, 8, 4, 2, false, true>
+                                        : ent ? row_stream_kernel<kStreamThreads, 8, 4, 1, true, true>
+                                              : row_stream_kernel<kStreamThreads, 8, 4, 1, false, true>))
+                       : (words == 8 ? (split ? row_stream_kernel<kStreamThreads, 4, 8, 2, false, false>
+                                        : ent ? row_stream_kernel<kStreamThreads, 4, 8, 1, true, false>
+                                              : row_stream_kernel<kStreamThreads, 4, 8, 1, false, false>)
+                                     : (split ? row_stream_kernel<kStreamThreads, 8, 4, 2, false, false>
+                                        : ent ? row_stream_kernel<kStreamThreads, 8, 4, 1, true, false>
+                                              : row_stream_kernel<kStreamThreads, 8, 4, 1, false, false>));
   if (park_bytes > 0) {
     // exactly the carve-out two CTAs per SM need, as a percentage of the 228 KB an SM can give: the rest stays L1
     const int carve = (int)((2 * (park_bytes + 2048) * 100 + 228 * 1024 - 1) / (228 * 1024));
@@ -1013,10 +1056,14 @@ int launch_rows_backward(const RowParams& p, int dtype, const float* g, const fl
   const int words = pick_stream_words(p, dtype);
   const unsigned n = (unsigned)p.N;
   mrl_profile_before(st);
-  if (words == 8)
-    row_backward_stream_kernel<kStreamThreads, 4, 8><<<n, kStreamThreads, 0, st>>>(p, g, lse2, zt);
+  if (words == 8 && dtype == MRL_BF16)
+    row_backward_stream_kernel<kStreamThreads, 4, 8, false><<<n, kStreamThreads, 0, st>>>(p, g, lse2, zt);
+  else if (words == 4 && dtype == MRL_BF16)
+    row_backward_stream_kernel<kStreamThreads, 8, 4, false><<<n, kStreamThreads, 0, st>>>(p, g, lse2, zt);
+  else if (words == 8)
+    row_backward_stream_kernel<kStreamThreads, 4, 8, true><<<n, kStreamThreads, 0, st>>>(p, g, lse2, zt);
   else if (words == 4)
-    row_backward_stream_kernel<kStreamThreads, 8, 4><<<n, kStreamThreads, 0, st>>>(p, g, lse2, zt);
+    row_backward_stream_kernel<kStreamThreads, 8, 4, true><<<n, kStreamThreads, 0, st>>>(p, g, lse2, zt);
   else if (dtype == MRL_BF16)
     row_backward_general_kernel<__nv_bfloat16><<<n, kThreads, 0, st>>>(p, g, lse2, zt);
   else
