@@ -1,11 +1,10 @@
 // Logits-in path: mrl_token_logprobs and mrl_policy_loss_fwd_bwd.
 //
-// Streaming kernel (bf16 or float32, 16- or 32-byte aligned rows of at least 4,096 columns): one CTA per logits row,
-// two CTAs per SM.  Pass 1
-// streams the row from HBM with wide loads while keeping a running (max, sum of exponentials) per thread;
-// after the block reduction and the ratio / clip / loss scalars, pass 2 re-reads the row -- from L2, which
-// holds every row in flight several times over -- and writes g * (softmax - onehot) with streaming stores.
-// The row crosses the HBM interface once in each direction; nothing is shared between CTAs.
+// Streaming kernel (bf16 or float32, 16- or 32-byte aligned rows of at least 4,096 columns): one CTA per logits
+// row, two CTAs per SM.  Pass 1 streams the row from HBM with wide loads while keeping a running (max, sum of
+// exponentials) per thread; after the block reduction and the ratio / clip / loss scalars, pass 2 takes the row
+// again -- from registers, shared memory and L2 -- and writes g * (softmax - onehot) with streaming stores.  The row
+// crosses the HBM interface once in each direction (plus what L2 has dropped); nothing is shared between CTAs.
 // General kernel (any dtype, any V, any alignment): one CTA per row, three passes over global
 // memory; used for short or unaligned rows.
 #include <type_traits>
