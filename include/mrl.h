@@ -18,8 +18,9 @@
  *    `status` word [device, int32[1], nullable], treats the offending row as masked and goes
  *    on.  The library never clears `status`; zero it before the first call and read it after
  *    your own synchronisation.  Bits: MRL_DEV_BAD_TOKEN_ID (an id outside [0, V)),
- *    MRL_DEV_TIMEOUT (fused LM head only: a bounded wait on the kernel's own asynchronous copy
- *    or tensor-core work ran out; outputs of that call are then unspecified).
+ *    MRL_DEV_TIMEOUT (a bounded wait inside a kernel ran out -- on the fused LM head's own asynchronous
+ *    copies or tensor-core work, or on the exchange between the two CTAs that share a logits row of
+ *    512 KB or more; outputs of that call are then unspecified), MRL_DEV_BAD_WORD_MAP (word alignment).
  *  - `workspace` [device] is scratch of at least mrl_workspace_bytes(...) bytes, 256-byte
  *    aligned, contents unspecified before and after.  Calls that share a workspace must not
  *    overlap on the device.
