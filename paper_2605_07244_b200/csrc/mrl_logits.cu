@@ -947,8 +947,8 @@ int launch_rows(RowParams p, int dtype, cudaStream_t st) {
   const bool split = (long long)p.V * (f32 ? 4 : 2) >= kSplitRowBytes && p.N <= 0x3fffffffll && p.entropy == nullptr;
   const bool ent = p.entropy != nullptr;
   const int C = split ? 2 : 1;
-  // gradient launches of whole rows park the vectors read first (whole groups of blockDim vectors)
-  p.keep_q = (p.dlogits != nullptr && !split) ? kParkBytes / (kStreamThreads * words * 4) : 0;
+  // gradient launches park the vectors each CTA reads first (whole groups of blockDim vectors)
+  p.keep_q = p.dlogits != nullptr ? kParkBytes / (kStreamThreads * words * 4) : 0;
   const size_t park_bytes = (size_t)p.keep_q * kStreamThreads * words * 4;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(n * (unsigned)C);
