@@ -518,6 +518,49 @@ def measure_tiny_latency(seed):
             "kernels_per_step": wl.kernels_per_step, "steps": reps, "status": int(wl.status.cpu())}
 
 
+def measure_float32_rows(seed, peaks):
+    """The same pass on float32 logits at the 151,936-column vocabulary (608 KB per row: each row is shared by a pair of
+    CTAs): 8,192 rows, 5 GB in and 5 GB out per step."""
+    from paper_2605_07244_b200 import binding as B
+    N, V, S = 8192, 151936, 16
+    g = torch.Generator(device="cuda")
+    g.manual_seed(seed)
+    z = torch.empty(N, V, device="cuda")
+    z.normal_(0.0, 2.0, generator=g)
+    ids = torch.randint(0, V, (N,), dtype=torch.int32, device="cuda", generator=g)
+    cu = torch.arange(0, N + 1, N // S, dtype=torch.int32, device="cuda")
+    adv = torch.randn(S, device="cuda", generator=g)
+    logp = torch.empty(N, device="cuda")
+    B.mrl_token_logprobs(z, ids, None, logp)
+    old = logp + 0.1 * torch.randn(N, device="cuda", generator=g)
+    dz = torch.empty_like(z)
+    loss = torch.zeros(2, device="cuda")
+    stats = torch.zeros(4, dtype=torch.int64, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ws = torch.empty(B.workspace_bytes(B.WS_POLICY_LOSS, N, V, 0, B.F32, S), dtype=torch.uint8, device="cuda")
+    lp = B.LossParams(0.2, 0.2, B.AGG_TOKEN_MEAN, 0, 0.0, 0.0, 0.0, 0)
+    f = lambda: B.mrl_policy_loss_fwd_bwd(z, ids, None, cu, adv, old, None, None, lp, dz, logp, loss, stats, status, ws)
+    for _ in range(3):
+        f()
+    steps = 20
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(steps):
+        f()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    alg = 2 * N * V * 4
+    gbs = alg / (ms * 1e-3) / 1e9
+    return {"metric": METRIC, "value": N / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms, "steps": steps, "rows": N, "V": V,
+            "logits_dtype": "f32", "status": int(status.cpu()),
+            "roofline": {"bound": "hbm", "kernel": "row_stream_kernel (float32, row split over two CTAs)", "achieved": gbs,
+                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+                         "peak_source": peaks["source"] + " (copy, burst)", "algorithmic_bytes_per_launch": alg,
+                         "traffic": None}}
+
+
 def measure_thl_align(seed, with_cpu):
     """THL word alignment on a batch shaped like one PRP step of App. G.1: 256 prompts x 5 peer rollouts of
     ~630 response tokens, words cut into 1..4 tokens by each tokenizer.  It is tiny next to the loss pass (a few
@@ -723,10 +766,11 @@ def run_ours(args, rank, world, local_rank):
         lmhead["skip_zero_rows"] = {k: r5b[k] for k in ("value", "ms_per_step", "steps", "config", "roofline")}
         del wl5b
 
-    thl = tiny = None
+    thl = tiny = f32 = None
     if args.workload == "C2" and not args.no_lmhead and rank == 0 and world == 1:
         thl = measure_thl_align(args.seed, not args.no_cpu_baseline)
         tiny = measure_tiny_latency(args.seed)
+        f32 = measure_float32_rows(args.seed, peaks)
 
     if rank == 0:
         line = {
@@ -745,6 +789,8 @@ def run_ours(args, rank, world, local_rank):
             line["thl_align"] = thl
         if tiny is not None:
             line["tiny_step_latency"] = tiny
+        if f32 is not None:
+            line["float32_logits"] = f32
         print(json.dumps(line))
 
 
