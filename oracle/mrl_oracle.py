@@ -22,7 +22,8 @@ Passages followed (by section / equation of the paper):
   * softmax score  grad log pi(a_i) = e_i - pi                            (App. H, proof of Prop. 1)
   * response-level ratio  w = exp(L_theta - L_behavior)                     (App. H, data-level coupling)
   * policy entropy diagnostic  H_t = - sum_v p_v log p_v                   (Sec. 6, App. B: entropy curves)
-  * THL word-level trace alignment  Z_w, C_w, Z_w / C_w                    (Sec. 4.2; App. D, Alg. 3; Thm. 1)
+  * THL word-level trace alignment  Z_w, C_w, Z_w / max(1, C_w)            (Sec. 4.2; Thm. 1; conventions of App. D)
+  * THL WordSpans: maximal non-whitespace runs as character intervals      (App. D, Alg. 2)
   * KL-style regulariser  beta R(theta): a per-token KL to a reference, its own loss term,
     coefficient 1e-3                                                      (Eq. (1); App. A, hyperparameters)
 
@@ -33,7 +34,8 @@ Pins (tests, CPU only): closed forms (uniform logits, V = 1, binary-reward
 advantages), brute force on tiny inputs, finite differences, the printed
 three-action example of Prop. 1, the rescue-gate probability of Def. 7, and
 library special cases (scipy logsumexp, torch cross_entropy), and for the word alignment the per-word mass
-conservation and the residual identity of Thm. 1 evaluated from its own set definitions; for the KL penalty
+conservation and the residual identity of Thm. 1 evaluated from its own set definitions (WordSpans: hand-counted
+intervals of the paper's example sentence, maximality and coverage); for the KL penalty
 the exact expectation identities E_pi[k1] = E_pi[k3] = KL(pi || ref) against scipy's rel_entr, second-order
 agreement of k2, non-negativity, closed forms for a constant log-ratio, and finite differences.
 Functions without a pin: none.
@@ -41,6 +43,7 @@ Functions without a pin: none.
 from __future__ import annotations
 
 import math
+import re
 from dataclasses import dataclass
 
 import torch
@@ -487,20 +490,23 @@ def fused_lmhead_loss(hidden, W, ids, mask, cu_seqlens, adv_seq, logp_old, tok_w
 
 
 # ---------------------------------------------------------------------------------------------------------------
-# THL WordAlignLogProbs (Sec. 4.2; App. D, Alg. 3; Thm. 1)
+# THL word-level trace alignment (Sec. 4.2; Thm. 1; App. D)
 # ---------------------------------------------------------------------------------------------------------------
 
 def thl_word_align_logprobs(src_logp, src_word, src_cu, tgt_word, tgt_cu, ignore_value: float = 0.0):
-    """Word-level trace alignment of App. D, Alg. 3, on packed response tokens, in the algorithm's own steps.
+    """Word-level trace alignment, written out from its definition (Sec. 4.2; Thm. 1 of App. H), on packed response
+    tokens.  Within one sequence, with S_w the source tokens and T_w the target tokens attributed to word w:
 
-    For sequence i the source tokens are src_cu[i] .. src_cu[i+1]-1 with log-probs `src_logp` and word ids
-    `src_word` (the token-to-word map of Alg. 1; -1 = None), the target tokens tgt_cu[i] .. with word ids
-    `tgt_word`.  (The response masks of the algorithm are already applied: only response tokens are passed.)
-      pass 1: per_word_sum[w] = sum of the source log-probs of the tokens mapped to w          (Z_w)
-      a sequence whose per_word_sum is empty is skipped: its outputs stay at ignore_value
-      pass 2: per_word_count[w] = number of target tokens mapped to w                        (C_w)
-      pass 3: every target token with a word gets per_word_sum.get(w, 0) / per_word_count[w]
-    Returns out f64[N_tgt] (ignore_value where nothing is assigned).
+        Z_w = sum_{s in S_w} l_src[s]          (word-level mass; 0 for a word with no source token)
+        C_w = |T_w|                            (target tokens of the word)
+        aligned[t] = Z_{w(t)} / max(1, C_{w(t)})   for every target token t that has a word
+
+    Sequence i owns source tokens [src_cu[i], src_cu[i+1]) and target tokens [tgt_cu[i], tgt_cu[i+1]); a word id
+    below zero means "no word".  Two conventions come from the routine of App. D rather than from the formula:
+    tokens without a word keep `ignore_value`, and so does every target token of a sequence in which no source
+    token has a word (such a sequence carries no mass to distribute).  The response masks m_src, m_tgt of the
+    formula are already applied: only response tokens are passed.
+    Returns f64[N_tgt].
     """
     src_logp = torch.as_tensor(src_logp).to(F64)
     src_word = torch.as_tensor(src_word).long()
@@ -509,29 +515,24 @@ def thl_word_align_logprobs(src_logp, src_word, src_cu, tgt_word, tgt_cu, ignore
     tgt_cu = torch.as_tensor(tgt_cu).long()
     out = torch.full((int(tgt_cu[-1]) if tgt_cu.numel() else 0,), float(ignore_value), dtype=F64)
     for i in range(src_cu.numel() - 1):
-        per_word_sum = {}
-        for p in range(int(src_cu[i]), int(src_cu[i + 1])):
-            wid = int(src_word[p])
-            if wid < 0:
-                continue
-            per_word_sum[wid] = per_word_sum.get(wid, 0.0) + float(src_logp[p])
-        if not per_word_sum:
+        sw = src_word[int(src_cu[i]):int(src_cu[i + 1])]
+        tw = tgt_word[int(tgt_cu[i]):int(tgt_cu[i + 1])]
+        s_has, t_has = sw >= 0, tw >= 0
+        if not bool(s_has.any()):
             continue
-        per_word_count = {}
-        for p in range(int(tgt_cu[i]), int(tgt_cu[i + 1])):
-            wid = int(tgt_word[p])
-            if wid < 0:
-                continue
-            per_word_count[wid] = per_word_count.get(wid, 0) + 1
-        for p in range(int(tgt_cu[i]), int(tgt_cu[i + 1])):
-            wid = int(tgt_word[p])
-            if wid < 0:
-                continue
-            cnt = per_word_count.get(wid, 0)
-            if cnt <= 0:
-                continue
-            out[p] = per_word_sum.get(wid, 0.0) / cnt
+        n_words = int(max(sw.max(), tw.max() if tw.numel() else -1)) + 1
+        Z = torch.zeros(n_words, dtype=F64).index_add_(0, sw[s_has], src_logp[int(src_cu[i]):int(src_cu[i + 1])][s_has])
+        C = torch.bincount(tw[t_has], minlength=n_words)
+        w_t = tw[t_has]
+        seg = out[int(tgt_cu[i]):int(tgt_cu[i + 1])]
+        seg[t_has] = Z[w_t] / torch.clamp(C[w_t], min=1).to(F64)
     return out
+
+
+def thl_word_spans(text: str):
+    """WordSpans (App. D, Alg. 2) as the paper defines it: one (start, end) character interval, end exclusive, per
+    match of the regular expression for a maximal run of non-whitespace characters, in order of appearance."""
+    return [(m.start(), m.end()) for m in re.finditer(r"\S+", text)]
 
 
 def thl_sequence_totals(src_logp, src_cu, aligned, tgt_word, tgt_cu, has_source):
