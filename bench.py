@@ -128,6 +128,52 @@ def aggregate_over_ranks(local_ms: float, local_units: float, world: int):
     return float(t.item()), float(u.item())
 
 
+def launch_ranks(n: int, argv, script=None, extra_env=None) -> int:
+    """Starts one process per GPU on this node (ranks 0 .. n-1, rendezvous on 127.0.0.1) running `script` with
+    `argv`, waits for all of them and returns 0 only if every rank exited 0.  As soon as one rank fails the others
+    are terminated (they would otherwise wait for it in a collective)."""
+    import socket
+    import subprocess
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    script = script or os.path.abspath(__file__)
+    procs = []
+    for r in range(n):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT=str(port))
+        env.update(extra_env or {})
+        procs.append(subprocess.Popen([sys.executable, script] + list(argv), env=env))
+    worst = 0
+    pending = set(range(n))
+    while pending:
+        for r in sorted(pending):
+            rc = procs[r].poll()
+            if rc is None:
+                continue
+            pending.discard(r)
+            if rc != 0:
+                worst = worst or (rc if rc > 0 else 1)
+                for q in sorted(pending):        # exact children of this process, nothing else
+                    procs[q].terminate()
+        time.sleep(0.05)
+    return worst
+
+
+def resolve_world(gpus: int):
+    """(rank, world, local_rank) from the launcher's environment; None when this process has to start the ranks
+    itself (`--gpus N` > 1 given to a plain `python bench.py`).  A world size that contradicts --gpus is an error:
+    a number labelled N GPUs must come from N ranks."""
+    if "WORLD_SIZE" not in os.environ:
+        if gpus > 1:
+            return None
+        return 0, 1, 0
+    world = int(os.environ["WORLD_SIZE"])
+    if world != gpus:
+        raise SystemExit(f"bench.py: --gpus {gpus} but the launcher started WORLD_SIZE={world} ranks")
+    return int(os.environ.get("RANK", "0")), world, int(os.environ.get("LOCAL_RANK", "0"))
+
+
 def barrier(world: int):
     if world > 1:
         import torch.distributed as dist
@@ -730,6 +776,8 @@ def measure(wl, steps, warmup, world, local_rank, rank, peaks, with_e2e, with_cp
 def run_ours(args, rank, world, local_rank):
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    if torch.cuda.device_count() <= local_rank:
+        raise SystemExit(f"bench.py: rank {rank} wants cuda:{local_rank} but {torch.cuda.device_count()} device(s) are visible")
     torch.cuda.set_device(local_rank)
     device = torch.device("cuda", local_rank)
     from paper_2605_07244_b200 import binding as B
@@ -817,9 +865,12 @@ def main():
                     help="fused LM-head workloads: 256-row tiles worked by CTA pairs (MRL_FLAG_PAIR_TILES)")
     ap.add_argument("--no-lmhead", action="store_true", help="skip the short config-5 leg of the default run")
     args = ap.parse_args()
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.gpus < 1:
+        raise SystemExit("bench.py: --gpus must be at least 1")
+    placed = resolve_world(args.gpus)
+    if placed is None:          # plain `python bench.py --gpus N`: start the N ranks here
+        sys.exit(launch_ranks(args.gpus, sys.argv[1:]))
+    rank, world, local_rank = placed
     if args.impl == "reference":
         run_reference(args, rank, world)
         return

@@ -39,7 +39,7 @@
 extern "C" {
 #endif
 
-#define MRL_VERSION 103
+#define MRL_VERSION 104
 
 /* return codes */
 #define MRL_OK 0
@@ -375,6 +375,7 @@ int mrl_fused_lmhead_loss_fwd_bwd(const void* hidden, const void* W, int64_t N, 
  *   src_word   [device] int32   [N_src]  word id of each source token (App. D, Alg. 1), negative = no word
  *   tgt_word   [device] int32   [N_tgt]  the same for the learner's tokens
  *   src_cu, tgt_cu, word_cu  [device] int32 [B+1], non-decreasing, starting at 0
+ *   N_src, N_tgt lengths of the source and target token arrays (src_cu[B] and tgt_cu[B])
  *   total_words  word_cu[B] (sizes the workspace)
  *   out        [device] float32 [N_tgt]  aligned trace; every element is written
  *   src_total  [device] float32 [B], nullable: sum of all source log-probs of the sequence (L_mu of Thm. 1)
@@ -385,11 +386,14 @@ int mrl_fused_lmhead_loss_fwd_bwd(const void* hidden, const void* W, int64_t N, 
  * Equal word ids must be contiguous within a sequence (what a span-by-span tokenisation yields); then every sum
  * is taken in token order by one thread and results are bitwise reproducible.  A word id seen in two separate
  * runs or outside the sequence's range sets MRL_DEV_BAD_WORD_MAP in `status` (such tokens count as "no word" /
- * their word's value is then unspecified).  float32 sums.  B = 0 is a no-op.
+ * their word's value is then unspecified).  So does an offset array that decreases or reaches past N_src, N_tgt or
+ * total_words: each sequence's ranges are cut to the arrays, nothing outside them is read or written, and the outputs
+ * of that sequence are unspecified.  float32 sums.  B = 0 is a no-op.
  */
 int mrl_thl_word_align_logprobs(const float* src_logp, const int32_t* src_word, const int32_t* src_cu,
                                 const int32_t* tgt_word, const int32_t* tgt_cu, const int32_t* word_cu, int32_t B,
-                                int64_t total_words, float ignore_value, float* out, float* src_total,
+                                int64_t N_src, int64_t N_tgt, int64_t total_words, float ignore_value, float* out,
+                                float* src_total,
                                 float* tgt_total, int32_t* status, void* workspace, size_t workspace_bytes,
                                 void* stream);
 

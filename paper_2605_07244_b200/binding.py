@@ -81,7 +81,8 @@ def lib() -> C.CDLL:
         L.mrl_fused_lmhead_loss_fwd_bwd.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, vp, vp, vp,
                                                     C.POINTER(LossParams), vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.mrl_fused_lmhead_loss_fwd_bwd.restype = C.c_int
-        L.mrl_thl_word_align_logprobs.argtypes = [vp, vp, vp, vp, vp, vp, i32, i64, C.c_float, vp, vp, vp, vp, vp, sz, vp]
+        L.mrl_thl_word_align_logprobs.argtypes = [vp, vp, vp, vp, vp, vp, i32, i64, i64, i64, C.c_float, vp, vp, vp, vp,
+                                                  vp, sz, vp]
         L.mrl_thl_word_align_logprobs.restype = C.c_int
         L.mrl_workspace_bytes.argtypes = [i32, i64, i32, i32, i32, i32]
         L.mrl_workspace_bytes.restype = sz
@@ -226,7 +227,8 @@ def mrl_thl_word_align_logprobs(src_logp, src_word, src_cu, tgt_word, tgt_cu, wo
     Bn = src_cu.numel() - 1
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     _check(lib().mrl_thl_word_align_logprobs(_p(src_logp), _p(src_word), _p(src_cu), _p(tgt_word), _p(tgt_cu),
-                                             _p(word_cu), Bn, int(total_words), float(ignore_value), _p(out),
+                                             _p(word_cu), Bn, src_word.numel(), out.numel(), int(total_words),
+                                             float(ignore_value), _p(out),
                                              _p(src_total), _p(tgt_total), _p(status), _p(workspace), ws_bytes,
                                              _stream(stream)), "mrl_thl_word_align_logprobs")
 

@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "mrl.h"
 
 #define MRL_LOG2E 1.4426950408889634f
@@ -17,6 +19,19 @@
   } while (0)
 
 static inline size_t mrl_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Runs `set` (the cudaFuncSetAttribute calls of one kernel) once per device instead of on every launch: `done` holds
+// one bit per device ordinal.  Two threads that race here both set the same attributes, which is harmless.
+template <typename F>
+static inline int mrl_once_per_device(std::atomic<uint64_t>& done, F set) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return MRL_ERR_CUDA;
+  const uint64_t bit = 1ull << (dev & 63);
+  if (done.load(std::memory_order_acquire) & bit) return MRL_OK;
+  if (set() != cudaSuccess) return MRL_ERR_CUDA;
+  done.fetch_or(bit, std::memory_order_release);
+  return MRL_OK;
+}
 
 // Carves sub-buffers out of the caller's workspace; every piece is 256-byte aligned.
 struct MrlCarver {

@@ -793,8 +793,15 @@ int launch_gemm(const void* A, long long lda, const void* B, long long ldb, Gemm
   p.n_tiles = (p.N + BN - 1) / BN;
   p.k_blocks = (p.K + BK - 1) / BK;
   // two-CTA tiles (256 rows) when asked for and pairs can be scheduled, else one CTA per 128-row tile
-  MRL_CUDA_OK(cudaFuncSetAttribute(lmhead_gemm_kernel<EPI, 2, kAMn, kBMn>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   (int)GemmCfg<2>::kSmem));
+  static std::atomic<uint64_t> attr_done;  // one per instantiation: both tile shapes' shared-memory limits, once per device
+  const int arc = mrl_once_per_device(attr_done, [] {
+    const cudaError_t e = cudaFuncSetAttribute(lmhead_gemm_kernel<EPI, 2, kAMn, kBMn>,
+                                               cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GemmCfg<2>::kSmem);
+    return e != cudaSuccess ? e
+                            : cudaFuncSetAttribute(lmhead_gemm_kernel<EPI, 1, kAMn, kBMn>,
+                                                   cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GemmCfg<1>::kSmem);
+  });
+  if (arc != MRL_OK) return arc;
   cudaLaunchConfig_t cfg = {};
   cfg.blockDim = dim3(kGemmThreads);
   cfg.dynamicSmemBytes = GemmCfg<2>::kSmem;
@@ -838,8 +845,6 @@ int launch_gemm(const void* A, long long lda, const void* B, long long ldb, Gemm
     return e == cudaSuccess ? MRL_OK : MRL_ERR_CUDA;
   }
   const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
-  MRL_CUDA_OK(cudaFuncSetAttribute(lmhead_gemm_kernel<EPI, 1, kAMn, kBMn>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   (int)GemmCfg<1>::kSmem));
   mrl_profile_before(st);
   lmhead_gemm_kernel<EPI, 1, kAMn, kBMn><<<grid, kGemmThreads, GemmCfg<1>::kSmem, st>>>(ta, tb, p);
   mrl_profile_after(st);

@@ -29,13 +29,20 @@ __global__ void __launch_bounds__(kAlignThreads) thl_word_align_kernel(
     const float* __restrict__ src_logp, const int32_t* __restrict__ src_word, const int32_t* __restrict__ src_cu,
     const int32_t* __restrict__ tgt_word, const int32_t* __restrict__ tgt_cu, const int32_t* __restrict__ word_cu,
     float ignore_value, float* __restrict__ out, float* __restrict__ src_total, float* __restrict__ tgt_total,
-    float* __restrict__ word_sum, int32_t* __restrict__ word_cnt, int32_t* status) {
+    float* __restrict__ word_sum, int32_t* __restrict__ word_cnt, long long n_src, long long n_tgt,
+    long long total_words, int32_t* status) {
   __shared__ float scratch[kAlignThreads / 32];
   __shared__ int any_source, bad;
   const int i = blockIdx.x, tid = threadIdx.x;
-  const int s0 = src_cu[i], ns = max(0, src_cu[i + 1] - s0);
-  const int t0 = tgt_cu[i], nt = max(0, tgt_cu[i + 1] - t0);
-  const int w0 = word_cu[i], nw = max(0, word_cu[i + 1] - w0);
+  // Offsets come from device memory the host cannot check: every range is cut to its array, so a corrupt offset
+  // array raises MRL_DEV_BAD_WORD_MAP instead of reaching outside the buffers.
+  const long long s_lo = src_cu[i], s_hi = src_cu[i + 1], t_lo = tgt_cu[i], t_hi = tgt_cu[i + 1];
+  const long long w_lo = word_cu[i], w_hi = word_cu[i + 1];
+  const bool bad_offsets = s_lo < 0 || s_hi < s_lo || s_hi > n_src || t_lo < 0 || t_hi < t_lo || t_hi > n_tgt ||
+                           w_lo < 0 || w_hi < w_lo || w_hi > total_words;
+  const int s0 = (int)min(max(s_lo, 0ll), n_src), ns = (int)(min(max(s_hi, (long long)s0), n_src) - s0);
+  const int t0 = (int)min(max(t_lo, 0ll), n_tgt), nt = (int)(min(max(t_hi, (long long)t0), n_tgt) - t0);
+  const int w0 = (int)min(max(w_lo, 0ll), total_words), nw = (int)(min(max(w_hi, (long long)w0), total_words) - w0);
   float* zsum = word_sum + w0;   // Z_w
   int32_t* cnt = word_cnt + w0;  // C_w; -1 while the word has not been seen on the source side either
   const int32_t* sw = src_word + s0;
@@ -43,7 +50,7 @@ __global__ void __launch_bounds__(kAlignThreads) thl_word_align_kernel(
 
   if (tid == 0) {
     any_source = 0;
-    bad = 0;
+    bad = bad_offsets ? 1 : 0;
   }
   for (int w = tid; w < nw; w += kAlignThreads) {
     zsum[w] = 0.f;
@@ -111,10 +118,13 @@ size_t mrl_thl_workspace_bytes(long long total_words) {
 
 extern "C" int mrl_thl_word_align_logprobs(const float* src_logp, const int32_t* src_word, const int32_t* src_cu,
                                            const int32_t* tgt_word, const int32_t* tgt_cu, const int32_t* word_cu,
-                                           int32_t B, int64_t total_words, float ignore_value, float* out,
+                                           int32_t B, int64_t N_src, int64_t N_tgt, int64_t total_words,
+                                           float ignore_value, float* out,
                                            float* src_total, float* tgt_total, int32_t* status, void* workspace,
                                            size_t workspace_bytes, void* stream) {
-  if (B < 0 || total_words < 0) return MRL_ERR_INVALID_ARG;
+  if (B < 0 || total_words < 0 || N_src < 0 || N_tgt < 0 || N_src > 0x7fffffffll || N_tgt > 0x7fffffffll ||
+      total_words > 0x7fffffffll)
+    return MRL_ERR_INVALID_ARG;
   if (B == 0) return MRL_OK;
   if (src_word == nullptr || src_cu == nullptr || tgt_word == nullptr || tgt_cu == nullptr || word_cu == nullptr ||
       src_logp == nullptr || out == nullptr)
@@ -128,7 +138,7 @@ extern "C" int mrl_thl_word_align_logprobs(const float* src_logp, const int32_t*
   mrl_profile_before(st);
   thl_word_align_kernel<<<(unsigned)B, kAlignThreads, 0, st>>>(src_logp, src_word, src_cu, tgt_word, tgt_cu, word_cu,
                                                                ignore_value, out, src_total, tgt_total, word_sum,
-                                                               word_cnt, status);
+                                                               word_cnt, N_src, N_tgt, total_words, status);
   mrl_profile_after(st);
   return cudaGetLastError() == cudaSuccess ? MRL_OK : MRL_ERR_CUDA;
 }

@@ -151,6 +151,13 @@ CASES = [
     (5, 65552, 2, torch.bfloat16, 16, None),    # 256-bit accesses, padded rows
     (4, 262160, 2, torch.bfloat16, 0, None),    # row split over a cluster of two CTAs, 256-bit accesses
     (3, 262152, 1, torch.bfloat16, 0, 0.7),     # the same with 128-bit accesses and a masked row
+    # rows kept on the SM between the passes (64 KB < row <= 304 KB, 256-bit accesses): registers plus a tail in shared memory
+    (6, 32784, 2, torch.bfloat16, 0, 0.8),      # one CTA, a tail of 32 bytes
+    (6, 50000, 3, torch.bfloat16, 0, None),     # one CTA, ragged tail
+    (4, 77824, 2, torch.bfloat16, 16, None),    # one CTA, the largest tail, padded rows
+    (5, 100016, 2, torch.bfloat16, 16, 0.8),    # two CTAs with unequal halves
+    (3, 155648, 2, torch.bfloat16, 0, None),    # two CTAs, the largest row that stays resident
+    (3, 155664, 1, torch.bfloat16, 0, None),    # one vector more: back to the streaming kernel
 ]
 
 
@@ -456,7 +463,7 @@ def test_config2_full_size_sampled_rows():
 
 
 @pytest.mark.parametrize("V,dtype", [(1000, torch.float32), (4096, torch.bfloat16), (40008, torch.bfloat16),
-                                     (262144 + 16, torch.bfloat16)])
+                                     (262144 + 16, torch.bfloat16), (50000, torch.bfloat16), (151936, torch.bfloat16)])
 def test_extreme_logits(V, dtype):
     """Vocabulary masking with -inf, a logit that dominates the row, large magnitudes, an exactly uniform row: the
     running maximum / rescaled sum must neither overflow nor produce NaN, and must match the oracle."""

@@ -97,3 +97,22 @@ def test_sequence_ratio_hidden_in(N, H, V, S, mask_p):
     dz = ref["dlogits"]
     assert rel_l2(got["dH"].double(), dz @ W.double()) <= GRAD_REL_L2_BF16
     assert rel_l2(got["dW"].double(), dz.T @ hidden.double()) <= GRAD_REL_L2_BF16
+
+
+@pytest.mark.parametrize("N,V,dtype", [(40, 1000, torch.float32), (36, 8192, torch.bfloat16)])
+def test_rows_outside_every_sequence_get_no_gradient(N, V, dtype):
+    """cu_seqlens may stop short of N (the contract asks for cu[S] = N, but only the device sees the array): the rows
+    no response covers must come out with zero gradient rows and logp = 0, and must not disturb the covered rows."""
+    S, Nc = 3, N - 9
+    z, ids, _, _, adv, old, nllw = toy(N, V, S, dtype, seed=5 + V)
+    cu = torch.tensor([0, 7, 19, Nc], dtype=torch.int32)
+    lp = make_lp(nll_coeff=0.05, ratio_level=B.RATIO_SEQUENCE)
+    got = run_gpu_policy_loss(z, ids, None, cu, adv, old, None, nllw, lp, V=V)
+    ref = O.policy_loss_sequence_ratio(z[:Nc, :V], ids[:Nc], None, cu, adv, old[:Nc], nllw[:Nc], oracle_lp(lp))
+    assert got["status"] == 0
+    assert float(got["dlogits"][Nc:].abs().max()) == 0 and float(got["logp"][Nc:].abs().max()) == 0
+    assert (got["logp"][:Nc].double() - ref["logp"]).abs().max() <= LOGP_ATOL
+    scale = max(abs(ref["loss_pg"]), float(ref["seq_term"].abs().sum()))
+    assert abs(float(got["loss"][0]) - ref["loss_pg"]) <= LOSS_RTOL * scale
+    tol = GRAD_REL_L2_BF16 if dtype == torch.bfloat16 else GRAD_REL_L2_F32
+    assert rel_l2(got["dlogits"][:Nc, :V].double(), ref["dlogits"]) <= tol

@@ -102,5 +102,36 @@ def test_degenerate_and_bad_maps():
     assert torch.equal(src_total, torch.tensor([0.0, -4.0, 0.0])) and torch.equal(tgt_total, torch.tensor([0.0, -4.0, 0.0]))
     # B = 0 is a no-op, null pointers with B > 0 are refused on the host
     f = B.lib().mrl_thl_word_align_logprobs
-    assert f(None, None, None, None, None, None, 0, 0, 0.0, None, None, None, None, None, 0, None) == 0
-    assert f(None, None, None, None, None, None, 1, 0, 0.0, None, None, None, None, None, 0, None) == 1
+    assert f(None, None, None, None, None, None, 0, 0, 0, 0, 0.0, None, None, None, None, None, 0, None) == 0
+    assert f(None, None, None, None, None, None, 1, 0, 0, 0, 0.0, None, None, None, None, None, 0, None) == 1
+
+
+def test_offsets_beyond_the_arrays_are_reported_and_stay_inside_the_buffers():
+    """Offset arrays live in device memory, so only the kernel can check them.  Offsets that run past the token
+    arrays or the word total are cut to the arrays and reported through the status word; the cells beyond the
+    arrays' stated lengths (guard cells here) are neither read into the result nor written."""
+    ig = -7.0
+    i32 = lambda x: torch.tensor(x, dtype=torch.int32)
+    n_src, n_tgt, n_words, guard = 3, 4, 2, 64
+    src_logp = torch.cat([torch.tensor([-1.0, -0.5, -2.0]), torch.full((guard,), 1e30)]).cuda()
+    src_word = torch.cat([i32([0, 0, 1]), torch.zeros(guard, dtype=torch.int32)]).cuda()
+    tgt_word = torch.cat([i32([0, 0, 0, 1]), torch.zeros(guard, dtype=torch.int32)]).cuda()
+    out = torch.full((n_tgt + guard,), 123.0, device="cuda")
+    ws = torch.full((2 * 256 + 4 * guard,), 0x5A, dtype=torch.uint8, device="cuda")
+    for src_cu, tgt_cu, word_cu in (([0, 3 + 40], [0, 4], [0, 2]),          # source range past N_src
+                                    ([0, 3], [0, 4 + 40], [0, 2]),          # target range past N_tgt
+                                    ([0, 3], [0, 4], [0, 2 + 40]),          # word range past total_words
+                                    ([0, 3], [2, 1], [0, 2])):              # decreasing offsets
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        out.fill_(123.0)
+        d_src_cu, d_tgt_cu, d_word_cu = i32(src_cu).cuda(), i32(tgt_cu).cuda(), i32(word_cu).cuda()
+        rc = B.lib().mrl_thl_word_align_logprobs(
+            src_logp.data_ptr(), src_word.data_ptr(), d_src_cu.data_ptr(), tgt_word.data_ptr(),
+            d_tgt_cu.data_ptr(), d_word_cu.data_ptr(), 1, n_src, n_tgt, n_words, ig,
+            out.data_ptr(), None, None, status.data_ptr(), ws.data_ptr(), 2 * 256, None)
+        torch.cuda.synchronize()
+        assert rc == 0
+        assert int(status.cpu()) & B.DEV_BAD_WORD_MAP
+        assert bool((out[n_tgt:] == 123.0).all())                  # nothing written past N_tgt
+        assert bool((ws[2 * 256:] == 0x5A).all())                   # nothing written past the stated workspace
+        assert bool(torch.isfinite(out[:n_tgt]).all()) and float(out[:n_tgt].abs().max()) < 1e3   # guard values unread
