@@ -1,13 +1,17 @@
 #!/usr/bin/env python
 """Benchmark of the policy-loss hot path on B200 (one process per GPU).
 
-    python bench.py --gpus N --steps K --warmup W [--impl reference] [--workload C2|C2s|C5|C5s|C5b]
+    python bench.py --gpus N --steps K --warmup W [--impl reference] [--workload C2|C2s|C3|C4|C5|C5s|C5b]
 
 A step is one pass of the whole hot path over one batch of synthetic input: group advantages and
 SGT gate (mrl_group_advantages), then log-probs, ratio, clipped surrogate, aggregation and dlogits
 (mrl_policy_loss_fwd_bwd).  The workload at N = 1 is the Qwen-size-vocabulary configuration (151,936 columns,
 logits in, bf16, packed ragged sequences; `C2` in synth.py); each rank of an N-GPU run processes its own batch of the
 same shape (independent replicas, no data-path collective), so scaling is weak.
+
+Beside the headline the default run times, as sub-objects of the same line, the same batch with every row live (KL
+penalty on), one slab of the PRP-pool shape and one of the XGRPO + SGT shape, and the fused LM head.  Started without a
+launcher, `--gpus N` starts the N ranks itself.
 
 Rank 0 prints ONE JSON line.  `--impl reference` times the CPU float64 oracle on a bounded sample
 of the same workload instead (rank 0 only).
@@ -51,10 +55,16 @@ def measured_peaks():
     return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
 
 
-# DRAM bytes per token (dram__bytes_read.sum + dram__bytes_write.sum over the rows of the capture) of the dominant
-# kernel as it stands, from the committed ncu summary profiles/row_stream_kernel_c2_logits_in.md; traffic grows in
-# proportion to the rows.  Set to None whenever that kernel changes, until the counters are taken again.
-ROW_STREAM_DRAM_BYTES_PER_TOKEN_V151936 = 642153
+# DRAM bytes per token (dram__bytes_read.sum + dram__bytes_write.sum over the rows of one ncu capture of the small
+# case) of the dominant kernel, keyed by the kernel the library reports it launched, the vocabulary and whether every
+# row had a gradient; traffic grows in proportion to the rows.  A launch of any other kernel, shape or batch kind
+# prints `traffic: null`, and so does an entry set to None because its kernel changed after the counters were taken.
+DRAM_BYTES_PER_TOKEN = {
+    ("row_stream_kernel", 151936, "half-live"): 642153,
+    ("row_stream_kernel", 151936, "all-live"): 687300,
+}
+NOMINAL_HBM_GBS = 8000.0        # B200 data sheet (7.7 TB/s on HGX boards): context beside the measured copy rate
+NOMINAL_BF16_TFLOPS = 2250.0    # dense bf16
 
 
 class ClockSampler:
@@ -270,6 +280,7 @@ class LogitsInWorkload:
                 "steps": steps, "gpu_launches": steps,
                 "roofline": {"bound": "hbm", "kernel": "row_stream_kernel (forward only)", "achieved": gbs,
                              "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+                             "frac_nominal": gbs / NOMINAL_HBM_GBS,
                              "peak_source": peaks["source"] + " (copy, burst)", "algorithmic_bytes_per_launch": alg,
                              "traffic": None}}
 
@@ -360,16 +371,17 @@ class LogitsInWorkload:
             live_rows = int(lens[(self.adv_own.reshape(-1) != 0).cpu()].sum()) - int(self.stats.cpu()[1])
             alg_bytes = (2 * self.tokens() + live_rows) * self.V * self.z.element_size()
         achieved = alg_bytes / (k_avg_ms * 1e-3) / 1e9
-        per_token = (ROW_STREAM_DRAM_BYTES_PER_TOKEN_V151936 if self.V == 151936 and self.ratio_level == 0
-                     and not self.lp.logp_ref and not self.lp.entropy else None)   # counters exist for the default pass only
-        kernel = "row_stream_kernel" if self.ratio_level == 0 else "row_stream_kernel (forward) + row_backward_stream_kernel"
+        launched = getattr(self, "last_kernel", "")
+        kind = "all-live" if self.lp.logp_ref else "half-live"
+        per_token = None if (self.ratio_level != 0 or self.lp.entropy) else DRAM_BYTES_PER_TOKEN.get((launched, self.V, kind))
+        kernel = launched if self.ratio_level == 0 else "row_stream_kernel (forward) + row_backward_stream_kernel"
         return {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peaks["hbm_gbs"],
-                "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "frac_nominal": achieved / NOMINAL_HBM_GBS,
                 "peak_source": peaks["source"] + " (copy, burst)", "algorithmic_bytes_per_launch": alg_bytes,
                 "kernel_ms": k_avg_ms, "traffic": None if per_token is None else per_token * self.tokens()}
 
-    def time_oracle(self):
-        O, oargs, n = self.oracle_sample(ORACLE_ROWS)
+    def time_oracle(self, scale=1):
+        O, oargs, n = self.oracle_sample(ORACLE_ROWS // scale)
         dt = time_oracle(O, oargs)
         return n, dt, f"first {n} rows of the same batch, full V, fwd+bwd, float64, {dt:.1f} s"
 
@@ -386,6 +398,130 @@ class LogitsInWorkload:
         adv_seq = adv[b.seq_p.long(), b.seq_m.long(), b.seq_g.long()][:s_end]
         args = (z, b.ids[:n], None, b.cu_seqlens[:s_end + 1], adv_seq, self.logp_old[:n].cpu())
         return O, args, n
+
+
+class PoolSlabWorkload:
+    """One seeded micro-batch (a slab of whole sequences, at most `slab_rows` rows) of a step that is too large to
+    exist at once, timed as the step's calls on that slab with the whole step's denominators:
+
+    C3 (PRP pool, Sec. 5.1): own and peer rollouts of the 16-candidate pool, V = 128,256, ragged peer lengths,
+        pooled advantages, stop-gradient density weights on peer rows.
+    C4 (XGRPO + SGT, Sec. 5.2-5.3): the learner's own rollouts with the pooled cross-policy baseline plus the peer
+        rollouts the rescue gate selected, which carry only the NLL weight; MRL_FLAG_SKIP_ZERO_ROWS on (rows of
+        zero-advantage groups are not read).
+    Slab generation and the behaviour trace are input preparation, outside the timed region."""
+
+    def __init__(self, name: str, seed: int, device, slab_rows: int):
+        from paper_2605_07244_b200 import binding as B
+        self.B = B
+        w = synth.CONFIGS[name]
+        self.w, self.name = w, name
+        self.ratio_level = 0
+        meta = synth.make_meta(w, seed)
+        P, M, G = w.P, w.M, w.G
+        dev = device
+        self.rewards = meta.rewards.to(dev)
+        self.seq_len = meta.seq_len.to(dev)
+        # per-prompt outputs of the advantage / gate call; adv_pool gets one more slot that stays zero, so that a
+        # sequence without a policy-gradient term (a selected peer rollout of config 4) can point at it
+        self.adv_own = torch.empty(P, M, G, device=dev)
+        self.adv_ext = torch.zeros(P * M * G + 1, device=dev)
+        self.adv_pool = self.adv_ext[:P * M * G].view(P, M, G)
+        self.rescue = torch.empty(P, dtype=torch.uint8, device=dev)
+        self.pick = torch.empty(P, dtype=torch.int32, device=dev)
+        self.nllw_seq = torch.empty(P, M, G, device=dev)
+        self.n_gated_dev = torch.empty(1, dtype=torch.int32, device=dev)
+        sgt = name == "C4"
+        self.ap = B.AdvParams(B.ADV_GROUP_ZNORM, 0, 1e-6, 0.8, 0.2, B.PICK_SHORTEST if sgt else B.PICK_NONE, 0)
+        B.mrl_group_advantages(self.rewards, self.seq_len, 0, self.ap, self.adv_own, self.adv_pool, self.rescue,
+                               self.pick, self.nllw_seq, self.n_gated_dev)
+        torch.cuda.synchronize()
+        select = torch.ones(P, M, G, dtype=torch.bool)
+        n_gated = 0
+        if sgt:      # the step's batch: own rollouts and the peer rollouts the gate selected (input preparation)
+            picked = self.nllw_seq.cpu() > 0
+            n_gated = int(self.n_gated_dev.cpu())
+            select = torch.zeros(P, M, G, dtype=torch.bool)
+            select[:, 0, :] = True
+            select |= picked
+        batch = synth.make_batch(meta, select)
+        self.step_rows, self.step_seqs = batch.N, batch.S
+        s1 = 1
+        while s1 < batch.S and int(batch.cu_seqlens[s1 + 1]) <= slab_rows:
+            s1 += 1
+        n = int(batch.cu_seqlens[s1])
+        self.N, self.V, self.S = n, w.V, s1
+        self.z = torch.empty(n, w.V, dtype=w.dtype, device=dev)
+        for a in range(0, n, 4096):
+            e = min(n, a + 4096)
+            self.z[a:e] = batch.logits_rows(a, e, device=dev)
+        self.dz = torch.empty_like(self.z)
+        self.ids = batch.ids[:n].to(dev)
+        self.cu = batch.cu_seqlens[:s1 + 1].to(dev)
+        flat = (batch.seq_p.long() * M + batch.seq_m.long()) * G + batch.seq_g.long()
+        lens = (batch.cu_seqlens[1:] - batch.cu_seqlens[:-1]).long()
+        self.tok_weight = self.nll_weight = None
+        if sgt:      # selected peer rollouts: no policy-gradient term (the zero slot), NLL weight 1 on their rows
+            peer = batch.seq_m != 0
+            flat = torch.where(peer, torch.full_like(flat, P * M * G), flat)
+            self.nll_weight = torch.repeat_interleave(peer.float(), lens)[:n].to(dev)
+            self.peer_rows = int(self.nll_weight.sum())
+        else:
+            self.tok_weight = batch.tok_weight[:n].to(dev)
+        self.adv_index = flat[:s1].to(dev)
+        self.adv_seq = torch.empty(s1, device=dev)
+        self.logp = torch.empty(n, device=dev)
+        self.loss = torch.zeros(2, device=dev)
+        self.stats = torch.zeros(4, dtype=torch.int64, device=dev)
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.ws = torch.empty(B.workspace_bytes(B.WS_POLICY_LOSS, n, w.V, 0, B.BF16, s1), dtype=torch.uint8, device=dev)
+        flags = B.FLAG_SKIP_ZERO_ROWS if sgt else 0
+        nll_coeff = 0.1 / n_gated if n_gated > 0 else 0.0        # lambda_SGT / n_gated (Eq. (2))
+        self.lp = B.LossParams(0.2, 0.2, B.AGG_TOKEN_MEAN, flags, float(batch.N), float(batch.S), nll_coeff, 0)
+        B.mrl_token_logprobs(self.z, self.ids, None, self.logp)
+        self.logp_old = self.logp + batch.noise[:n].to(dev)
+        torch.cuda.synchronize()
+        self.kernels_per_step = 5        # adv_prompt, seq_count, row_coef, row_stream, row_terms (+ one torch gather)
+        self.dominant_per_step = 1
+        self.n_gated = n_gated
+
+    def step(self):
+        B = self.B
+        B.mrl_group_advantages(self.rewards, self.seq_len, 0, self.ap, self.adv_own, self.adv_pool, self.rescue,
+                               self.pick, self.nllw_seq, self.n_gated_dev)
+        # the slab's sequences pick their advantage out of the [P, M, G] array (one small gather between the two calls)
+        torch.index_select(self.adv_ext, 0, self.adv_index, out=self.adv_seq)
+        B.mrl_policy_loss_fwd_bwd(self.z, self.ids, None, self.cu, self.adv_seq, self.logp_old, self.tok_weight,
+                                  self.nll_weight, self.lp, self.dz, self.logp, self.loss, self.stats, self.status,
+                                  self.ws)
+
+    def tokens(self):
+        return self.N
+
+    def describe(self):
+        what = {"C3": "PRP pool (Sec. 5.1): own + peer rollouts of the 16-candidate pool, ragged peer lengths, pooled "
+                      "advantages, per-token density weights on peer rows",
+                "C4": "XGRPO + SGT (Sec. 5.2-5.3): own rollouts with the pooled baseline, rescue-selected peer rollouts "
+                      "with NLL weight 1, MRL_FLAG_SKIP_ZERO_ROWS"}[self.name]
+        d = {"workload": f"{self.w.name}: one slab of {self.S} whole sequences ({self.N} rows, "
+                         f"{self.z.numel() * 2 / 1e9:.1f} GB of bf16 logits) of a step of {self.step_rows} rows / "
+                         f"{self.step_seqs} sequences; {what}",
+             "rows": self.N, "sequences": self.S, "V": self.V, "logits_dtype": "bf16", "step_rows": self.step_rows,
+             "l2": "the slab exceeds the 126 MB L2 by two orders of magnitude; no flush needed"}
+        if self.name == "C4":
+            d.update(selected_peer_rollouts_in_step=self.n_gated, nll_rows_in_slab=self.peer_rows)
+        return d
+
+    def roofline(self, kernel_ms, peaks):
+        k_avg_ms = sum(kernel_ms) / len(kernel_ms)
+        streamed = int(self.stats.cpu()[2])
+        row_bytes = self.V * self.z.element_size()
+        alg_bytes = streamed * 2 * row_bytes + (self.N - streamed) * row_bytes      # unread rows are still zero-filled
+        achieved = alg_bytes / (k_avg_ms * 1e-3) / 1e9
+        return {"bound": "hbm", "kernel": getattr(self, "last_kernel", ""), "achieved": achieved, "peak": peaks["hbm_gbs"],
+                "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "frac_nominal": achieved / NOMINAL_HBM_GBS,
+                "peak_source": peaks["source"] + " (copy, burst)", "algorithmic_bytes_per_launch": alg_bytes,
+                "rows_read": streamed, "kernel_ms": k_avg_ms, "traffic": None}
 
 
 class LmheadWorkload:
@@ -482,11 +618,16 @@ class LmheadWorkload:
         per_step_ms = sum(kernel_ms) / (len(kernel_ms) / self.dominant_per_step)
         achieved = self.flops_executed / (per_step_ms * 1e-3) / 1e12
         peak = peaks["bf16_tflops_sustained"]
+        alg = self.flops_algorithmic / (per_step_ms * 1e-3) / 1e12
         return {"bound": "tensor", "kernel": "lmhead_gemm_kernel (forward, dZ recompute, dHidden, dW launches)",
                 "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                 "peak_source": peaks["source"] + " (cuBLAS bf16, sustained)",
+                # the same rate against the other denominators: the burst cuBLAS rate and the data-sheet dense peak;
+                # and the rate on algorithmic flops (the dZ recompute not counted) against all three
+                "frac_burst": achieved / peaks["bf16_tflops"], "frac_nominal": achieved / NOMINAL_BF16_TFLOPS,
                 "flops_per_step_executed": self.flops_executed, "flops_per_step_algorithmic": self.flops_algorithmic,
-                "achieved_algorithmic": self.flops_algorithmic / (per_step_ms * 1e-3) / 1e12,
+                "achieved_algorithmic": alg, "frac_algorithmic": alg / peak,
+                "frac_algorithmic_burst": alg / peaks["bf16_tflops"], "frac_algorithmic_nominal": alg / NOMINAL_BF16_TFLOPS,
                 "kernel_ms": per_step_ms, "launches_per_step": self.dominant_per_step, "traffic": None}
 
     def e2e_setup(self):
@@ -513,10 +654,10 @@ class LmheadWorkload:
         self.h_logp.copy_(self.logp, non_blocking=True)
         self.h_loss.copy_(self.loss, non_blocking=True)
 
-    def time_oracle(self):
+    def time_oracle(self, scale=1):
         from oracle import mrl_oracle as O
         b = self.batch
-        n_seq = max(1, LMHEAD_ORACLE_ROWS // int(b.cu_seqlens[1]))
+        n_seq = max(1, LMHEAD_ORACLE_ROWS // scale // int(b.cu_seqlens[1]))
         n = int(b.cu_seqlens[n_seq])
         adv, _ = O.group_advantages(self.meta.rewards)
         adv_seq = adv[b.seq_p.long(), b.seq_m.long(), b.seq_g.long()][:n_seq]
@@ -603,6 +744,7 @@ def measure_float32_rows(seed, peaks):
             "logits_dtype": "f32", "status": int(status.cpu()),
             "roofline": {"bound": "hbm", "kernel": "row_stream_kernel (float32, row split over two CTAs)", "achieved": gbs,
                          "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+                         "frac_nominal": gbs / NOMINAL_HBM_GBS,
                          "peak_source": peaks["source"] + " (copy, burst)", "algorithmic_bytes_per_launch": alg,
                          "traffic": None}}
 
@@ -734,7 +876,7 @@ def run_e2e(args, wl, world):
             "logp and loss"}
 
 
-def measure(wl, steps, warmup, world, local_rank, rank, peaks, with_e2e, with_cpu, args):
+def measure(wl, steps, warmup, world, local_rank, rank, peaks, with_e2e, with_cpu, args, single_thread=True):
     """Warm up, time `steps` steps with CUDA events (max over ranks), and build the result fields."""
     B = wl.B
     for _ in range(max(warmup, 3)):
@@ -753,6 +895,7 @@ def measure(wl, steps, warmup, world, local_rank, rank, peaks, with_e2e, with_cp
     barrier(world)
     local_ms = ev0.elapsed_time(ev1)
     kernel_ms = timer.elapsed_ms(steps * wl.dominant_per_step)
+    wl.last_kernel = timer.last_kernel
     status = int(wl.status.cpu())
     if status != 0:
         raise SystemExit(f"device status word is {status} after the timed region")
@@ -762,7 +905,7 @@ def measure(wl, steps, warmup, world, local_rank, rank, peaks, with_e2e, with_cp
            "gpu_launches": wl.kernels_per_step * steps, "roofline": wl.roofline(kernel_ms, peaks)}
     # end to end: pinned host buffers -> device -> kernels -> pinned host buffers
     out["e2e"] = run_e2e(args, wl, world) if with_e2e else None
-    if world == 1 and hasattr(wl, "measure_skip_zero_rows") and wl.ratio_level == 0 and not wl.lp.logp_ref:
+    if world == 1 and with_e2e and hasattr(wl, "measure_skip_zero_rows") and wl.ratio_level == 0 and not wl.lp.logp_ref:
         out["skip_zero_rows"] = wl.measure_skip_zero_rows()
         out["token_logprobs"] = wl.measure_forward_only(peaks)
     out["cpu_baseline"] = None
@@ -770,6 +913,17 @@ def measure(wl, steps, warmup, world, local_rank, rank, peaks, with_e2e, with_cp
         n, dt, sample = wl.time_oracle()
         out["cpu_baseline"] = {"value": n / dt, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
                                "sample": sample}
+        if not single_thread:
+            return out
+        # the same oracle on one thread, on a sample an eighth the size
+        threads = torch.get_num_threads()
+        torch.set_num_threads(1)
+        try:
+            n1, dt1, sample1 = wl.time_oracle(scale=8)
+        finally:
+            torch.set_num_threads(threads)
+        out["cpu_baseline"]["single_thread"] = {"value": n1 / dt1, "unit": UNIT, "cores": 1, "kind": "oracle",
+                                                "sample": sample1}
     return out
 
 
@@ -784,34 +938,53 @@ def run_ours(args, rank, world, local_rank):
     from paper_2605_07244_b200 import build
     build.build()
     B.lib()
-    if args.workload not in ("C2", "C2s", "C5", "C5s", "C5b"):
-        raise SystemExit("bench.py times config 2 (logits-in; C2s is its small profiling case) and config 5 "
-                         "(fused LM head); the other configs are parity-test cases")
+    if args.workload not in ("C2", "C2s", "C5", "C5s", "C5b", "C3", "C4"):
+        raise SystemExit("bench.py times config 2 (logits-in; C2s is its small profiling case), config 5 (fused LM "
+                         "head) and one slab of config 3 or 4; configs 1 and 6 are parity-test cases")
     peaks = measured_peaks()
     lmhead_main = args.workload in ("C5", "C5s", "C5b")
+    slab_main = args.workload in ("C3", "C4")
     cls = LmheadWorkload if lmhead_main else LogitsInWorkload
-    wl = (cls(synth.CONFIGS[args.workload], args.seed + rank, device, args.pair_tiles, args.skip_zero_rows)
+    wl = (PoolSlabWorkload(args.workload, args.seed + rank, device, args.slab_rows) if slab_main else
+          cls(synth.CONFIGS[args.workload], args.seed + rank, device, args.pair_tiles, args.skip_zero_rows)
           if lmhead_main else
           cls(synth.CONFIGS[args.workload], args.seed + rank, device, 1 if args.ratio_level == "sequence" else 0,
               args.with_entropy, args.with_kl))
-    res = measure(wl, args.steps, args.warmup, world, local_rank, rank, peaks, not args.no_e2e,
-                  not args.no_cpu_baseline, args)
+    res = measure(wl, args.steps, args.warmup, world, local_rank, rank, peaks, not args.no_e2e and not slab_main,
+                  not args.no_cpu_baseline and not slab_main, args)
     del wl
     torch.cuda.empty_cache()
 
-    # the tensor-core family beside the headline: a short config-5 leg in the default run
+    # beside the headline: the shapes the paper's setup runs, one sub-object each with its own roofline and clocks
+    sub_keys = ("value", "ms_per_step", "steps", "config", "clocks", "gpu_launches", "roofline")
+    shapes = {}
+    if args.workload == "C2" and not args.no_lmhead:
+        sub_steps = min(args.steps, 20)
+        # every row with a gradient: the KL penalty of Eq. (1) on (App. A: beta = 1e-3), same batch as the headline
+        wl_kl = LogitsInWorkload(synth.CONFIGS["C2"], args.seed + rank, device, 0, False, True)
+        r = measure(wl_kl, sub_steps, 3, world, local_rank, rank, peaks, False, False, args)
+        shapes["all_rows_live"] = {"metric": METRIC, "unit": UNIT, **{k: r[k] for k in sub_keys}}
+        del wl_kl
+        torch.cuda.empty_cache()
+        for key, name in (("prp_pool_slab", "C3"), ("xgrpo_sgt_slab", "C4")):
+            wls = PoolSlabWorkload(name, args.seed + rank, device, args.slab_rows)
+            r = measure(wls, sub_steps, 3, world, local_rank, rank, peaks, False, False, args)
+            shapes[key] = {"metric": METRIC, "unit": UNIT, **{k: r[k] for k in sub_keys}}
+            del wls
+            torch.cuda.empty_cache()
+
+    # the tensor-core family: a short config-5 leg in the default run
     lmhead = None
     if args.workload == "C2" and not args.no_lmhead:
         wl5 = LmheadWorkload(synth.CONFIGS["C5"], args.seed + rank, device)
         r5 = measure(wl5, min(args.steps, LMHEAD_SUB_STEPS), 3, world, local_rank, rank, peaks, False,
-                     not args.no_cpu_baseline, args)
-        lmhead = {"metric": METRIC, "unit": UNIT, **{k: r5[k] for k in ("value", "ms_per_step", "steps", "config",
-                                                                         "gpu_launches", "roofline", "cpu_baseline")}}
+                     not args.no_cpu_baseline, args, single_thread=False)
+        lmhead = {"metric": METRIC, "unit": UNIT, **{k: r5[k] for k in sub_keys + ("cpu_baseline",)}}
         del wl5
         # the same shape with success rates drawn per prompt (many all-success / all-failure groups), zero rows skipped
         wl5b = LmheadWorkload(synth.CONFIGS["C5b"], args.seed + rank, device, False, True)
         r5b = measure(wl5b, min(args.steps, LMHEAD_SUB_STEPS), 3, world, local_rank, rank, peaks, False, False, args)
-        lmhead["skip_zero_rows"] = {k: r5b[k] for k in ("value", "ms_per_step", "steps", "config", "roofline")}
+        lmhead["skip_zero_rows"] = {k: r5b[k] for k in ("value", "ms_per_step", "steps", "config", "clocks", "roofline")}
         del wl5b
 
     thl = tiny = f32 = None
@@ -831,6 +1004,7 @@ def run_ours(args, rank, world, local_rank):
         if res.get("skip_zero_rows") is not None:
             line["skip_zero_rows"] = res["skip_zero_rows"]
             line["token_logprobs"] = res["token_logprobs"]
+        line.update(shapes)
         if lmhead is not None:
             line["lmhead"] = lmhead
         if thl is not None:
@@ -863,7 +1037,10 @@ def main():
                     help="fused LM-head workloads: MRL_FLAG_SKIP_ZERO_ROWS (zero-multiplier rows are not produced)")
     ap.add_argument("--pair-tiles", action="store_true",
                     help="fused LM-head workloads: 256-row tiles worked by CTA pairs (MRL_FLAG_PAIR_TILES)")
-    ap.add_argument("--no-lmhead", action="store_true", help="skip the short config-5 leg of the default run")
+    ap.add_argument("--no-lmhead", action="store_true",
+                    help="skip the legs beside the headline (all-rows-live, config-3 / config-4 slabs, config 5, ...)")
+    ap.add_argument("--slab-rows", type=int, default=40960,
+                    help="config-3 / config-4 legs: largest slab (whole sequences) in rows; 40,960 rows are 10.5 / 12.4 GB of logits")
     args = ap.parse_args()
     if args.gpus < 1:
         raise SystemExit("bench.py: --gpus must be at least 1")

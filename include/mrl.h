@@ -408,6 +408,10 @@ int mrl_thl_word_align_logprobs(const float* src_logp, const int32_t* src_word, 
  */
 int mrl_profile_dominant_kernel(void** start_events, void** stop_events, int32_t n);
 
+/* Name of the dominant kernel launched last while events were registered (a static string; "" before the first
+ * such launch): lets a benchmark say which kernel its timings and counters belong to.  Not thread-safe. */
+const char* mrl_profile_last_kernel(void);
+
 /* Scratch bytes an entry point needs for the given sizes (0 if none).  Pure host arithmetic. */
 size_t mrl_workspace_bytes(int32_t which, int64_t N, int32_t V, int32_t H, int32_t dtype, int32_t S);
 

@@ -26,7 +26,7 @@ DEV_BAD_TOKEN_ID, DEV_TIMEOUT, DEV_BAD_WORD_MAP = 1, 2, 4
 EXPORTS = ("mrl_group_advantages", "mrl_token_logprobs", "mrl_policy_loss_fwd_bwd",
            "mrl_fused_lmhead_loss_fwd_bwd", "mrl_workspace_bytes", "mrl_status_string", "mrl_version",
            "mrl_profile_dominant_kernel", "mrl_policy_loss_fwd_bwd_static", "mrl_thl_word_align_logprobs",
-           "mrl_policy_loss_fwd_bwd_host", "mrl_host_pipeline_workspace_bytes")
+           "mrl_policy_loss_fwd_bwd_host", "mrl_host_pipeline_workspace_bytes", "mrl_profile_last_kernel")
 STATIC_MAX_ROWS, STATIC_MAX_SEQS = 65536, 65536
 ERR_STATIC_SCRATCH_TOO_SMALL = 8
 
@@ -90,6 +90,8 @@ def lib() -> C.CDLL:
         L.mrl_status_string.restype = C.c_char_p
         L.mrl_profile_dominant_kernel.argtypes = [C.POINTER(vp), C.POINTER(vp), i32]
         L.mrl_profile_dominant_kernel.restype = C.c_int
+        L.mrl_profile_last_kernel.argtypes = []
+        L.mrl_profile_last_kernel.restype = C.c_char_p
         L.mrl_version.argtypes = []
         L.mrl_version.restype = C.c_int
         _lib = L
@@ -252,6 +254,7 @@ class DominantKernelTimer:
         return self
 
     def __exit__(self, *exc):
+        self.last_kernel = lib().mrl_profile_last_kernel().decode()
         lib().mrl_profile_dominant_kernel(None, None, 0)
 
     def elapsed_ms(self, count: int):

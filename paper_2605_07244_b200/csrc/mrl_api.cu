@@ -44,7 +44,10 @@ void** g_prof_start = nullptr;
 void** g_prof_stop = nullptr;
 int g_prof_n = 0;
 long long g_prof_i = 0;
+const char* g_prof_last = "";
 }  // namespace
+
+extern "C" const char* mrl_profile_last_kernel(void) { return g_prof_last; }
 
 extern "C" int mrl_profile_dominant_kernel(void** start_events, void** stop_events, int32_t n) {
   if (n < 0) return MRL_ERR_INVALID_ARG;
@@ -60,7 +63,8 @@ extern "C" int mrl_profile_dominant_kernel(void** start_events, void** stop_even
   return MRL_OK;
 }
 
-void mrl_profile_before(cudaStream_t st) {
+void mrl_profile_before(cudaStream_t st, const char* kernel_name) {
+  if (g_prof_n > 0) g_prof_last = kernel_name;
   if (g_prof_n > 0) cudaEventRecord(static_cast<cudaEvent_t>(g_prof_start[g_prof_i % g_prof_n]), st);
 }
 

@@ -81,7 +81,7 @@ static inline bool mrl_kl_args_ok(const mrl_loss_params* lp) {
 }
 
 // Benchmark instrumentation (mrl_profile_dominant_kernel): event pairs recorded around dominant kernels.
-void mrl_profile_before(cudaStream_t st);
+void mrl_profile_before(cudaStream_t st, const char* kernel_name);  // a static string naming the launch
 void mrl_profile_after(cudaStream_t st);
 
 namespace mrl {

@@ -839,13 +839,13 @@ int launch_gemm(const void* A, long long lda, const void* B, long long ldb, Gemm
   if (kC == 2) {
     const long long units = tiles < pairs ? tiles : pairs;
     cfg.gridDim = dim3((unsigned)(2 * units));
-    mrl_profile_before(st);
+    mrl_profile_before(st, "lmhead_gemm_kernel (pair tiles)");
     const cudaError_t e = cudaLaunchKernelEx(&cfg, lmhead_gemm_kernel<EPI, 2, kAMn, kBMn>, ta, tb, p);
     mrl_profile_after(st);
     return e == cudaSuccess ? MRL_OK : MRL_ERR_CUDA;
   }
   const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
-  mrl_profile_before(st);
+  mrl_profile_before(st, "lmhead_gemm_kernel");
   lmhead_gemm_kernel<EPI, 1, kAMn, kBMn><<<grid, kGemmThreads, GemmCfg<1>::kSmem, st>>>(ta, tb, p);
   mrl_profile_after(st);
   MRL_CUDA_OK(cudaGetLastError());

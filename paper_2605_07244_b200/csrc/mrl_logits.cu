@@ -15,8 +15,7 @@ namespace {
 
 constexpr int kThreads = 256;        // general kernel
 constexpr int kStreamThreads = 512;  // streaming kernel: two CTAs per SM
-constexpr long long kSplitRowBytes = 512 * 1024;
-constexpr long long kResidentMinBytes = 64 * 1024;  // shorter rows stay with the streaming kernel (whole row in registers)  // rows at least this long are split over a cluster of two CTAs
+constexpr long long kSplitRowBytes = 512 * 1024;  // rows at least this long are split over a cluster of two CTAs
 // Shared memory per CTA that holds the oldest vectors of its row between the passes.  More is not better: the
 // carve-out comes out of L1, and L1 is what keeps this kernel's loads in flight (measured on B200, ms per step on
 // 34 k rows of 304 KB, half / all of them with a gradient: 0 KB 3.40 / 3.88, 32 KB 3.35 / 3.82, 48 KB 3.35 / 3.79,
@@ -509,337 +508,6 @@ __global__ void __launch_bounds__(kT, 1024 / kT) row_stream_kernel(const RowPara
 }
 
 // ------------------------------------------------------------------------------------------------
-// Resident kernel (bf16 gradient launches, 32-byte aligned rows of up to kC * kResPartMaxBytes): the row stays on the
-// SMs between the passes, so nothing depends on what L2 keeps.  kC CTAs of 512 threads (a cluster when kC = 2, two
-// CTAs per SM) take 1 / kC of a row each.  Of its part a CTA loads the first 64 KB into registers (four 256-bit
-// vectors per thread) and has the rest fetched into shared memory by bulk asynchronous copies (cp.async.bulk, no
-// multicast), everything requested before the first byte is needed.  Pass 1 replaces every logit, in place, by its
-// exponential relative to a per-thread maximum (one for the register part, one for the shared-memory part; bf16, like
-// the logit it replaces) while summing the float32 values; the halves' (max, sum, target) triples cross through
-// distributed shared memory; pass 2 multiplies the cached exponentials by g 2^(m - lse2) and stores.  One ex2 per
-// logit instead of two, and no second read of the row from anywhere off the SM.
-// ------------------------------------------------------------------------------------------------
-constexpr int kResThreads = 512;
-constexpr int kResVecs = 4;                                   // 256-bit vectors per thread kept in registers
-constexpr int kResRegBytes = kResThreads * kResVecs * 32;      // 64 KB of a CTA's part live in registers
-constexpr int kResTailMaxBytes = 88 * 1024;                   // and up to 88 KB in shared memory
-constexpr int kResPartMaxBytes = kResRegBytes + kResTailMaxBytes;
-constexpr int kResBulkBytes = 32 * 1024;                      // size of one bulk copy
-constexpr uint32_t kBulkSpinLimit = 1u << 22;
-
-__device__ __forceinline__ bool mbar_try_wait_cta(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ StreamVec<4> lds_v4(uint32_t a) {
-  StreamVec<4> t;
-  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(t.w[0]), "=r"(t.w[1]), "=r"(t.w[2]), "=r"(t.w[3]) : "r"(a));
-  return t;
-}
-
-template <int kC, bool kEnt>
-__global__ void __launch_bounds__(kResThreads, 2) row_resident_kernel(const RowParams p) {
-  constexpr int kT = kResThreads, kWarpsT = kT / 32;
-  using Vec = StreamVec<8>;
-  __shared__ float red[3 * 32];
-  __shared__ float fin[4];
-  __shared__ __align__(16) float4 xchg[2];
-  __shared__ __align__(8) uint64_t xbar;
-  __shared__ __align__(8) uint64_t bulk_bar;
-  extern __shared__ __align__(128) unsigned char tail[];  // this CTA's part beyond its first kResRegBytes bytes
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const long long row = blockIdx.x / kC;
-  const int rank = blockIdx.x % kC;  // rank in the 1-D cluster
-  const int row_nvec = p.V / 16;     // 256-bit vectors of the row
-  const int part_nvec = (row_nvec + kC - 1) / kC;
-  const int part_off = rank * part_nvec * 16;  // first element of this CTA's part
-  const int my_nvec = max(0, min(row_nvec - rank * part_nvec, part_nvec));
-  const int part_bytes = my_nvec * 32;
-  const int reg_bytes = min(part_bytes, kResRegBytes);
-  const int nvec = reg_bytes / 32;                // vectors of the register part
-  const int tail_bytes = part_bytes - reg_bytes;  // multiple of 32
-  const int nunit = tail_bytes / 16;              // 16-byte units of the shared-memory part
-  const __nv_bfloat16* grow = static_cast<const __nv_bfloat16*>(p.logits) + row * p.ld + part_off;
-  __nv_bfloat16* orow = static_cast<__nv_bfloat16*>(p.dlogits) + row * p.ld_out + part_off;
-  char* out = reinterpret_cast<char*>(orow) + (size_t)tid * 32;
-
-  // (only the validity and the id stay live over the passes; the thread that finishes the row loads the rest again)
-  bool row_valid;
-  int row_id;
-  {
-    const RowCtx ctx = load_row_ctx(p, row);
-    row_valid = ctx.valid;
-    row_id = ctx.id;
-    if (ctx.dead) {
-      for (int i = tid; i < my_nvec; i += kT) stream_st<8>(out + (size_t)(i - tid) * 32, stream_fill<8>(0u));
-      if (rank == 0 && tid == 0) {
-        write_row_scalars(p, row, ctx, 0.f, 0.f, mrl::lse2_empty(), 0.f, false, false);
-        if (kEnt) p.entropy[row] = 0.f;
-      }
-      return;  // both CTAs of a cluster take this branch: no cluster barrier is left waiting
-    }
-  }
-  // ---- request the whole part: the tail by bulk copies, the head by register loads
-  const uint32_t tail_base = smem_u32(tail), bar = smem_u32(&bulk_bar);
-  if (tid == 0) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar) : "memory");
-    if (kC > 1) asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&xbar)), "r"(kC - 1) : "memory");
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    if (tail_bytes > 0) {
-      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"((uint32_t)tail_bytes) : "memory");
-      const char* src = reinterpret_cast<const char*>(grow) + reg_bytes;
-      for (int o = 0; o < tail_bytes; o += kResBulkBytes) {
-        const uint32_t bytes = (uint32_t)min(kResBulkBytes, tail_bytes - o);
-        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                         tail_base + (uint32_t)o),
-                     "l"(src + o), "r"(bytes), "r"(bar)
-                     : "memory");
-      }
-    }
-  }
-  const char* in = reinterpret_cast<const char*>(grow) + (size_t)tid * 32;
-  Vec v[kResVecs];
-#pragma unroll
-  for (int c = 0; c < kResVecs; ++c)
-    v[c] = (c * kT + tid < nvec) ? stream_ld<8, kHintLast>(in + (size_t)c * kT * 32) : stream_fill<8>(0xff80ff80u);
-  const int rel = row_id - part_off;  // target column relative to this part
-  const bool owner = row_valid && rel >= 0 && rel < my_nvec * 16;
-  float zt = 0.f;
-  if (tid == 0 && owner) zt = __bfloat162float(grow[rel]);  // before anything is written in place
-  __syncthreads();  // the barriers are initialised for everyone
-  // "my exchange barrier exists": the peer waits for this just before its remote store
-  if (kC > 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-
-  // ---- pass 1: maximum, then exponentials in place and their float32 sum -- register part, then shared-memory part
-  float M = -INFINITY, S = 0.f, U = 0.f;  // thread totals: max, sum of 2^(x - M), (entropy) sum of 2^(x - M) z
-  float m_reg, m_tail = -INFINITY;
-  {
-    uint32_t mx = 0xff80ff80u;
-#pragma unroll
-    for (int c = 0; c < kResVecs; ++c) {
-#pragma unroll
-      for (int j = 0; j < 8; ++j) mx = hmax2_u32(mx, v[c].w[j]);
-    }
-    m_reg = fmaxf(mrl::bf16lo_to_f32(mx), mrl::bf16hi_to_f32(mx)) * MRL_LOG2E;
-    if (m_reg != -INFINITY) {
-      const float neg_m = -m_reg;
-      float s0 = 0.f, s1 = 0.f, u0 = 0.f, u1 = 0.f;
-#pragma unroll
-      for (int c = 0; c < kResVecs; ++c) {
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const float zlo = mrl::bf16lo_to_f32(v[c].w[j]), zhi = mrl::bf16hi_to_f32(v[c].w[j]);
-          const float a = mrl::ex2_approx(fmaf(zlo, MRL_LOG2E, neg_m)), e = mrl::ex2_approx(fmaf(zhi, MRL_LOG2E, neg_m));
-          s0 += a;
-          s1 += e;
-          if (kEnt) {  // a = 0 exactly where z = -inf: keep 0 * inf out of the sum
-            u0 = a != 0.f ? fmaf(a, zlo, u0) : u0;
-            u1 = e != 0.f ? fmaf(e, zhi, u1) : u1;
-          }
-          v[c].w[j] = mrl::pack_bf16x2(a, e);
-        }
-      }
-      M = m_reg;
-      S = s0 + s1;
-      if (kEnt) U = u0 + u1;
-    }
-  }
-  // (a part that is all -inf keeps its logits: pass 2 writes zeros for it instead of scaling)
-  bool ok = true;
-  if (tail_bytes > 0) {
-    bool got = false;
-    for (uint32_t i = 0; i < kBulkSpinLimit && !got; ++i) got = mbar_try_wait_cta(bar, 0);
-    ok = got;
-    if (got) {
-      uint32_t mx = 0xff80ff80u;
-      for (int u = tid; u < nunit; u += kT) {
-        const StreamVec<4> t = lds_v4(tail_base + (uint32_t)u * 16u);
-#pragma unroll
-        for (int k = 0; k < 4; ++k) mx = hmax2_u32(mx, t.w[k]);
-      }
-      m_tail = fmaxf(mrl::bf16lo_to_f32(mx), mrl::bf16hi_to_f32(mx)) * MRL_LOG2E;
-      if (m_tail != -INFINITY) {
-        const float neg_m = -m_tail;
-        float s0 = 0.f, s1 = 0.f, u0 = 0.f, u1 = 0.f;
-#pragma unroll 2
-        for (int u = tid; u < nunit; u += kT) {
-          StreamVec<4> t = lds_v4(tail_base + (uint32_t)u * 16u);
-#pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            const float zlo = mrl::bf16lo_to_f32(t.w[k]), zhi = mrl::bf16hi_to_f32(t.w[k]);
-            const float a = mrl::ex2_approx(fmaf(zlo, MRL_LOG2E, neg_m)), e = mrl::ex2_approx(fmaf(zhi, MRL_LOG2E, neg_m));
-            s0 += a;
-            s1 += e;
-            if (kEnt) {
-              u0 = a != 0.f ? fmaf(a, zlo, u0) : u0;
-              u1 = e != 0.f ? fmaf(e, zhi, u1) : u1;
-            }
-            t.w[k] = mrl::pack_bf16x2(a, e);
-          }
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(tail_base + (uint32_t)u * 16u), "r"(t.w[0]),
-                       "r"(t.w[1]), "r"(t.w[2]), "r"(t.w[3])
-                       : "memory");
-        }
-        // merge the two parts of the thread (fixed order)
-        const float Mn = fmaxf(M, m_tail);
-        const float fo = M != -INFINITY ? mrl::ex2_approx(M - Mn) : 0.f, fn = mrl::ex2_approx(m_tail - Mn);
-        S = S * fo + (s0 + s1) * fn;
-        if (kEnt) U = U * fo + (u0 + u1) * fn;
-        M = Mn;
-      }
-    }
-  }
-  // ---- block totals: maximum first, one rescale, then a plain sum (fixed order: reproducible)
-  float m = M;
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-  const float rescale = M != -INFINITY ? mrl::ex2_approx(M - m) : 0.f;
-  float sum = S * rescale, usum = kEnt ? U * rescale : 0.f;
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    sum += __shfl_xor_sync(0xffffffffu, sum, o);
-    if (kEnt) usum += __shfl_xor_sync(0xffffffffu, usum, o);
-  }
-  if (lane == 0) {
-    red[warp] = m;
-    red[32 + warp] = sum;
-    if (kEnt) red[64 + warp] = usum;
-  }
-  // (a bulk copy that did not land within the limit: only thread-local `ok` differs; the finishing thread needs the
-  // block's verdict, and nobody may leave while a copy into this CTA's shared memory can still be in flight)
-  const bool copies_ok = __syncthreads_and(ok);
-  if (warp == 0) {
-    const float wm = lane < kWarpsT ? red[lane] : -INFINITY, ws = lane < kWarpsT ? red[32 + lane] : 0.f;
-    float tm = wm;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) tm = fmaxf(tm, __shfl_xor_sync(0xffffffffu, tm, o));
-    const float wscale = wm != -INFINITY ? mrl::ex2_approx(wm - tm) : 0.f;
-    float ts = ws * wscale, tu = (kEnt && lane < kWarpsT) ? red[64 + lane] * wscale : 0.f;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      ts += __shfl_xor_sync(0xffffffffu, ts, o);
-      if (kEnt) tu += __shfl_xor_sync(0xffffffffu, tu, o);
-    }
-    bool good = copies_ok;
-    if (kC > 1) {
-      asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");  // the peer's barrier is initialised
-      if (lane == 0) {
-        // a CTA whose copy timed out still sends its (meaningless) triple, flagged, so that the peer is not left waiting
-        const float flag = !copies_ok ? -1.f : (owner ? 1.f : 0.f);
-        xchg[rank] = make_float4(tm, ts, zt, flag);
-        const uint32_t peer = (uint32_t)(rank ^ 1);
-        const uint32_t dst = mapa_u32(smem_u32(&xchg[rank]), peer);
-        asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(tm), "f"(ts), "f"(zt), "f"(flag)
-                     : "memory");
-        asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(mapa_u32(smem_u32(&xbar), peer))
-                     : "memory");
-        bool got = false;
-        for (uint32_t i = 0; i < kExchangeSpinLimit && !got; ++i) got = mbar_try_wait_cluster(&xbar, 0);
-        good = good && got;
-        if (got) {  // rank order, so both CTAs form the same sums
-          const float4 a = xchg[0], b = xchg[1];
-          if (a.w < 0.f || b.w < 0.f) good = false;
-          tm = fmaxf(a.x, b.x);
-          ts = (a.x != -INFINITY ? a.y * mrl::ex2_approx(a.x - tm) : 0.f) +
-               (b.x != -INFINITY ? b.y * mrl::ex2_approx(b.x - tm) : 0.f);
-          zt = a.w > 0.f ? a.z : (b.w > 0.f ? b.z : 0.f);
-        }
-      }
-    }
-    if (lane == 0) {
-      if (!good && p.status != nullptr) atomicOr(p.status, MRL_DEV_TIMEOUT);
-      const RowCtx ctx = load_row_ctx(p, row);
-      const float lse2 = tm + log2f(ts);
-      const float lse = lse2 * MRL_LN2;
-      float logp = 0.f, g = 0.f;
-      bool clipped = false;
-      if (ctx.valid && good) {
-        logp = zt - lse;
-        if (p.loss_mode) {
-          const mrl::RowOut ro = mrl::mrl_row_loss(logp, ctx.in, p.eps_lo, p.eps_hi);
-          g = ro.g;
-          clipped = ro.clipped;
-        }
-      }
-      if (rank == 0 && good) write_row_scalars(p, row, ctx, logp, ctx.valid ? lse : 0.f, mrl::Lse2{tm, ts}, zt, clipped, true);
-      if (kEnt && kC == 1) p.entropy[row] = ctx.valid ? lse - tu / ts : 0.f;  // H = lse - sum_v p_v z_v
-      fin[0] = lse2;
-      fin[1] = g;
-      fin[2] = g * (mrl::ex2_approx(fmaf(zt, MRL_LOG2E, -lse2)) - 1.0f);
-      fin[3] = good ? 1.f : 0.f;
-    }
-  } else if (kC > 1) {
-    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");  // pairs with the arrive above
-  }
-  __syncthreads();
-  // Neither CTA of a pair may leave while its peer can still write into its shared memory (the exchange's remote
-  // store and remote arrive): each CTA signals here, after its own remote accesses were issued, and waits for the
-  // peer's signal just before it exits.
-  if (kC > 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-  auto leave = [] {
-    if (kC > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-  };
-  if (fin[3] == 0.f) {
-    if (!copies_ok && tail_bytes > 0) {  // one more bounded wait for this CTA's own copies before its memory is given up
-      bool got = false;
-      for (uint32_t i = 0; i < kBulkSpinLimit && !got; ++i) got = mbar_try_wait_cta(bar, 0);
-    }
-    leave();
-    return;
-  }
-  const float lse2 = fin[0], g = fin[1], tfix = fin[2];
-
-  // ---- pass 2: dlogits = g 2^(m - lse2) * (cached exponential), the target column patched after
-  if (g == 0.f) {
-    for (int i = tid; i < my_nvec; i += kT) stream_st<8>(out + (size_t)(i - tid) * 32, stream_fill<8>(0u));
-    leave();
-    return;
-  }
-  const float neg_k = -(lse2 - log2f(fabsf(g)));  // 2^(m - k) = |g| 2^(m - lse2)
-  const uint32_t sign = g < 0.f ? 0x80008000u : 0u;
-  {
-    const bool none = m_reg == -INFINITY;
-    const float sc = none ? 0.f : mrl::ex2_approx(m_reg + neg_k);
-#pragma unroll
-    for (int c = 0; c < kResVecs; ++c) {
-      Vec r;
-#pragma unroll
-      for (int j = 0; j < 8; ++j)
-        r.w[j] = none ? 0u : mrl::pack_bf16x2(mrl::bf16lo_to_f32(v[c].w[j]) * sc, mrl::bf16hi_to_f32(v[c].w[j]) * sc) ^ sign;
-      if (c * kT + tid < nvec) stream_st<8>(out + (size_t)c * kT * 32, r);
-    }
-  }
-  if (tail_bytes > 0) {
-    const bool none = m_tail == -INFINITY;
-    const float sc = none ? 0.f : mrl::ex2_approx(m_tail + neg_k);
-    char* out_tail = reinterpret_cast<char*>(orow) + reg_bytes;
-#pragma unroll 2
-    for (int u = tid; u < nunit; u += kT) {
-      const StreamVec<4> t = lds_v4(tail_base + (uint32_t)u * 16u);
-      StreamVec<4> r;
-#pragma unroll
-      for (int k = 0; k < 4; ++k)
-        r.w[k] = none ? 0u : mrl::pack_bf16x2(mrl::bf16lo_to_f32(t.w[k]) * sc, mrl::bf16hi_to_f32(t.w[k]) * sc) ^ sign;
-      stream_st<4>(out_tail + (size_t)u * 16, r);
-    }
-  }
-  // the thread whose vector store covered the target column patches it (program order on one address)
-  if (owner) {
-    const int reg_elems = reg_bytes / 2;
-    const int owner_tid = rel < reg_elems ? (rel / 16) % kT : ((rel - reg_elems) / 8) % kT;
-    if (tid == owner_tid) orow[rel] = __float2bfloat16_rn(tfix);
-  }
-  leave();
-}
-
-// ------------------------------------------------------------------------------------------------
 // General kernel: one CTA per row, any dtype / V / alignment.
 // ------------------------------------------------------------------------------------------------
 
@@ -1294,48 +962,13 @@ int launch_rows(RowParams p, int dtype, cudaStream_t st) {
   const int words = pick_stream_words(p, dtype);
   const unsigned n = (unsigned)p.N;
   if (words == 0) {
-    mrl_profile_before(st);
+    mrl_profile_before(st, "row_general_kernel");
     if (dtype == MRL_BF16)
       row_general_kernel<__nv_bfloat16><<<n, kThreads, 0, st>>>(p);
     else
       row_general_kernel<float><<<n, kThreads, 0, st>>>(p);
     mrl_profile_after(st);
     return cudaGetLastError() == cudaSuccess ? MRL_OK : MRL_ERR_CUDA;
-  }
-  // bf16 gradient launches whose rows fit on one SM or a pair of them (registers + shared memory) keep the row there
-  // between the passes (the entropy diagnostic is carried by the single-CTA shape only)
-  const long long row_bytes = (long long)p.V * 2;
-  if (dtype == MRL_BF16 && words == 8 && p.dlogits != nullptr && row_bytes > kResidentMinBytes &&
-      row_bytes <= (p.entropy != nullptr ? 1 : 2) * (long long)kResPartMaxBytes && p.N <= 0x3fffffffll) {
-    const int C = row_bytes <= kResPartMaxBytes ? 1 : 2;
-    const int part_bytes = ((p.V / 16 + C - 1) / C) * 32;
-    const int tail_bytes = part_bytes > kResRegBytes ? part_bytes - kResRegBytes : 0;
-    using Kernel = void (*)(const RowParams);
-    const bool ent = p.entropy != nullptr;
-    const Kernel k = C == 2 ? row_resident_kernel<2, false> : ent ? row_resident_kernel<1, true> : row_resident_kernel<1, false>;
-    static std::atomic<uint64_t> attr_done[3];
-    const int rc = mrl_once_per_device(attr_done[C == 2 ? 0 : ent ? 1 : 2], [&] {
-      // the carve-out two CTAs per SM need at the largest tail; the rest stays L1
-      const cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kResTailMaxBytes);
-      return e != cudaSuccess ? e : cudaFuncSetAttribute(k, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
-    });
-    if (rc != MRL_OK) return rc;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(n * (unsigned)C);
-    cfg.blockDim = dim3(kResThreads);
-    cfg.dynamicSmemBytes = (size_t)tail_bytes;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = C;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    mrl_profile_before(st);
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, k, p);
-    mrl_profile_after(st);
-    return e == cudaSuccess ? MRL_OK : MRL_ERR_CUDA;
   }
   // Two CTAs per SM stream one row each, or -- for rows so long that two rows per SM would be evicted from L2
   // before the second pass reads them back -- the two halves of one row as a cluster of two.  (At 300 KB rows the
@@ -1385,7 +1018,7 @@ int launch_rows(RowParams p, int dtype, cudaStream_t st) {
     });
     if (rc != MRL_OK) return rc;
   }
-  mrl_profile_before(st);
+  mrl_profile_before(st, split ? "row_stream_kernel (row split over a CTA pair)" : "row_stream_kernel");
   const cudaError_t e = cudaLaunchKernelEx(&cfg, k, p);
   mrl_profile_after(st);
   return e == cudaSuccess ? MRL_OK : MRL_ERR_CUDA;
@@ -1454,7 +1087,7 @@ int launch_rows_backward(const RowParams& p, int dtype, const float* g, const fl
   if (p.N == 0) return MRL_OK;
   const int words = pick_stream_words(p, dtype);
   const unsigned n = (unsigned)p.N;
-  mrl_profile_before(st);
+  mrl_profile_before(st, words != 0 ? "row_backward_stream_kernel" : "row_backward_general_kernel");
   if (words == 8 && dtype == MRL_BF16)
     row_backward_stream_kernel<kStreamThreads, 4, 8, false><<<n, kStreamThreads, 0, st>>>(p, g, lse2, zt);
   else if (words == 4 && dtype == MRL_BF16)

@@ -135,7 +135,7 @@ extern "C" int mrl_thl_word_align_logprobs(const float* src_logp, const int32_t*
   float* word_sum = static_cast<float*>(workspace);
   int32_t* word_cnt = reinterpret_cast<int32_t*>(static_cast<char*>(workspace) + need / 2);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  mrl_profile_before(st);
+  mrl_profile_before(st, "thl_word_align_kernel");
   thl_word_align_kernel<<<(unsigned)B, kAlignThreads, 0, st>>>(src_logp, src_word, src_cu, tgt_word, tgt_cu, word_cu,
                                                                ignore_value, out, src_total, tgt_total, word_sum,
                                                                word_cnt, N_src, N_tgt, total_words, status);

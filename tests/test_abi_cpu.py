@@ -33,7 +33,7 @@ def test_header_declarations_are_all_exported(lib):
 
 
 def test_version_and_status_strings(lib):
-    assert B.version() == 103
+    assert B.version() == 104
     assert B.status_string(0) == "MRL_OK"
     assert B.status_string(4) == "MRL_ERR_WORKSPACE_TOO_SMALL"
     assert B.status_string(12345) == "MRL_ERR_UNKNOWN"

@@ -47,3 +47,23 @@ def test_lmhead_line_small_case():
     assert r["bound"] == "tensor" and r["unit"] == "TFLOP/s" and 0.2 < r["frac"] < 1.2
     assert d["dtype"] == "bf16" and d["gpu_launches"] > 0 and d["e2e"]["value"] > 0
     assert d["config"]["rows_worked_on"]["backward"] <= d["config"]["rows"]
+
+
+def test_single_thread_oracle_figure_and_nominal_fractions_are_reported():
+    d = run_bench("--workload", "C2s", "--steps", "3", "--warmup", "3", "--no-e2e")
+    c = d["cpu_baseline"]
+    assert c["single_thread"]["cores"] == 1 and c["single_thread"]["value"] > 0
+    r = d["roofline"]
+    assert r["kernel"].startswith("row_stream_kernel") and 0 < r["frac_nominal"] < r["frac"]
+
+
+@pytest.mark.parametrize("workload,rows", [("C3", 4200), ("C4", 3000)])
+def test_slab_legs_of_the_pool_and_gate_shapes(workload, rows):
+    """One slab of the PRP-pool shape (config 3) and of the XGRPO + SGT shape (config 4), cut small."""
+    d = run_bench("--workload", workload, "--steps", "3", "--warmup", "3", "--slab-rows", str(rows))
+    cfg, r = d["config"], d["roofline"]
+    assert cfg["rows"] <= rows and cfg["rows"] >= 1024 and cfg["step_rows"] > 500_000
+    assert r["bound"] == "hbm" and 0 < r["frac"] < 1.2 and r["rows_read"] <= cfg["rows"]
+    assert d["e2e"] is None and d["cpu_baseline"] is None       # the legs beside the headline carry neither
+    if workload == "C4":
+        assert r["rows_read"] < cfg["rows"]                      # zero-advantage groups are not read

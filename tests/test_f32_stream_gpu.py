@@ -8,7 +8,7 @@ from oracle import mrl_oracle as O
 from paper_2605_07244_b200 import binding as B
 from paper_2605_07244_b200 import build
 
-from helpers import (GRAD_REL_L2_F32, LOGP_ATOL, KlTerm, compare_policy_loss, dev, make_lp, oracle_lp, rel_l2,
+from helpers import (GRAD_REL_L2_F32, LOGP_ATOL, KlTerm, compare_policy_loss, dev, loss_close, make_lp, oracle_lp, rel_l2,
                      run_gpu_policy_loss)
 import test_seqratio_gpu as SR
 
@@ -35,7 +35,7 @@ def test_fused_pass_float32_streaming(N, V, pad, agg):
     got = run_gpu_policy_loss(z, ids, mask, cu, adv, old, tw, nllw, lp, V=V)
     ref = O.policy_loss(z[:, :V], ids, mask, cu, adv, old, tw, nllw, oracle_lp(lp))
     assert got["status"] == 0
-    compare_policy_loss(got, ref, V, F32, loss_floor=0.1 * float(ref["pg_term"].abs().sum()))
+    compare_policy_loss(got, ref, V, F32, cancelling=True)
     if pad:
         assert torch.isnan(got["dlogits"][:, V:]).all()
     # in place gives the same bits
@@ -75,4 +75,4 @@ def test_response_level_ratio_and_kl_float32_streaming(N, V, pad):
     got = run_gpu_policy_loss(z, ids, mask, cu, adv, old, None, nllw, lp, V=V)
     ref = O.policy_loss_sequence_ratio(z[:, :V], ids, mask, cu, adv, old, nllw, oracle_lp(lp), logp_ref=ref_trace)
     SR.compare(got, ref, got["dlogits"][:, :V].double(), ref["dlogits"], GRAD_REL_L2_F32)
-    assert abs(kl.value() - ref["loss_kl"]) <= 1e-5 * max(abs(ref["loss_kl"]), 0.1 * float(ref["kl_term"].abs().sum()))
+    assert loss_close(kl.value(), ref["loss_kl"])          # k3 terms share one sign: the strict form

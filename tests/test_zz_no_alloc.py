@@ -85,18 +85,16 @@ def test_static_scratch_variant_matches_the_workspace_variant_on_two_calls_in_a_
         assert float(want["dz"].float().norm()) > 0
         # nothing is allocated: after the calls above (the first one on a device looks the array's address up and may
         # load code), one more call leaves the device's free memory and the framework's own counters where they were
-        torch.cuda.synchronize()
-        free_before, _ = torch.cuda.mem_get_info()
-        held_before = torch.cuda.memory_allocated()
         z, ids, mask, cu, adv, logp_old, nllw = inp
         out = (torch.empty_like(z), torch.empty(N, device="cuda"), torch.empty(2, device="cuda"))
-        held_with_outputs = torch.cuda.memory_allocated()
-        free_with_outputs, _ = torch.cuda.mem_get_info()
-        B.mrl_policy_loss_fwd_bwd_static(z, ids, mask, cu, adv, logp_old, None, nllw, make_lp(nll_coeff=0.05), out[0], out[1],
-                                         out[2])
+        lp = make_lp(nll_coeff=0.05)
         torch.cuda.synchronize()
-        assert torch.cuda.memory_allocated() == held_with_outputs >= held_before
-        assert torch.cuda.mem_get_info()[0] == free_with_outputs <= free_before
+        held_before = torch.cuda.memory_allocated()
+        free_before, _ = torch.cuda.mem_get_info()
+        B.mrl_policy_loss_fwd_bwd_static(z, ids, mask, cu, adv, logp_old, None, nllw, lp, out[0], out[1], out[2])
+        torch.cuda.synchronize()
+        assert torch.cuda.memory_allocated() == held_before
+        assert torch.cuda.mem_get_info()[0] == free_before
         assert torch.equal(out[0].cpu().view(torch.int16), want["dz"].view(torch.int16))
 
 
