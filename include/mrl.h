@@ -24,6 +24,10 @@
  *  - `workspace` [device] is scratch of at least mrl_workspace_bytes(...) bytes, 256-byte
  *    aligned, contents unspecified before and after.  Calls that share a workspace must not
  *    overlap on the device.
+ *  - Threads.  Calls from several host threads are fine as long as they do not share a workspace, with these
+ *    exceptions, which keep per-device state inside the library and must not be called concurrently for one device:
+ *    mrl_policy_loss_fwd_bwd_host (its copy streams and events), mrl_policy_loss_fwd_bwd_static (its scratch array),
+ *    and the profiling hook (process-wide).
  *  - Row-major everywhere.  "Row t" is one response-token position: its logits row predicts
  *    ids[t] (the caller has already applied the next-token shift and dropped prompt rows).
  *  - Notation follows the paper: P prompts, M policies, G (the paper's K) rollouts per policy
@@ -247,11 +251,12 @@ int mrl_token_logprobs(const void* logits, int32_t dtype, int64_t N, int32_t V, 
  *   workspace: mrl_workspace_bytes(MRL_WS_POLICY_LOSS, N, V, 0, dtype, S)
  *
  * float32 row arithmetic on the input dtype, float64 for the final N-term sums (fixed order:
- * bitwise reproducible).  dlogits is rounded to nearest even.  The fast path (one CTA per row: the
- * row is streamed from HBM once and read a second time from L2) needs bf16, V >= 4096, and either
- * V % 16 == 0, ld % 16 == 0, ld_out % 16 == 0 with 32-byte aligned logits / dlogits, or the same
- * with 8 and 16 bytes; anything else takes a general kernel with the same results.  Rows much
- * longer than ~200,000 entries no longer fit L2 while in flight and are then read from HBM twice.
+ * bitwise reproducible from run to run for one entry point and one set of arguments; a forward-only call and a
+ * gradient call may differ in the last bits).  dlogits is rounded to nearest even.  The fast path (one CTA per row:
+ * the row is streamed from HBM once and read a second time from L2) takes bf16 or float32 rows with V >= 4096 and
+ * either 32-byte aligned logits / dlogits with V, ld, ld_out multiples of 32 bytes' worth of elements, or the same
+ * with 16 bytes; anything else takes a general kernel with the same results.  Rows of 512 KB or more are shared by
+ * two CTAs; rows much longer than 1 MB no longer fit L2 while in flight and are then read from HBM twice.
  * N = 0: loss (and stats) are zeroed unless ACCUMULATE_LOSS.
  */
 int mrl_policy_loss_fwd_bwd(const void* logits, int32_t dtype, int64_t N, int32_t V, int64_t ld,

@@ -181,7 +181,14 @@ extern "C" int mrl_policy_loss_fwd_bwd_host(const void* h_logits, int32_t dtype,
 
   // ---- the slabs: copy in | kernels in place | copy out, three buffers in rotation
   const size_t row_bytes = (size_t)ld * elem;
-  for (int k = 0; k < n_slabs; ++k) {
+  // If queueing fails half-way, what is already queued on the two copy streams is ordered before the end of the
+  // caller's stream, so that a caller who synchronises its stream after the error return has nothing left in flight.
+  auto give_up = [&](int code) {
+    if (cudaEventRecord(P.small_in, P.in) == cudaSuccess) (void)cudaStreamWaitEvent(st, P.small_in, 0);
+    if (cudaEventRecord(P.start, P.out) == cudaSuccess) (void)cudaStreamWaitEvent(st, P.start, 0);
+    return code;
+  };
+  auto queue_slab = [&](int k) -> int {
     const int b = k % kBufs, s0 = slab_first[k], s1 = slab_first[k + 1];
     const long long a = h_cu_seqlens[s0], n = (long long)h_cu_seqlens[s1] - a;
     if (k >= kBufs) MRL_CUDA_OK(cudaStreamWaitEvent(P.in, P.out_done[b], 0));  // the buffer's last gradient has left
@@ -210,6 +217,11 @@ extern "C" int mrl_policy_loss_fwd_bwd_host(const void* h_logits, int32_t dtype,
                                     (size_t)ld_out * elem, w.buf[b], row_bytes, (size_t)V * elem, (size_t)n,
                                     cudaMemcpyDeviceToHost, P.out));
     MRL_CUDA_OK(cudaEventRecord(P.out_done[b], P.out));
+    return MRL_OK;
+  };
+  for (int k = 0; k < n_slabs; ++k) {
+    rc = queue_slab(k);
+    if (rc != MRL_OK) return give_up(rc);
   }
   // ---- the caller's stream ends after the last gradients have left, then the small results follow on it
   for (int k = n_slabs > kBufs ? n_slabs - kBufs : 0; k < n_slabs; ++k)
