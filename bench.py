@@ -244,9 +244,9 @@ class LogitsInWorkload:
             self.lp.logp_ref, self.lp.kl_loss = self.logp_ref.data_ptr(), self.kl_loss.data_ptr()
             self.lp.kl_coeff, self.lp.kl_estimator = 1e-3, B.KL_K3
         torch.cuda.synchronize()
-        # adv_prompt, seq_count, row_coef, row_stream, row_terms, finalize; the response-level ratio has a forward
-        # launch, the per-response kernel and a backward launch instead of one fused row kernel
-        self.kernels_per_step = 6 if ratio_level == 0 else 7
+        # adv_prompt, seq_prepare, row_stream, row_terms (which also finalises); the response-level ratio has a forward
+        # launch, the per-response kernel, the partial sums and a backward launch instead of one fused row kernel
+        self.kernels_per_step = 4 if ratio_level == 0 else 6
         self.dominant_per_step = 1 if ratio_level == 0 else 2
         # read V + write V elements; the response-level ratio reads the row a second time from HBM
         self.bytes_per_token = (2 if ratio_level == 0 else 3) * self.V * self.z.element_size()
@@ -481,7 +481,7 @@ class PoolSlabWorkload:
         B.mrl_token_logprobs(self.z, self.ids, None, self.logp)
         self.logp_old = self.logp + batch.noise[:n].to(dev)
         torch.cuda.synchronize()
-        self.kernels_per_step = 5        # adv_prompt, seq_count, row_coef, row_stream, row_terms (+ one torch gather)
+        self.kernels_per_step = 4        # adv_prompt, seq_prepare, row_stream, row_terms (+ one torch gather)
         self.dominant_per_step = 1
         self.n_gated = n_gated
 
@@ -575,9 +575,9 @@ class LmheadWorkload:
         torch.cuda.synchronize()
         chunks = -(-self.V // 16384)
         self.dominant_per_step = 1 + 3 * chunks          # forward GEMM, then (dZ, dHidden, dW) per vocabulary chunk
-        # adv, seq_count, row_coef, forward GEMM, rows, row_terms, finalize, two live-block list builds of two kernels
-        # each (forward, backward), then 3 GEMMs per chunk
-        self.kernels_per_step = 11 + 3 * chunks
+        # adv, seq_prepare, forward GEMM, rows, row_terms, two live-block list builds of two kernels each (forward,
+        # backward), then 3 GEMMs per chunk
+        self.kernels_per_step = 9 + 3 * chunks
         # Blocks of 256 rows without any gradient are left out of the three backward products, and of the forward one
         # too under MRL_FLAG_SKIP_ZERO_ROWS: count the rows of the blocks that are worked on (a block whose rows are
         # all clipped is not expected and not counted as skipped).

@@ -50,12 +50,13 @@ struct MrlCarver {
 struct MrlLossWs {
   float *rowA, *rowcu, *rowcn;        // A_t, c_t u_t, cn_t
   float* rowck;                       // beta c_t of the KL term (0 when the term is off)
+  float* cscale;                      // [1] factor still to be applied to rowcu and rowck (1, or the token-mean 1 / D)
   float *row_m2, *row_s, *row_zt;     // base-2 running max, sum of 2^(x - max), target logit
   double *pg_term, *nll_term, *kl_term;  // per-row terms (response-level ratio only)
   double* partials;                      // [ceil(N / 256)][6] block sums of the terms and the row statistics
   uint8_t* rowstat;                   // MRL_ROW_* bits
   int32_t* seq_cnt;
-  unsigned long long* totals;
+  unsigned long long* totals;         // [0] valid tokens, [1] bad ids, [2] / [3] tickets of the last-block sums
   size_t bytes;
 };
 #define MRL_ROW_VALID 1

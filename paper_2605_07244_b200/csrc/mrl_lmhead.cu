@@ -664,6 +664,7 @@ __global__ void __launch_bounds__(256) lmhead_rows_kernel(long long N, int V, in
                                                            const float* __restrict__ rowcu,
                                                            const float* __restrict__ rowcn,
                                                            const float* __restrict__ rowck,
+                                                           const float* __restrict__ cscale,
                                                            const float* __restrict__ logp_ref, int kl_est,
                                                            const float* __restrict__ logp_old, float eps_lo,
                                                            float eps_hi, float* __restrict__ row_m2,
@@ -696,11 +697,11 @@ __global__ void __launch_bounds__(256) lmhead_rows_kernel(long long N, int V, in
     const float logp = zt[t] - l2 * MRL_LN2;
     mrl::RowIn in;
     in.A = rowA[t];
-    in.cu = rowcu[t];
+    in.cu = rowcu[t] * cscale[0];
     in.cn = rowcn[t];
     in.has_old = logp_old != nullptr;
     in.logp_old = in.has_old ? logp_old[t] : 0.f;
-    in.ck = logp_ref != nullptr ? rowck[t] : 0.f;
+    in.ck = logp_ref != nullptr ? rowck[t] * cscale[0] : 0.f;
     in.logp_ref = logp_ref != nullptr ? logp_ref[t] : 0.f;
     in.kl_est = kl_est;
     const mrl::RowOut ro = mrl::mrl_row_loss(logp, in, eps_lo, eps_hi);
@@ -1016,7 +1017,7 @@ extern "C" int mrl_fused_lmhead_loss_fwd_bwd(const void* hidden, const void* W, 
   }
   lmhead_rows_kernel<<<(unsigned)((N + 255) / 256), 256, 0, st>>>(N, V, w.n_tiles_fwd, w.partial, w.partial_u, lp->entropy,
                                                                   w.part_ld, w.zt, ids,
-                                                                  mask, rw.rowA, rw.rowcu, rw.rowcn, rw.rowck,
+                                                                  mask, rw.rowA, rw.rowcu, rw.rowcn, rw.rowck, rw.cscale,
                                                                   seq_ratio ? nullptr : lp->logp_ref, lp->kl_estimator,
                                                                   seq_ratio ? nullptr : logp_old, lp->eps_lo,
                                                                   lp->eps_hi, rw.row_m2, rw.row_s, rw.row_zt,

@@ -41,6 +41,7 @@ struct RowParams {
   const float* rowcu;
   const float* rowcn;
   const float* rowck;     // KL term: beta c_t; read only when logp_ref is given
+  const float* cscale;    // [1] common factor of rowcu and rowck (the token-mean 1 / D when it was not known up front, else 1)
   const float* logp_ref;  // nullable
   int kl_est;
   const float* logp_old;
@@ -80,13 +81,14 @@ __device__ __forceinline__ RowCtx load_row_ctx(const RowParams& p, long long row
   c.in.logp_ref = 0.f;
   c.in.kl_est = p.kl_est;
   if (p.loss_mode) {
+    const float cs = p.cscale[0];
     c.in.A = p.rowA[row];
-    c.in.cu = p.rowcu[row];
+    c.in.cu = p.rowcu[row] * cs;
     c.in.cn = p.rowcn[row];
     c.in.has_old = p.logp_old != nullptr;
     if (c.in.has_old) c.in.logp_old = p.logp_old[row];
     if (p.logp_ref != nullptr) {
-      c.in.ck = p.rowck[row];
+      c.in.ck = p.rowck[row] * cs;
       c.in.logp_ref = p.logp_ref[row];
     }
   }
@@ -669,7 +671,8 @@ __global__ void __launch_bounds__(256) seq_ratio_kernel(const int32_t* __restric
                                                          const float* __restrict__ adv_seq,
                                                          const float* __restrict__ logp_old,
                                                          const float* __restrict__ nll_weight,
-                                                         const float* __restrict__ rowck, mrl_loss_params lp,
+                                                         const float* __restrict__ rowck,
+                                                         const float* __restrict__ cscale, mrl_loss_params lp,
                                                          double* __restrict__ pg_term, double* __restrict__ nll_term,
                                                          double* __restrict__ kl_term, float* __restrict__ logp,
                                                          float* g_out, float* lse2_out) {
@@ -717,10 +720,11 @@ __global__ void __launch_bounds__(256) seq_ratio_kernel(const int32_t* __restric
       const float cn = nll_weight ? (float)cn_base * nll_weight[t] : 0.f;
       g = g_pg + cn;
       if (cn != 0.f) nl = -(double)cn * lpv;
-      if (lp.logp_ref != nullptr && rowck[t] != 0.f) {  // the KL term stays per token (App. A)
+      const float ck = lp.logp_ref != nullptr ? rowck[t] * cscale[0] : 0.f;
+      if (ck != 0.f) {  // the KL term stays per token (App. A)
         const double d = lpv - (double)lp.logp_ref[t];
-        kl = (double)rowck[t] * mrl::kl_value(d, lp.kl_estimator);
-        g -= rowck[t] * mrl::kl_slope((float)d, lp.kl_estimator);
+        kl = (double)ck * mrl::kl_value(d, lp.kl_estimator);
+        g -= ck * mrl::kl_slope((float)d, lp.kl_estimator);
       }
       if (clipped) rowstat[t] = st | kStatClipped;
     }
@@ -736,12 +740,23 @@ __global__ void __launch_bounds__(256) seq_ratio_kernel(const int32_t* __restric
 // ------------------------------------------------------------------------------------------------
 // Per-sequence bookkeeping around the row kernel.
 // ------------------------------------------------------------------------------------------------
-// valid-token count of each sequence, the total, and bad-id detection
-__global__ void __launch_bounds__(128) seq_count_kernel(const int32_t* __restrict__ cu, int S, long long N, int V,
-                                                         const int32_t* __restrict__ ids,
-                                                         const uint8_t* __restrict__ mask, int32_t* seq_cnt,
-                                                         unsigned long long* totals, int32_t* status) {
+// One block per sequence: its valid-token count (and bad-id detection), then A_t, c_t u_t, cn_t and beta c_t of its
+// rows (Eq. (1) aggregation and regulariser, Eq. (2) per-token average).  When the token-mean denominator is the valid
+// tokens of this very call, it is only known once every block has counted: the rows then get u_t and beta, and the
+// common factor 1 / D is published in cscale[0] by the block that finishes last; consumers multiply by cscale[0],
+// which is exactly 1 in every other case (the products are the same floats either way).  Rows that no sequence
+// covers (before cu[0], after cu[S]) get zero coefficients from the first and the last block.
+__global__ void __launch_bounds__(128) seq_prepare_kernel(const int32_t* __restrict__ cu, int S, long long N, int V,
+                                                           const int32_t* __restrict__ ids,
+                                                           const uint8_t* __restrict__ mask,
+                                                           const float* __restrict__ adv_seq,
+                                                           const float* __restrict__ tok_weight,
+                                                           const float* __restrict__ nll_weight, mrl_loss_params lp,
+                                                           int32_t* seq_cnt, unsigned long long* totals, float* cscale,
+                                                           float* rowA, float* rowcu, float* rowcn, float* rowck,
+                                                           int32_t* status) {
   __shared__ int red[2][4];
+  __shared__ int len_sh;
   const int s = blockIdx.x;
   const long long a = max(0ll, min((long long)cu[s], N)), b = max(a, min((long long)cu[s + 1], N));
   int cnt = 0, bad = 0;
@@ -761,38 +776,31 @@ __global__ void __launch_bounds__(128) seq_count_kernel(const int32_t* __restric
     red[1][threadIdx.x >> 5] = bad;
   }
   __syncthreads();
+  const bool defer = lp.agg_mode == MRL_AGG_TOKEN_MEAN && !(lp.pg_denominator > 0);
   if (threadIdx.x == 0) {
     cnt = red[0][0] + red[0][1] + red[0][2] + red[0][3];
     bad = red[1][0] + red[1][1] + red[1][2] + red[1][3];
     seq_cnt[s] = cnt;
+    len_sh = cnt;
     atomicAdd(&totals[0], (unsigned long long)cnt);  // integer sums: order does not matter
     if (bad) {
       atomicAdd(&totals[1], (unsigned long long)bad);
       if (status != nullptr) atomicOr(status, MRL_DEV_BAD_TOKEN_ID);
     }
+    __threadfence();
+    if (atomicAdd(&totals[3], 1ull) == (unsigned long long)S - 1) {  // every block has added its count
+      __threadfence();
+      const double D = (double)atomicAdd(&totals[0], 0ull);
+      cscale[0] = defer ? (D > 0 ? (float)(1.0 / D) : 0.f) : 1.0f;
+    }
   }
-}
-
-// A_t, c_t u_t, cn_t and beta c_t of every row (Eq. (1) aggregation and regulariser, Eq. (2) per-token average)
-__global__ void __launch_bounds__(128) row_coef_kernel(const int32_t* __restrict__ cu, int S, long long N, int V,
-                                                        const int32_t* __restrict__ ids,
-                                                        const uint8_t* __restrict__ mask,
-                                                        const float* __restrict__ adv_seq,
-                                                        const float* __restrict__ tok_weight,
-                                                        const float* __restrict__ nll_weight,
-                                                        const int32_t* __restrict__ seq_cnt,
-                                                        const unsigned long long* __restrict__ totals,
-                                                        mrl_loss_params lp, float* rowA, float* rowcu, float* rowcn,
-                                                        float* rowck) {
-  const int s = blockIdx.x;
-  const long long a = max(0ll, min((long long)cu[s], N)), b = max(a, min((long long)cu[s + 1], N));
-  const double len = (double)seq_cnt[s];
-  const double D = lp.pg_denominator > 0 ? lp.pg_denominator : (double)totals[0];
+  __syncthreads();
+  const double len = (double)len_sh;
   const double Sd = lp.seq_denominator > 0 ? lp.seq_denominator : (double)S;
   float c = 0.f, cn_base = 0.f;
   if (len > 0) {
     if (lp.agg_mode == MRL_AGG_TOKEN_MEAN)
-      c = D > 0 ? (float)(1.0 / D) : 0.f;
+      c = defer ? 1.0f : (float)(1.0 / lp.pg_denominator);
     else
       c = (float)(1.0 / (Sd * len));
     cn_base = (float)((double)lp.nll_coeff / len);
@@ -807,6 +815,11 @@ __global__ void __launch_bounds__(128) row_coef_kernel(const int32_t* __restrict
     rowcn[t] = (valid && nll_weight) ? cn_base * nll_weight[t] : 0.f;
     rowck[t] = (valid && lp.logp_ref != nullptr) ? lp.kl_coeff * c : 0.f;
   }
+  // rows outside every sequence must contribute nothing
+  const long long z0 = s == 0 ? 0 : N, z1 = s == 0 ? a : N;
+  for (long long t = z0 + threadIdx.x; t < z1; t += blockDim.x) rowA[t] = rowcu[t] = rowcn[t] = rowck[t] = 0.f;
+  if (s == S - 1)
+    for (long long t = b + threadIdx.x; t < N; t += blockDim.x) rowA[t] = rowcu[t] = rowcn[t] = rowck[t] = 0.f;
 }
 
 // Sum of six per-thread float64 values over a block of 256 threads in a fixed order (shuffle tree inside a warp, then
@@ -883,6 +896,7 @@ __global__ void __launch_bounds__(256) row_terms_kernel(long long N, const float
                                                          const float* __restrict__ rowcu,
                                                          const float* __restrict__ rowcn,
                                                          const float* __restrict__ rowck,
+                                                         const float* __restrict__ cscale,
                                                          const float* __restrict__ logp_ref, int kl_est,
                                                          const float* __restrict__ logp_old, float eps_lo,
                                                          float eps_hi, const FinalizeArgs fa,
@@ -894,14 +908,16 @@ __global__ void __launch_bounds__(256) row_terms_kernel(long long N, const float
   if ((st & kStatValid) && (st & kStatRead)) {
     const double lse = ((double)row_m2[t] + log2((double)row_s[t])) * 0.693147180559945309417232121458;
     lp = (double)row_zt[t] - lse;
-    const double A = rowA[t], cu = rowcu[t], cn = rowcn[t];
+    const float cs = cscale[0];
+    const double A = rowA[t], cu = rowcu[t] * cs, cn = rowcn[t];  // (the float products the row kernel formed)
+    const float ck = logp_ref != nullptr ? rowck[t] * cs : 0.f;
     if (cu != 0.0 && A != 0.0) {
       const double rho = logp_old ? exp(lp - (double)logp_old[t]) : 1.0;
       const double lo = 1.0 - (double)eps_lo, hi = 1.0 + (double)eps_hi;
       pg = -cu * fmin(rho * A, fmin(fmax(rho, lo), hi) * A);
     }
     if (cn != 0.0) nl = -cn * lp;
-    if (logp_ref != nullptr && rowck[t] != 0.f) kl = (double)rowck[t] * mrl::kl_value(lp - (double)logp_ref[t], kl_est);
+    if (ck != 0.f) kl = (double)ck * mrl::kl_value(lp - (double)logp_ref[t], kl_est);
   }
   if (t < N && logp != nullptr) logp[t] = (float)lp;
   double v[6] = {pg, nl, (st & kStatValid) ? 1.0 : 0.0, (st & kStatClipped) ? 1.0 : 0.0, (st & kStatRead) ? 1.0 : 0.0, kl};
@@ -927,7 +943,8 @@ __global__ void __launch_bounds__(256) rows_partial_kernel(long long N, const do
 MrlLossWs carve_loss_ws(void* ws, long long N, int S) {
   MrlCarver c(ws);
   MrlLossWs w;
-  w.totals = c.take<unsigned long long>(4);
+  w.totals = c.take<unsigned long long>(4);  // (one 256-byte piece: cleared by a single small memset per call)
+  w.cscale = reinterpret_cast<float*>(w.totals + 4);
   w.rowA = c.take<float>((size_t)N);
   w.rowcu = c.take<float>((size_t)N);
   w.rowcn = c.take<float>((size_t)N);
@@ -1037,12 +1054,9 @@ int mrl_rows_prepare(void* workspace, long long N, int V, int S, const int32_t* 
                      const float* nll_weight, const mrl_loss_params* lp, int32_t* status, cudaStream_t st,
                      MrlLossWs* out) {
   MrlLossWs w = carve_loss_ws(workspace, N, S);
-  // rows no sequence covers must contribute nothing: clear the coefficient arrays and the totals
-  MRL_CUDA_OK(cudaMemsetAsync(w.totals, 0, (size_t)((char*)w.row_m2 - (char*)w.totals), st));
-  seq_count_kernel<<<S, 128, 0, st>>>(cu_seqlens, S, N, V, ids, mask, w.seq_cnt, w.totals, status);
-  MRL_CUDA_OK(cudaGetLastError());
-  row_coef_kernel<<<S, 128, 0, st>>>(cu_seqlens, S, N, V, ids, mask, adv_seq, tok_weight, nll_weight, w.seq_cnt,
-                                     w.totals, *lp, w.rowA, w.rowcu, w.rowcn, w.rowck);
+  MRL_CUDA_OK(cudaMemsetAsync(w.totals, 0, 64, st));  // the counters, the tickets, cscale
+  seq_prepare_kernel<<<S, 128, 0, st>>>(cu_seqlens, S, N, V, ids, mask, adv_seq, tok_weight, nll_weight, *lp, w.seq_cnt,
+                                        w.totals, w.cscale, w.rowA, w.rowcu, w.rowcn, w.rowck, status);
   MRL_CUDA_OK(cudaGetLastError());
   *out = w;
   return MRL_OK;
@@ -1054,7 +1068,7 @@ int mrl_rows_finish(const MrlLossWs& w, long long N, const float* logp_old, cons
   const FinalizeArgs fa = {w.partials, w.totals, lp->flags, loss, lp->logp_ref != nullptr ? lp->kl_loss : nullptr,
                            reinterpret_cast<long long*>(stats)};
   row_terms_kernel<<<(unsigned)((N + 255) / 256), 256, 0, st>>>(N, w.row_m2, w.row_s, w.row_zt, w.rowstat, w.rowA,
-                                                                w.rowcu, w.rowcn, w.rowck, lp->logp_ref,
+                                                                w.rowcu, w.rowcn, w.rowck, w.cscale, lp->logp_ref,
                                                                 lp->kl_estimator, logp_old, lp->eps_lo, lp->eps_hi, fa,
                                                                 logp);
   MRL_CUDA_OK(cudaGetLastError());
@@ -1071,7 +1085,7 @@ int mrl_rows_finish_sequence(const MrlLossWs& w, long long N, int S, const int32
   MRL_CUDA_OK(cudaMemsetAsync(w.kl_term, 0, (size_t)N * sizeof(double), st));
   if (logp != nullptr) MRL_CUDA_OK(cudaMemsetAsync(logp, 0, (size_t)N * sizeof(float), st));
   seq_ratio_kernel<<<S, 256, 0, st>>>(cu_seqlens, S, N, w.row_m2, w.row_s, w.row_zt, w.rowstat, w.seq_cnt, adv_seq,
-                                      logp_old, nll_weight, w.rowck, *lp, w.pg_term, w.nll_term, w.kl_term, logp, g_out,
+                                      logp_old, nll_weight, w.rowck, w.cscale, *lp, w.pg_term, w.nll_term, w.kl_term, logp, g_out,
                                       lse2_out);
   MRL_CUDA_OK(cudaGetLastError());
   const FinalizeArgs fa = {w.partials, w.totals, lp->flags, loss, lp->logp_ref != nullptr ? lp->kl_loss : nullptr,
@@ -1176,6 +1190,7 @@ extern "C" int mrl_policy_loss_fwd_bwd(const void* logits, int32_t dtype, int64_
   p.rowcu = w.rowcu;
   p.rowcn = w.rowcn;
   p.rowck = w.rowck;
+  p.cscale = w.cscale;
   p.logp_ref = lp->logp_ref;
   p.kl_est = lp->kl_estimator;
   p.logp_old = logp_old;
