@@ -73,6 +73,7 @@ class ClockSampler:
     def __init__(self, device_index: int, period_s: float = 0.005):
         self.period = period_s
         self.samples = []
+        self.timed = []          # (host time, SM MHz, board power in W) of every sample
         self.reasons = set()
         self.max_mhz = None
         self._stop = threading.Event()
@@ -97,7 +98,13 @@ class ClockSampler:
                  0x4: "sw_power_cap", 0x80: "hw_power_brake_slowdown"}
         while not self._stop.is_set():
             try:
-                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                mhz = int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+                self.samples.append(mhz)
+                try:
+                    watts = nv.nvmlDeviceGetPowerUsage(self._h) / 1000.0
+                except Exception:
+                    watts = None
+                self.timed.append((time.perf_counter(), mhz, watts))
                 r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
                 for bit, name in names.items():
                     if r & bit:
@@ -116,6 +123,12 @@ class ClockSampler:
         self._stop.set()
         if self._thread is not None:
             self._thread.join()
+
+    def median_between(self, t0: float, t1: float):
+        """(median SM MHz, median W, samples) over the samples taken in [t0, t1] of the host clock."""
+        mhz = sorted(m for t, m, _ in self.timed if t0 <= t <= t1)
+        w = sorted(p for t, _, p in self.timed if t0 <= t <= t1 and p is not None)
+        return (mhz[len(mhz) // 2] if mhz else None, w[len(w) // 2] if w else None, len(mhz))
 
     def summary(self):
         if not self.samples:
@@ -600,6 +613,23 @@ class LmheadWorkload:
                                         None, None, self.lp, self.dH, self.dW, self.logp, self.loss, self.stats,
                                         self.status, self.ws)
 
+    def product_kinds(self, steps):
+        """Kind of every tensor-core launch of `steps` steps, in launch order, and the flops of one launch of each kind
+        (all rows worked on, as in config 5; the last, ragged vocabulary chunk is kept apart)."""
+        vchunk = 16384
+        chunks = -(-self.V // vchunk)
+        last = self.V - (chunks - 1) * vchunk
+        one = ["forward"]
+        for c in range(chunks):
+            tag = "" if (c < chunks - 1 or last == vchunk) else " (last chunk)"
+            one += ["dZ" + tag, "dHidden" + tag, "dW" + tag]
+        nh = 2.0 * self.rows_worked["backward"] * self.H
+        flops = {"forward": 2.0 * self.rows_worked["forward"] * self.H * self.V}
+        for k in ("dZ", "dHidden", "dW"):
+            flops[k] = nh * min(vchunk, self.V)
+            flops[k + " (last chunk)"] = nh * last
+        return one * steps, flops
+
     def tokens(self):
         return self.N
 
@@ -792,6 +822,83 @@ def measure_thl_align(seed, with_cpu):
     return res
 
 
+def per_product_table(kinds, flops, offsets_ms, durations_ms, t_start, clocks: ClockSampler, sms: int):
+    """Time x SM clock of every kind of tensor-core launch: mean duration, the median SM clock and board power sampled
+    while launches of that kind ran (their start offsets are CUDA-event times after `t_start`, the host time at which
+    the device was idle and the first launch was queued), and from them flop per clock per SM."""
+    out = {}
+    for kind in sorted(set(kinds)):
+        idx = [i for i, k in enumerate(kinds) if k == kind]
+        ms = sum(durations_ms[i] for i in idx) / len(idx)
+        mhz, watts = [], []
+        for i in idx:
+            a = t_start + offsets_ms[i] * 1e-3
+            m, w, _ = clocks.median_between(a, a + durations_ms[i] * 1e-3)
+            if m is not None:
+                mhz.append(m)
+            if w is not None:
+                watts.append(w)
+        mhz.sort()
+        watts.sort()
+        med = mhz[len(mhz) // 2] if mhz else None
+        out[kind] = {"launches": len(idx), "ms": ms, "sm_mhz": med, "watts": watts[len(watts) // 2] if watts else None,
+                     "tflops": flops[kind] / (ms * 1e-3) / 1e12,
+                     "flop_per_clk_per_sm": None if not med else flops[kind] / (ms * 1e-3 * med * 1e6 * sms)}
+    return out
+
+
+def library_loop_per_product(N, H, V, vchunk, steps, device_index):
+    """The same five product shapes as torch.matmul calls (the vendor library), in the step's order: the forward product
+    with its [N, V] store, then per full vocabulary chunk the dZ-, dHidden- and dW-shaped products.  A comparison leg
+    only: nothing of the library is on the product path."""
+    dev = torch.device("cuda", device_index)
+    g = torch.Generator(device=dev)
+    g.manual_seed(1)
+    hid = torch.randn(N, H, device=dev, dtype=torch.bfloat16, generator=g)
+    W = torch.randn(V, H, device=dev, dtype=torch.bfloat16, generator=g) * 0.02
+    Z = torch.empty(N, V, device=dev, dtype=torch.bfloat16)
+    D = torch.randn(N, vchunk, device=dev, dtype=torch.bfloat16, generator=g) * 0.01
+    Dz = torch.empty(N, vchunk, device=dev, dtype=torch.bfloat16)
+    dH = torch.empty(N, H, device=dev, dtype=torch.bfloat16)
+    dW = torch.empty(vchunk, H, device=dev, dtype=torch.bfloat16)
+    Wc = W[:vchunk]
+    chunks = V // vchunk
+    names = ["forward"] + ["dZ", "dHidden", "dW"] * chunks
+
+    def run(events):
+        calls = [lambda: torch.matmul(hid, W.t(), out=Z)]
+        for _ in range(chunks):
+            calls += [lambda: torch.matmul(hid, Wc.t(), out=Dz), lambda: torch.matmul(D, Wc, out=dH),
+                      lambda: torch.matmul(D.t(), hid, out=dW)]
+        for j, call in enumerate(calls):
+            if events is not None:
+                events[2 * j].record()
+            call()
+            if events is not None:
+                events[2 * j + 1].record()
+
+    run(None)
+    run(None)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(2 * len(names))] for _ in range(steps)]
+    with ClockSampler(device_index, 0.002) as clocks:
+        torch.cuda.synchronize()
+        t_start = time.perf_counter()
+        for ev in evs:
+            run(ev)
+        torch.cuda.synchronize()
+    kinds, offs, durs = [], [], []
+    for ev in evs:
+        for j, nm in enumerate(names):
+            kinds.append(nm)
+            offs.append(evs[0][0].elapsed_time(ev[2 * j]))
+            durs.append(ev[2 * j].elapsed_time(ev[2 * j + 1]))
+    fl = {"forward": 2.0 * N * H * V, "dZ": 2.0 * N * H * vchunk, "dHidden": 2.0 * N * H * vchunk, "dW": 2.0 * N * H * vchunk}
+    sms = torch.cuda.get_device_properties(device_index).multi_processor_count
+    table = per_product_table(kinds, fl, offs, durs, t_start, clocks, sms)
+    return {"what": "torch.matmul (vendor library) on the step's product shapes, full chunks only, plain bf16 stores",
+            "ms_per_pass": (offs[-1] + durs[-1]) / steps, "per_product": table}
+
+
 def time_oracle(O, args, repeats=1):
     best = None
     for _ in range(repeats):
@@ -886,7 +993,8 @@ def measure(wl, steps, warmup, world, local_rank, rank, peaks, with_e2e, with_cp
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier(world)
     torch.cuda.synchronize()
-    with ClockSampler(local_rank) as clocks, timer:
+    with ClockSampler(local_rank, 0.002 if hasattr(wl, "product_kinds") else 0.005) as clocks, timer:
+        t_start = time.perf_counter()        # the device is idle: the first launch starts about now
         ev0.record()
         for _ in range(steps):
             wl.step()
@@ -896,6 +1004,13 @@ def measure(wl, steps, warmup, world, local_rank, rank, peaks, with_e2e, with_cp
     local_ms = ev0.elapsed_time(ev1)
     kernel_ms = timer.elapsed_ms(steps * wl.dominant_per_step)
     wl.last_kernel = timer.last_kernel
+    per_product = None
+    if hasattr(wl, "product_kinds"):       # time x clock of every kind of tensor-core launch
+        n = steps * wl.dominant_per_step
+        kinds, flops = wl.product_kinds(steps)
+        offsets = [ev0.elapsed_time(timer.start[i]) for i in range(n)]
+        per_product = per_product_table(kinds, flops, offsets, kernel_ms[:n], t_start, clocks,
+                                        torch.cuda.get_device_properties(local_rank).multi_processor_count)
     status = int(wl.status.cpu())
     if status != 0:
         raise SystemExit(f"device status word is {status} after the timed region")
@@ -903,6 +1018,8 @@ def measure(wl, steps, warmup, world, local_rank, rank, peaks, with_e2e, with_cp
     out = {"value": total_tokens / (total_ms * 1e-3), "ms_per_step": total_ms / steps, "steps": steps,
            "config": dict(wl.describe(), parallelism=f"replicas x{world}"), "clocks": clocks.summary(),
            "gpu_launches": wl.kernels_per_step * steps, "roofline": wl.roofline(kernel_ms, peaks)}
+    if per_product is not None:
+        out["roofline"]["per_product"] = per_product
     # end to end: pinned host buffers -> device -> kernels -> pinned host buffers
     out["e2e"] = run_e2e(args, wl, world) if with_e2e else None
     if world == 1 and with_e2e and hasattr(wl, "measure_skip_zero_rows") and wl.ratio_level == 0 and not wl.lp.logp_ref:
@@ -952,6 +1069,13 @@ def run_ours(args, rank, world, local_rank):
               args.with_entropy, args.with_kl))
     res = measure(wl, args.steps, args.warmup, world, local_rank, rank, peaks, not args.no_e2e and not slab_main,
                   not args.no_cpu_baseline and not slab_main, args)
+    if lmhead_main and args.library_loop and world == 1:
+        N_, H_, V_ = wl.N, wl.H, wl.V
+        del wl
+        torch.cuda.empty_cache()
+        res["roofline"]["library_loop"] = library_loop_per_product(N_, H_, V_, min(16384, V_), max(2, min(args.steps, 4)),
+                                                                    local_rank)
+        wl = None
     del wl
     torch.cuda.empty_cache()
 
@@ -1035,6 +1159,9 @@ def main():
                     help="logits-in end-to-end leg: rows per micro-batch of the host pipeline")
     ap.add_argument("--skip-zero-rows", action="store_true",
                     help="fused LM-head workloads: MRL_FLAG_SKIP_ZERO_ROWS (zero-multiplier rows are not produced)")
+    ap.add_argument("--library-loop", action="store_true",
+                    help="fused LM-head workloads: also time torch.matmul (the vendor library) on the same product shapes, "
+                         "per product with the SM clock, beside the step's own per-product table (a comparison leg)")
     ap.add_argument("--pair-tiles", action="store_true",
                     help="fused LM-head workloads: 256-row tiles worked by CTA pairs (MRL_FLAG_PAIR_TILES)")
     ap.add_argument("--no-lmhead", action="store_true",
