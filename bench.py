@@ -60,8 +60,8 @@ def measured_peaks():
 # row had a gradient; traffic grows in proportion to the rows.  A launch of any other kernel, shape or batch kind
 # prints `traffic: null`, and so does an entry set to None because its kernel changed after the counters were taken.
 DRAM_BYTES_PER_TOKEN = {
-    ("row_stream_kernel", 151936, "half-live"): 642153,
-    ("row_stream_kernel", 151936, "all-live"): 687300,
+    ("row_stream_kernel", 151936, "half-live"): 637544,
+    ("row_stream_kernel", 151936, "all-live"): 668781,
 }
 NOMINAL_HBM_GBS = 8000.0        # B200 data sheet (7.7 TB/s on HGX boards): context beside the measured copy rate
 NOMINAL_BF16_TFLOPS = 2250.0    # dense bf16

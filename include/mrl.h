@@ -251,8 +251,7 @@ int mrl_token_logprobs(const void* logits, int32_t dtype, int64_t N, int32_t V, 
  *   workspace: mrl_workspace_bytes(MRL_WS_POLICY_LOSS, N, V, 0, dtype, S)
  *
  * float32 row arithmetic on the input dtype, float64 for the final N-term sums (fixed order:
- * bitwise reproducible from run to run for one entry point and one set of arguments; a forward-only call and a
- * gradient call may differ in the last bits).  dlogits is rounded to nearest even.  The fast path (one CTA per row:
+ * bitwise reproducible from run to run).  dlogits is rounded to nearest even.  The fast path (one CTA per row:
  * the row is streamed from HBM once and read a second time from L2) takes bf16 or float32 rows with V >= 4096 and
  * either 32-byte aligned logits / dlogits with V, ld, ld_out multiples of 32 bytes' worth of elements, or the same
  * with 16 bytes; anything else takes a general kernel with the same results.  Rows of 512 KB or more are shared by
