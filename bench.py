@@ -297,6 +297,27 @@ class LogitsInWorkload:
                              "peak_source": peaks["source"] + " (copy, burst)", "algorithmic_bytes_per_launch": alg,
                              "traffic": None}}
 
+    def measure_in_place(self, peaks, steps=20):
+        """The same step with dlogits written over the logits (the buffer a trainer would reuse for the gradient):
+        pass 2's stores then land on lines L2 already holds, so they take no capacity from the rows waiting for their
+        second read.  Runs on a copy of the logits; after the first step that copy holds gradients, which changes no
+        access pattern (rows keep their live / dead kind: it depends on the advantages, and on the KL term when on)."""
+        zc = self.z.clone()
+        for _ in range(3):
+            self.step(zc, zc)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(steps):
+            self.step(zc, zc)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / steps
+        gbs = self.bytes_per_token * self.N / (ms * 1e-3) / 1e9
+        return {"value": self.N / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms, "steps": steps,
+                "algorithmic_gbs_whole_step": gbs, "frac_whole_step": gbs / peaks["hbm_gbs"],
+                "note": "dlogits aliases logits (ld_out = ld); whole step by CUDA events, not the kernel alone"}
+
     def measure_skip_zero_rows(self, steps=10):
         """The same step with MRL_FLAG_SKIP_ZERO_ROWS: rows of zero-advantage groups are not read (their gradient
         rows are still written, as zeros).  Reported beside the headline, which streams every row."""
@@ -1025,6 +1046,8 @@ def measure(wl, steps, warmup, world, local_rank, rank, peaks, with_e2e, with_cp
     if world == 1 and with_e2e and hasattr(wl, "measure_skip_zero_rows") and wl.ratio_level == 0 and not wl.lp.logp_ref:
         out["skip_zero_rows"] = wl.measure_skip_zero_rows()
         out["token_logprobs"] = wl.measure_forward_only(peaks)
+    if world == 1 and hasattr(wl, "measure_in_place") and wl.ratio_level == 0 and getattr(args, "in_place_leg", True):
+        out["in_place"] = wl.measure_in_place(peaks)
     out["cpu_baseline"] = None
     if with_cpu and rank == 0 and world == 1:
         n, dt, sample = wl.time_oracle()
@@ -1087,7 +1110,7 @@ def run_ours(args, rank, world, local_rank):
         # every row with a gradient: the KL penalty of Eq. (1) on (App. A: beta = 1e-3), same batch as the headline
         wl_kl = LogitsInWorkload(synth.CONFIGS["C2"], args.seed + rank, device, 0, False, True)
         r = measure(wl_kl, sub_steps, 3, world, local_rank, rank, peaks, False, False, args)
-        shapes["all_rows_live"] = {"metric": METRIC, "unit": UNIT, **{k: r[k] for k in sub_keys}}
+        shapes["all_rows_live"] = {"metric": METRIC, "unit": UNIT, **{k: r[k] for k in sub_keys}, "in_place": r.get("in_place")}
         del wl_kl
         torch.cuda.empty_cache()
         for key, name in (("prp_pool_slab", "C3"), ("xgrpo_sgt_slab", "C4")):
@@ -1128,6 +1151,8 @@ def run_ours(args, rank, world, local_rank):
         if res.get("skip_zero_rows") is not None:
             line["skip_zero_rows"] = res["skip_zero_rows"]
             line["token_logprobs"] = res["token_logprobs"]
+        if res.get("in_place") is not None:
+            line["in_place"] = res["in_place"]
         line.update(shapes)
         if lmhead is not None:
             line["lmhead"] = lmhead
