@@ -293,6 +293,27 @@ def test_slab_accumulated_loss_that_does_not_cancel_matches_the_oracle_to_1e5(ag
     assert int(stats[0]) == ref["stats"][0]
 
 
+@pytest.mark.parametrize("V,dtype", [(1000, torch.float32), (8192, torch.bfloat16)])
+def test_rows_outside_every_sequence_contribute_nothing(V, dtype):
+    """cu_seqlens may start after row 0 or stop short of N (the contract asks for cu[0] = 0 and cu[S] = N, but only the
+    device sees the array): uncovered rows get zero gradient rows and no loss term; they still report their log-prob
+    and count as valid rows, and the covered rows are what a call on them alone gives."""
+    N, S, a, b = 48, 3, 5, 40
+    z, ids, _, _, adv, logp_old, g = toy_inputs(N, V, S, dtype, seed=91 + V)
+    cu = torch.tensor([a, 17, 29, b], dtype=torch.int32)
+    nllw = (torch.rand(N, generator=g) < 0.3).float()
+    lp = make_lp(nll_coeff=0.05, pg_den=float(b - a))
+    got = run_gpu_policy_loss(z, ids, None, cu, adv, logp_old, None, nllw, lp)
+    ref = O.policy_loss(z[a:b], ids[a:b], None, cu - a, adv, logp_old[a:b], None, nllw[a:b], oracle_lp(lp))
+    assert got["status"] == 0
+    outside = torch.ones(N, dtype=torch.bool)
+    outside[a:b] = False
+    assert float(got["dlogits"][outside].float().abs().max()) == 0
+    inner = dict(got, logp=got["logp"][a:b], dlogits=got["dlogits"][a:b])
+    compare_policy_loss(inner, ref, V, dtype, check_stats=False, cancelling=True)
+    assert int(got["stats"][0]) == N          # every row with a valid id counts as valid, covered or not
+
+
 def test_clip_boundary_neighbourhood():
     # ratios a few float32 ulps either side of 1 + eps and 1 - eps: decisions must match the oracle
     V, S = 4096, 1
