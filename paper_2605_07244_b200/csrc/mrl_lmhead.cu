@@ -24,13 +24,20 @@ constexpr int kAccStages = 2;
 constexpr int kTmemCols = kAccStages * BN;  // 512: all of tensor memory
 constexpr int kGemmThreads = 192;
 constexpr uint32_t kABytes = BM * BK * 2;  // a CTA's A tile of one stage
+// Epilogue staging: each of the four epilogue warps owns 32 rows of 128 bytes (+ 16 bytes of padding per row, which
+// keeps both the row-wise writes and the line-wise reads free of bank conflicts).  A thread holds one row of the
+// accumulator; written out directly, every warp store would touch 32 different lines with 16 bytes each, and those
+// requests compete with the operand copies for the SM's path to L2 (the dZ product lost 8 % of its tensor time to
+// them).  Staged through shared memory the same bytes leave as whole 128-byte lines.
+constexpr uint32_t kEpiRowBytes = 144, kEpiWarpBytes = 32 * kEpiRowBytes, kEpiStageBytes = 4 * kEpiWarpBytes;
 // kC CTAs share a tile of kC * 128 rows: each holds its own 128 rows of A and 256 / kC rows of B per stage
 template <int kC>
 struct GemmCfg {
   static constexpr int kBRows = BN / kC;
   static constexpr uint32_t kBBytes = kBRows * BK * 2, kStageBytes = kABytes + kBBytes;
   static constexpr int kStages = kC == 2 ? 6 : 4;  // 192 KB of stages either way
-  static constexpr size_t kSmem = (size_t)kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  static constexpr size_t kSmem = (size_t)kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/ +
+                                  kEpiStageBytes /*epilogue staging*/;
 };
 constexpr uint32_t kWaitLimit = 1u << 24;   // mbarrier polls before a wait gives up (of the order of a second)
 constexpr int kVChunk = 16384;              // vocabulary columns per backward chunk (multiple of BN)
@@ -275,6 +282,15 @@ __device__ __forceinline__ void store_bf16x32(__nv_bfloat16* dst, const float* d
   }
 }
 
+__device__ __forceinline__ void sts_v4(uint32_t addr, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+}
+__device__ __forceinline__ uint4 lds_v4(uint32_t addr) {
+  uint4 u;
+  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(u.x), "=r"(u.y), "=r"(u.z), "=r"(u.w) : "r"(addr));
+  return u;
+}
+
 // ------------------------------------------------------------------------------------------ the GEMM kernel
 // kAMn / kBMn: the operand is stored MN-major (its M / N index contiguous, K strided) instead of K-major.
 template <int EPI, int kC, bool kAMn, bool kBMn>
@@ -298,6 +314,7 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
   auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kStages + kAccStages + a); };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 2 * kAccStages);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const uint32_t epi_stage0 = bar0 + 256u;  // after the 256 bytes reserved for barriers and flags
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // a pair of CTAs (kC = 2) works on one tile of 256 rows: rank 0 leads (arms the barriers, issues the MMAs)
@@ -459,6 +476,13 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
       if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)acc * BN;
+      // staging area of this warp, and which of its 16-byte pieces this lane moves when a staged block is written out:
+      // piece i of the lane is bytes [16 (lane % 8), + 16) of row lane / 8 + 4 i, so a warp instruction covers four
+      // whole rows of 128 bytes
+      const uint32_t stg = epi_stage0 + (uint32_t)quad * kEpiWarpBytes;
+      const uint32_t stg_mine = stg + (uint32_t)lane * kEpiRowBytes;
+      const int piece_row = lane >> 3, piece_col = lane & 7;
+      const long long tile_row0 = (long long)(m * kC + rank) * BM + quad * 32;
 #pragma unroll 1
       for (int c = 0; c < BN; c += 32) {
         if (c >= ncols_valid) break;  // uniform across the CTA
@@ -480,54 +504,87 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
                 if (rel_id == c + j) d[j] = g * (mrl::ex2_approx(fmaf(v[j], MRL_LOG2E, -l2)) - 1.0f);
             }
           }
-          if (row_ok) {
+          // whole blocks of 64 columns with 128-byte aligned rows leave through the staging area as whole lines
+          const bool lines = (ncols_valid & 63) == 0 && (p.ldD & 63) == 0 && (reinterpret_cast<uintptr_t>(p.D) & 127) == 0;
+          if (lines) {
+            const uint32_t dst = stg_mine + (uint32_t)(c & 32) * 2u;
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+              sts_v4(dst + 16u * q, mrl::pack_bf16x2(d[q * 8 + 0], d[q * 8 + 1]), mrl::pack_bf16x2(d[q * 8 + 2], d[q * 8 + 3]),
+                     mrl::pack_bf16x2(d[q * 8 + 4], d[q * 8 + 5]), mrl::pack_bf16x2(d[q * 8 + 6], d[q * 8 + 7]));
+            if (c & 32) {  // 64 columns of 32 rows are staged: 4 KB, eight 16-byte pieces per lane
+              __syncwarp();
+              __nv_bfloat16* base = p.D + (long long)n * BN + (c - 32) + piece_col * 8;
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                const int r = piece_row + 4 * i;
+                const uint4 u = lds_v4(stg + (uint32_t)r * kEpiRowBytes + (uint32_t)piece_col * 16u);
+                if (tile_row0 + r < p.M) *reinterpret_cast<uint4*>(base + (tile_row0 + r) * p.ldD) = u;
+              }
+              __syncwarp();
+            }
+          } else if (row_ok) {
             const int nvalid = ncols_valid - c;
             store_bf16x32(p.D + (long long)row * p.ldD + (long long)n * BN + c, d, nvalid);
           }
         } else {
-          if (row_ok) {
-            const int nvalid = ncols_valid - c;
-            const long long col = (long long)n * BN + c;
+          const int nvalid = ncols_valid - c;
+          const long long col = (long long)n * BN + c;
+          const bool f32_out = p.c_mode == C_F32 || p.c_mode == C_F32_ADD;
+          // float32 accumulator traffic (read-modify-write of C, or the read of the running sum): one staged block is
+          // 32 rows x 32 floats = 32 whole lines
+          const float* acc_in = p.c_mode == C_F32_ADD ? static_cast<const float*>(p.C) : p.Cacc;
+          const long long ld_in = p.c_mode == C_F32_ADD ? p.ldc : p.ldacc;
+          const bool lines = p.c_mode != C_BF16 && nvalid >= 32 && (ld_in & 3) == 0 &&
+                             (reinterpret_cast<uintptr_t>(acc_in) & 15) == 0 &&
+                             (f32_out ? ((p.ldc & 3) == 0 && (reinterpret_cast<uintptr_t>(p.C) & 15) == 0)
+                                      : ((p.ldc & 3) == 0 && (reinterpret_cast<uintptr_t>(p.C) & 7) == 0));
+          if (lines) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+              sts_v4(stg_mine + 16u * q, __float_as_uint(v[4 * q + 0]), __float_as_uint(v[4 * q + 1]),
+                     __float_as_uint(v[4 * q + 2]), __float_as_uint(v[4 * q + 3]));
+            __syncwarp();
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const int r = piece_row + 4 * i;
+              const uint4 u = lds_v4(stg + (uint32_t)r * kEpiRowBytes + (uint32_t)piece_col * 16u);
+              if (tile_row0 + r < p.M) {
+                float4 t = make_float4(__uint_as_float(u.x), __uint_as_float(u.y), __uint_as_float(u.z), __uint_as_float(u.w));
+                const long long off = col + piece_col * 4;
+                if (p.c_mode != C_F32) {
+                  const float4 o = *reinterpret_cast<const float4*>(acc_in + (tile_row0 + r) * ld_in + off);
+                  t.x += o.x;
+                  t.y += o.y;
+                  t.z += o.z;
+                  t.w += o.w;
+                }
+                if (f32_out) {
+                  *reinterpret_cast<float4*>(static_cast<float*>(p.C) + (tile_row0 + r) * p.ldc + off) = t;
+                } else {
+                  uint2 w;
+                  w.x = mrl::pack_bf16x2(t.x, t.y);
+                  w.y = mrl::pack_bf16x2(t.z, t.w);
+                  *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(p.C) + (tile_row0 + r) * p.ldc + off) = w;
+                }
+              }
+            }
+            __syncwarp();
+          } else if (row_ok) {
             if (p.c_mode == C_BF16) {
               store_bf16x32(static_cast<__nv_bfloat16*>(p.C) + (long long)row * p.ldc + col, v, nvalid);
             } else if (p.c_mode == C_BF16_FROM_ACC) {
               const float* a = p.Cacc + (long long)row * p.ldacc + col;
-              if (nvalid >= 32 && (reinterpret_cast<uintptr_t>(a) & 15) == 0) {
 #pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                  const float4 t = reinterpret_cast<const float4*>(a)[q];
-                  v[4 * q + 0] += t.x;
-                  v[4 * q + 1] += t.y;
-                  v[4 * q + 2] += t.z;
-                  v[4 * q + 3] += t.w;
-                }
-              } else {
-#pragma unroll
-                for (int j = 0; j < 32; ++j)
-                  if (j < nvalid) v[j] += a[j];
-              }
+              for (int j = 0; j < 32; ++j)
+                if (j < nvalid) v[j] += a[j];
               store_bf16x32(static_cast<__nv_bfloat16*>(p.C) + (long long)row * p.ldc + col, v, nvalid);
             } else {
               float* o = static_cast<float*>(p.C) + (long long)row * p.ldc + col;
               const bool add = p.c_mode == C_F32_ADD;
-              if (nvalid >= 32 && (reinterpret_cast<uintptr_t>(o) & 15) == 0) {
 #pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                  float4 t = make_float4(v[4 * q + 0], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
-                  if (add) {
-                    const float4 r = reinterpret_cast<const float4*>(o)[q];
-                    t.x += r.x;
-                    t.y += r.y;
-                    t.z += r.z;
-                    t.w += r.w;
-                  }
-                  reinterpret_cast<float4*>(o)[q] = t;
-                }
-              } else {
-#pragma unroll
-                for (int j = 0; j < 32; ++j)
-                  if (j < nvalid) o[j] = add ? o[j] + v[j] : v[j];
-              }
+              for (int j = 0; j < 32; ++j)
+                if (j < nvalid) o[j] = add ? o[j] + v[j] : v[j];
             }
           }
         }
