@@ -49,6 +49,7 @@ struct GemmParams {
   int M, N, K;
   int m_tiles, n_tiles, k_blocks;
   int group_m;            // row-tiles per raster group
+  int a_blocks, b_blocks; // MN-major operand with a three-dimensional map (make_tmap_mn_blocks): fetched by one copy
   // Optional compaction (device arrays; the counts are read by the kernel, so the host never waits for them):
   const int* m_list;      // ascending indices of the row-tiles (of BM * kC rows) to work on; null = all of them
   const int* m_count;     // [1] how many
@@ -112,6 +113,13 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
       : "memory");
 }
+// the same for a three-dimensional box (an MN-major operand fetched as several 64-wide blocks by one instruction)
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
+      : "memory");
+}
 __device__ __forceinline__ uint32_t mapa_u32(uint32_t addr, uint32_t rank) {
   uint32_t r;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
@@ -127,6 +135,12 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap
   asm volatile(
       "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
       : "memory");
 }
 // commit of a CTA pair's MMAs: one arrival on the barrier at this offset in every CTA of `mask`
@@ -392,16 +406,27 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
             auto load = [&](uint32_t dst, const CUtensorMap* map, int x, int y) {
               if (kC == 2) tma_load_2d_pair(dst, map, x, y, bar); else tma_load_2d(dst, map, x, y, bar);
             };
-            if (kAMn) {  // boxes of 64 rows-of-the-tile x BK
+            auto load_blocks = [&](uint32_t dst, const CUtensorMap* map, int block0, int y) {
+              if (kC == 2) tma_load_3d_pair(dst, map, 0, y, block0, bar); else tma_load_3d(dst, map, 0, y, block0, bar);
+            };
+            if (kAMn) {  // blocks of 64 rows-of-the-tile x BK: one copy, or one per block
+              if (p.a_blocks) {
+                load_blocks(a_dst, &tmapA, a_row / 64, kx);
+              } else {
 #pragma unroll
-              for (int q = 0; q < BM / 64; ++q) load(a_dst + (uint32_t)q * (BK * 128), &tmapA, a_row + 64 * q, kx);
+                for (int q = 0; q < BM / 64; ++q) load(a_dst + (uint32_t)q * (BK * 128), &tmapA, a_row + 64 * q, kx);
+              }
             } else {
               load(a_dst, &tmapA, kx, a_row);
             }
             if (kBMn) {
+              if (p.b_blocks) {
+                load_blocks(a_dst + kABytes, &tmapB, b_row / 64, kx);
+              } else {
 #pragma unroll
-              for (int q = 0; q < Cfg::kBRows / 64; ++q)
-                load(a_dst + kABytes + (uint32_t)q * (BK * 128), &tmapB, b_row + 64 * q, kx);
+                for (int q = 0; q < Cfg::kBRows / 64; ++q)
+                  load(a_dst + kABytes + (uint32_t)q * (BK * 128), &tmapB, b_row + 64 * q, kx);
+              }
             } else {
               load(a_dst + kABytes, &tmapB, kx, b_row);
             }
@@ -807,6 +832,23 @@ int make_tmap(CUtensorMap* map, const void* base, long long rows, long long cols
   return r == CUDA_SUCCESS ? MRL_OK : MRL_ERR_CUDA;
 }
 
+// Tensor map of an MN-major operand -- a row-major bf16 matrix [k_rows, mn] (ld elements between rows) whose mn is a
+// multiple of 64 -- as a three-dimensional tensor {64 elements, k_rows, mn / 64 blocks}: one box of {64, 64, blocks}
+// then lands in shared memory as `blocks` consecutive 8 KB atoms of 64 K-rows x 128 bytes, which is the layout the
+// MMA reads an MN-major operand from, with a single copy instruction instead of one per block.
+int make_tmap_mn_blocks(CUtensorMap* map, const void* base, long long k_rows, long long mn, long long ld, int blocks) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return MRL_ERR_CUDA;
+  const cuuint64_t dims[3] = {64, (cuuint64_t)k_rows, (cuuint64_t)(mn / 64)};
+  const cuuint64_t strides[2] = {(cuuint64_t)ld * 2, 128};
+  const cuuint32_t box[3] = {64, (cuuint32_t)BK, (cuuint32_t)blocks};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? MRL_OK : MRL_ERR_CUDA;
+}
+
 int sm_count() {
   static int n[64] = {};
   int dev = 0;
@@ -875,9 +917,16 @@ int launch_gemm(const void* A, long long lda, const void* B, long long ldb, Gemm
   const int kC = pairs > 0 ? 2 : 1;
   CUtensorMap ta, tb;
   // K-major: tiles of [box rows x 64 of K]; MN-major: boxes of [64 of K rows x 64 of M / N]
-  int rc = kAMn ? make_tmap(&ta, A, p.K, p.M, lda, BK) : make_tmap(&ta, A, p.M, p.K, lda, BM);
+  // (an MN-major operand whose M / N extent is a multiple of 64 gets the three-dimensional map: one copy per stage)
+  p.a_blocks = (kAMn && p.M % 64 == 0) ? BM / 64 : 0;
+  p.b_blocks = (kBMn && p.N % 64 == 0) ? BN / kC / 64 : 0;
+  int rc = !kAMn        ? make_tmap(&ta, A, p.M, p.K, lda, BM)
+           : p.a_blocks ? make_tmap_mn_blocks(&ta, A, p.K, p.M, lda, p.a_blocks)
+                        : make_tmap(&ta, A, p.K, p.M, lda, BK);
   if (rc != MRL_OK) return rc;
-  rc = kBMn ? make_tmap(&tb, B, p.K, p.N, ldb, BK) : make_tmap(&tb, B, p.N, p.K, ldb, BN / kC);
+  rc = !kBMn        ? make_tmap(&tb, B, p.N, p.K, ldb, BN / kC)
+       : p.b_blocks ? make_tmap_mn_blocks(&tb, B, p.K, p.N, ldb, p.b_blocks)
+                    : make_tmap(&tb, B, p.K, p.N, ldb, BK);
   if (rc != MRL_OK) return rc;
   p.m_tiles = (p.M + BM * kC - 1) / (BM * kC);
   if (m_rows != nullptr) {
