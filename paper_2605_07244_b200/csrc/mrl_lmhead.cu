@@ -570,19 +570,28 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
               sts_v4(stg_mine + 16u * q, __float_as_uint(v[4 * q + 0]), __float_as_uint(v[4 * q + 1]),
                      __float_as_uint(v[4 * q + 2]), __float_as_uint(v[4 * q + 3]));
             __syncwarp();
+            // (all eight reads of the running sum are issued before the first of them is used: one round trip to
+            // memory per block, not eight)
+            const long long off = col + piece_col * 4;
+            float4 o[8];
+            if (p.c_mode != C_F32) {
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                const long long rr = tile_row0 + piece_row + 4 * i;
+                o[i] = rr < p.M ? *reinterpret_cast<const float4*>(acc_in + rr * ld_in + off) : make_float4(0.f, 0.f, 0.f, 0.f);
+              }
+            }
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
               const int r = piece_row + 4 * i;
               const uint4 u = lds_v4(stg + (uint32_t)r * kEpiRowBytes + (uint32_t)piece_col * 16u);
               if (tile_row0 + r < p.M) {
                 float4 t = make_float4(__uint_as_float(u.x), __uint_as_float(u.y), __uint_as_float(u.z), __uint_as_float(u.w));
-                const long long off = col + piece_col * 4;
                 if (p.c_mode != C_F32) {
-                  const float4 o = *reinterpret_cast<const float4*>(acc_in + (tile_row0 + r) * ld_in + off);
-                  t.x += o.x;
-                  t.y += o.y;
-                  t.z += o.z;
-                  t.w += o.w;
+                  t.x += o[i].x;
+                  t.y += o[i].y;
+                  t.z += o[i].z;
+                  t.w += o[i].w;
                 }
                 if (f32_out) {
                   *reinterpret_cast<float4*>(static_cast<float*>(p.C) + (tile_row0 + r) * p.ldc + off) = t;
