@@ -1,0 +1,131 @@
+"""Seeded random shapes and option mixes through both loss entry points, against the oracle.
+
+The hand-picked cases elsewhere pin each kernel path; this sweep draws the combinations nobody thought of:
+empty sequences between non-empty ones, one-row batches, masks that empty a whole sequence, token weights with
+exact zeros, either aggregation, a given or a derived denominator, the KL term on or off, forward only or with
+the gradient, padded rows.  Every draw is a pure function of its seed.
+"""
+import pytest
+import torch
+
+from oracle import mrl_oracle as O
+from paper_2605_07244_b200 import binding as B
+from paper_2605_07244_b200 import build
+
+from helpers import KlTerm, compare_policy_loss, loss_close, make_lp, oracle_lp, run_gpu_policy_loss
+from test_lmhead_gpu import compare as compare_lmhead
+from test_lmhead_gpu import run_gpu_lmhead
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+    B.lib()
+
+
+def _cuts_with_empty_sequences(N, S, g):
+    """cu_seqlens of S sequences over N rows, non-decreasing, some sequences empty."""
+    inner = torch.sort(torch.randint(0, N + 1, (S - 1,), generator=g)).values.tolist() if S > 1 else []
+    return torch.tensor([0] + inner + [N], dtype=torch.int32)
+
+
+def _draw_logits_case(seed):
+    g = torch.Generator().manual_seed(1000 + seed)
+    pick = lambda xs: xs[int(torch.randint(0, len(xs), (1,), generator=g))]
+    dtype = pick([torch.bfloat16, torch.bfloat16, torch.float32])
+    V = pick([1, 2, 7, 130, 1000, 4096, 4100, 8192 + 16, 12296, 40000 + 8])
+    N = pick([1, 2, 3, 17, 64, 150])
+    S = pick([1, 2, 5, 9])
+    pad = pick([0, 0, 8, 16, 5])
+    z = (torch.randn(N, V + pad, generator=g) * 2.0).to(dtype)
+    z[:, V:] = 25.0                                    # would wreck the sums if anything read past V
+    ids = torch.randint(0, V, (N,), generator=g, dtype=torch.int32)
+    cu = _cuts_with_empty_sequences(N, S, g)
+    adv = torch.randn(S, generator=g)
+    adv[torch.rand(S, generator=g) < 0.25] = 0.0       # zero-advantage sequences
+    mask = None
+    if pick([True, False]):
+        mask = (torch.rand(N, generator=g) < 0.75).to(torch.uint8)
+        if S > 1 and int(cu[1]) > 0:
+            mask[:int(cu[1])] = 0                       # the first sequence has no valid token at all
+    logp, _, _ = O.token_logprobs(z[:, :V], ids, mask)
+    logp_old = (logp + 0.15 * torch.randn(N, generator=g, dtype=torch.float64)).float()
+    u = None
+    if pick([True, False]):
+        u = torch.rand(N, generator=g) + 0.25
+        u[torch.rand(N, generator=g) < 0.2] = 0.0
+    nllw = (torch.rand(N, generator=g) < 0.3).float() if pick([True, False]) else None
+    agg = pick([B.AGG_TOKEN_MEAN, B.AGG_SEQ_MEAN_TOKEN_MEAN])
+    n_valid = int(N if mask is None else mask.sum())
+    given = pick([True, False])
+    lp = make_lp(agg=agg, nll_coeff=0.07 if nllw is not None else 0.0, pg_den=float(n_valid + 11) if given else 0.0,
+                 seq_den=float(S + 2) if given else 0.0,
+                 flags=B.FLAG_SKIP_ZERO_ROWS if pick([True, False, False]) else 0)
+    ref_trace = (logp + 0.3 * torch.randn(N, generator=g, dtype=torch.float64)).float() if pick([True, False, False]) else None
+    return dict(z=z, V=V, ids=ids, mask=mask, cu=cu, adv=adv, logp_old=logp_old, u=u, nllw=nllw, lp=lp, dtype=dtype,
+                ref_trace=ref_trace, want_grad=pick([True, True, False]), estimator=pick([B.KL_K1, B.KL_K2, B.KL_K3]))
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_logits_in_random_case(seed):
+    c = _draw_logits_case(seed)
+    lp = c["lp"]
+    kl = KlTerm(lp, c["ref_trace"], 0.01, c["estimator"]) if c["ref_trace"] is not None else None
+    got = run_gpu_policy_loss(c["z"], c["ids"], c["mask"], c["cu"], c["adv"], c["logp_old"], c["u"], c["nllw"], lp,
+                              V=c["V"], want_dlogits=c["want_grad"])
+    ref = O.policy_loss(c["z"][:, :c["V"]], c["ids"], c["mask"], c["cu"], c["adv"], c["logp_old"], c["u"], c["nllw"],
+                        oracle_lp(lp), logp_ref=c["ref_trace"])
+    assert got["status"] == 0
+    if lp.flags & B.FLAG_SKIP_ZERO_ROWS:
+        # rows whose multiplier is known to be zero beforehand are not read: they report logp = 0 (and still count)
+        dead = ref["valid"] & ((ref["cu"] == 0) | (ref["A"] == 0)) & (ref["cn"] == 0)
+        if c["ref_trace"] is not None:
+            dead = torch.zeros_like(dead)           # the KL term keeps every valid row live
+        if dead.any():
+            assert float(got["logp"][dead].abs().max()) == 0
+        # ... and cannot be classified as clipped or not
+        clipped = int((ref["valid"] & ~dead & (ref["A"] != 0) & ref["clipped"]).sum())
+        ref = dict(ref, logp=torch.where(dead, torch.zeros_like(ref["logp"]), ref["logp"]), stats=(ref["stats"][0], clipped))
+    # A float32 log-prob carries about 1e-7 of absolute error, so an NLL term whose |logp| is tiny (a two-word
+    # vocabulary with a dominant logit) cannot be held to 1e-5 of itself: floor at 2e-2 of the sum of its coefficients (2e-7 absolute per log-prob).
+    compare_policy_loss(got, ref, c["V"], c["dtype"], cancelling=True, loss_floor=2e-2 * float(ref["cn"].abs().sum()))
+    if kl is not None:
+        assert loss_close(kl.value(), ref["loss_kl"], ref["kl_term"].abs().sum())
+
+
+def _draw_lmhead_case(seed):
+    g = torch.Generator().manual_seed(5000 + seed)
+    pick = lambda xs: xs[int(torch.randint(0, len(xs), (1,), generator=g))]
+    N = pick([1, 31, 128, 129, 300, 513])
+    H = pick([64, 128, 192, 320])
+    V = pick([37, 256, 1000, 4099, 16384 + 64, 20000])
+    S = pick([1, 3, 6])
+    hidden = torch.randn(N, H, generator=g).to(torch.bfloat16)
+    W = (torch.randn(V, H, generator=g) * (2.0 / H ** 0.5)).to(torch.bfloat16)
+    ids = torch.randint(0, V, (N,), generator=g, dtype=torch.int32)
+    cu = _cuts_with_empty_sequences(N, S, g)
+    adv = torch.randn(S, generator=g)
+    adv[torch.rand(S, generator=g) < 0.2] = 0.0
+    mask = (torch.rand(N, generator=g) < 0.8).to(torch.uint8) if pick([True, False]) else None
+    zz = hidden.double() @ W.double().T
+    logp, _, _ = O.token_logprobs(zz, ids, mask)
+    logp_old = (logp + 0.1 * torch.randn(N, generator=g, dtype=torch.float64)).float()
+    u = (torch.rand(N, generator=g) + 0.5) if pick([True, False]) else None
+    nllw = (torch.rand(N, generator=g) < 0.25).float() if pick([True, False]) else None
+    lp = make_lp(agg=pick([B.AGG_TOKEN_MEAN, B.AGG_SEQ_MEAN_TOKEN_MEAN]), nll_coeff=0.05 if nllw is not None else 0.0,
+                 flags=B.FLAG_PAIR_TILES if pick([True, False, False]) else 0)
+    return hidden, W, ids, mask, cu, adv, logp_old, u, nllw, lp
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_hidden_in_random_case(seed):
+    hidden, W, ids, mask, cu, adv, logp_old, u, nllw, lp = _draw_lmhead_case(seed)
+    got = run_gpu_lmhead(hidden, W, ids, mask, cu, adv, logp_old, u, nllw, lp)
+    ref = O.fused_lmhead_loss(hidden, W, ids, mask, cu, adv, logp_old, u, nllw, oracle_lp(lp))
+    tie = bool((ref["valid"] & (ref["margin"] < 2e-5)).any())
+    no_gradient = float(ref["g"].abs().max()) == 0
+    if no_gradient:
+        assert float(got["dH"].float().abs().max()) == 0 and float(got["dW"].float().abs().max()) == 0
+    compare_lmhead(got, ref, check_grads=not tie and not no_gradient)
