@@ -5,6 +5,7 @@
 // place on the staging buffer, device-to-host copy of its gradient -- run on three streams over three staging
 // buffers, so that the bus carries data in both directions while the kernels work.  Everything the pass computes
 // is computed by mrl_policy_loss_fwd_bwd; this file only plans the slabs and orders the copies.
+#include <mutex>
 #include <vector>
 
 #include "mrl_common.cuh"
@@ -24,11 +25,13 @@ struct HostPipe {
   cudaEvent_t in_done[kBufs] = {}, comp_done[kBufs] = {}, out_done[kBufs] = {};
 };
 HostPipe g_pipe[kMaxDevices];
+std::mutex g_pipe_mutex;  // guards the one-time creation (calls on one device must still not overlap: they share the pipe)
 
 int pipe_for_current_device(HostPipe** out) {
   int dev = -1;
   MRL_CUDA_OK(cudaGetDevice(&dev));
   if (dev < 0 || dev >= kMaxDevices) return MRL_ERR_UNSUPPORTED_SHAPE;
+  std::lock_guard<std::mutex> lock(g_pipe_mutex);
   HostPipe& p = g_pipe[dev];
   if (!p.ready) {
     MRL_CUDA_OK(cudaStreamCreateWithFlags(&p.in, cudaStreamNonBlocking));

@@ -7,6 +7,7 @@
 // crosses the HBM interface once in each direction (plus what L2 has dropped); nothing is shared between CTAs.
 // General kernel (any dtype, any V, any alignment): one CTA per row, three passes over global
 // memory; used for short or unaligned rows.
+#include <mutex>
 #include <type_traits>
 
 #include "mrl_common.cuh"
@@ -1244,6 +1245,8 @@ int static_ws_address(void** out) {
   int dev = -1;
   MRL_CUDA_OK(cudaGetDevice(&dev));
   if (dev < 0 || dev >= kMaxDevices) return MRL_ERR_UNSUPPORTED_SHAPE;
+  static std::mutex lookup_mutex;  // the one-time look-up may be raced by threads; the array itself is still shared
+  std::lock_guard<std::mutex> lock(lookup_mutex);
   if (g_static_ws_ptr[dev] == nullptr) {
     void* ptr = nullptr;
     MRL_CUDA_OK(cudaGetSymbolAddress(&ptr, g_static_loss_ws));
