@@ -62,6 +62,7 @@ def measured_peaks():
 DRAM_BYTES_PER_TOKEN = {
     ("row_stream_kernel", 151936, "half-live"): 637544,
     ("row_stream_kernel", 151936, "all-live"): 668781,
+    ("row_stream_kernel", 128256, "prp-pool"): 535630,      # config-3 slab of 12,288 rows (pooled advantages, density weights)
 }
 NOMINAL_HBM_GBS = 8000.0        # B200 data sheet (7.7 TB/s on HGX boards): context beside the measured copy rate
 NOMINAL_BF16_TFLOPS = 2250.0    # dense bf16
@@ -552,10 +553,17 @@ class PoolSlabWorkload:
         row_bytes = self.V * self.z.element_size()
         alg_bytes = streamed * 2 * row_bytes + (self.N - streamed) * row_bytes      # unread rows are still zero-filled
         achieved = alg_bytes / (k_avg_ms * 1e-3) / 1e9
-        return {"bound": "hbm", "kernel": getattr(self, "last_kernel", ""), "achieved": achieved, "peak": peaks["hbm_gbs"],
+        # DRAM traffic from the small-slab captures, scaled by the rows: config 3 by its own figure; config 4's read rows
+        # all carry a gradient (the others are not read), so they take the every-row-live figure of the same vocabulary
+        # (a 10,240-row slab of config 4 measured 669,884 B per token against that figure's 668,781) and its unread
+        # rows one row of zeros each
+        launched = getattr(self, "last_kernel", "")
+        per_token = DRAM_BYTES_PER_TOKEN.get((launched, self.V, "prp-pool" if self.name == "C3" else "all-live"))
+        traffic = None if per_token is None else per_token * streamed + (self.N - streamed) * row_bytes
+        return {"bound": "hbm", "kernel": launched, "achieved": achieved, "peak": peaks["hbm_gbs"],
                 "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "frac_nominal": achieved / NOMINAL_HBM_GBS,
                 "peak_source": peaks["source"] + " (copy, burst)", "algorithmic_bytes_per_launch": alg_bytes,
-                "rows_read": streamed, "kernel_ms": k_avg_ms, "traffic": None}
+                "rows_read": streamed, "kernel_ms": k_avg_ms, "traffic": traffic}
 
 
 class LmheadWorkload:

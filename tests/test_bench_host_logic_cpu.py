@@ -44,8 +44,8 @@ def test_per_product_table_without_samples_reports_no_clock():
 def test_traffic_figures_are_keyed_by_kernel_vocabulary_and_batch_kind():
     keys = set(bench.DRAM_BYTES_PER_TOKEN)
     assert ("row_stream_kernel", 151936, "half-live") in keys and ("row_stream_kernel", 151936, "all-live") in keys
-    alg = 2 * 151936 * 2
     for k, v in bench.DRAM_BYTES_PER_TOKEN.items():
+        alg = 2 * k[1] * 2
         assert v is None or alg <= v < 1.3 * alg, k         # measured traffic is at least the algorithmic bytes
     assert bench.DRAM_BYTES_PER_TOKEN.get(("row_general_kernel", 151936, "half-live")) is None
 
