@@ -243,7 +243,8 @@ int mrl_token_logprobs(const void* logits, int32_t dtype, int64_t N, int32_t V, 
  *   nll_weight [device] float32 [N] SGT weight (1 on rows of a selected y*); nullable = 0
  *   lp         [host]
  *   dlogits    [device] dtype [N, ld_out]; may equal `logits` with ld_out = ld (in place);
- *              nullable = forward only.  Every row is written (zeros where g_t = 0).
+ *              nullable = forward only.  Every row is written (zeros where g_t = 0).  In place is also the
+ *              faster way to call (measured 3-4 % on B200: the stores then land on lines L2 already holds).
  *   logp       [device] float32 [N], nullable
  *   loss       [device] float32 [2]: policy-gradient term, NLL term
  *   stats      [device] int64 [4], nullable: valid rows, clipped rows (valid, A != 0), rows
