@@ -10,7 +10,12 @@
 #include "mrl.h"
 
 #define MRL_LOG2E 1.4426950408889634f
-#define MRL_LN2 0.6931471805599453f
+// The base-2 domain of the running sums is x = z * MRL_LOG2E with the FLOAT constant above, so the way back to nats
+// divides by that float: 1 / float(log2 e) = MRL_NAT_HI + MRL_NAT_LO (to 2e-16).  Multiplying by ln 2 instead is 1.06e-8
+// off, a bias of 1e-7 in every log-sum-exp, which a response-level ratio adds up over the tokens of a response.
+#define MRL_NAT_HI 0.6931471824645996f
+#define MRL_NAT_LO 7.348693209507928e-09f
+#define MRL_NAT_F64 0.6931471898132927
 
 #define MRL_CUDA_OK(expr)                       \
   do {                                          \
@@ -92,6 +97,9 @@ __device__ __forceinline__ float ex2_approx(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+
+// base-2 log-sum-exp (in units of MRL_LOG2E) -> nats
+__device__ __forceinline__ float lse2_to_nats(float lse2) { return fmaf(lse2, MRL_NAT_HI, lse2 * MRL_NAT_LO); }
 
 __device__ __forceinline__ float bf16lo_to_f32(uint32_t packed) { return __uint_as_float(packed << 16); }
 __device__ __forceinline__ float bf16hi_to_f32(uint32_t packed) { return __uint_as_float(packed & 0xffff0000u); }

@@ -785,7 +785,7 @@ __global__ void __launch_bounds__(256) lmhead_rows_kernel(long long N, int V, in
   uint8_t st = 0;
   if (valid) {
     l2 = acc.m + log2f(acc.s);
-    const float logp = zt[t] - l2 * MRL_LN2;
+    const float logp = zt[t] - mrl::lse2_to_nats(l2);
     mrl::RowIn in;
     in.A = rowA[t];
     in.cu = rowcu[t] * cscale[0];
@@ -800,7 +800,7 @@ __global__ void __launch_bounds__(256) lmhead_rows_kernel(long long N, int V, in
     st = MRL_ROW_VALID | MRL_ROW_READ;
     if (ro.clipped && in.A != 0.f) st |= MRL_ROW_CLIPPED;
   }
-  if (entropy != nullptr) entropy[t] = valid ? l2 * MRL_LN2 - usum / acc.s : 0.f;  // H = lse - sum_v p_v z_v
+  if (entropy != nullptr) entropy[t] = valid ? mrl::lse2_to_nats(l2) - usum / acc.s : 0.f;  // H = lse - sum_v p_v z_v
   row_m2[t] = acc.m;
   row_s[t] = acc.s;
   row_zt[t] = valid ? zt[t] : 0.f;

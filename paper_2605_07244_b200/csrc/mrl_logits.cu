@@ -434,7 +434,7 @@ __global__ void __launch_bounds__(kT, 1024 / kT) row_stream_kernel(const RowPara
     }
     if (lane == 0) {
       const float lse2 = tm + log2f(ts);
-      const float lse = lse2 * MRL_LN2;
+      const float lse = mrl::lse2_to_nats(lse2);
       float logp = 0.f, g = 0.f;
       bool clipped = false;
       if (ctx.valid && ok) {
@@ -543,7 +543,7 @@ __global__ void __launch_bounds__(kThreads) row_general_kernel(const RowParams p
   }
   const mrl::Lse2 tot = mrl::lse2_block_reduce<kThreads>(acc, scratch);
   const float lse2 = tot.m + log2f(tot.s);
-  const float lse = lse2 * MRL_LN2;
+  const float lse = mrl::lse2_to_nats(lse2);
   const float logp = zt - lse;
   float g = 0.f;
   bool clipped = false;
@@ -681,12 +681,12 @@ __global__ void __launch_bounds__(256) seq_ratio_kernel(const int32_t* __restric
   __shared__ double diff_sh;
   const int s = blockIdx.x, tid = threadIdx.x;
   const long long a = max(0ll, min((long long)cu[s], N)), b = max(a, min((long long)cu[s + 1], N));
-  const double kLn2 = 0.693147180559945309417232121458;
+  const double kNat = MRL_NAT_F64;  // nats per unit of the base-2 sums (1 / the float log2 e they were scaled with)
   double d = 0.0;
   for (long long t = a + tid; t < b; t += 256) {
     const uint8_t st = rowstat[t];
     if ((st & kStatValid) && (st & kStatRead)) {
-      const double lpv = (double)row_zt[t] - ((double)row_m2[t] + log2((double)row_s[t])) * kLn2;
+      const double lpv = (double)row_zt[t] - ((double)row_m2[t] + log2((double)row_s[t])) * kNat;
       d += lpv - (logp_old ? (double)logp_old[t] : lpv);
     }
   }
@@ -717,7 +717,7 @@ __global__ void __launch_bounds__(256) seq_ratio_kernel(const int32_t* __restric
     double nl = 0.0, kl = 0.0;
     if (valid) {
       l2 = row_m2[t] + log2f(row_s[t]);
-      lpv = (double)row_zt[t] - ((double)row_m2[t] + log2((double)row_s[t])) * kLn2;
+      lpv = (double)row_zt[t] - ((double)row_m2[t] + log2((double)row_s[t])) * kNat;
       const float cn = nll_weight ? (float)cn_base * nll_weight[t] : 0.f;
       g = g_pg + cn;
       if (cn != 0.f) nl = -(double)cn * lpv;

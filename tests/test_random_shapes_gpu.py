@@ -129,3 +129,60 @@ def test_hidden_in_random_case(seed):
     if no_gradient:
         assert float(got["dH"].float().abs().max()) == 0 and float(got["dW"].float().abs().max()) == 0
     compare_lmhead(got, ref, check_grads=not tie and not no_gradient)
+
+
+def _draw_sequence_ratio_case(seed):
+    g = torch.Generator().manual_seed(9000 + seed)
+    pick = lambda xs: xs[int(torch.randint(0, len(xs), (1,), generator=g))]
+    dtype = pick([torch.bfloat16, torch.float32])
+    V = pick([3, 130, 1000, 4096, 8192 + 16, 40000 + 8])
+    N = pick([1, 5, 33, 90])
+    S = pick([1, 2, 4, 7])
+    z = (torch.randn(N, V, generator=g) * 2.0).to(dtype)
+    ids = torch.randint(0, V, (N,), generator=g, dtype=torch.int32)
+    cu = _cuts_with_empty_sequences(N, S, g)
+    adv = torch.randn(S, generator=g)
+    adv[torch.rand(S, generator=g) < 0.25] = 0.0
+    mask = None
+    if pick([True, False]):
+        mask = (torch.rand(N, generator=g) < 0.8).to(torch.uint8)
+        if S > 1 and int(cu[1]) > 0:
+            mask[:int(cu[1])] = 0                       # a response without a valid token
+    logp, _, _ = O.token_logprobs(z, ids, mask)
+    old = (logp + 0.06 * torch.randn(N, generator=g, dtype=torch.float64)).float()
+    nllw = (torch.rand(N, generator=g) < 0.3).float() if pick([True, False]) else None
+    lp = make_lp(nll_coeff=0.05 if nllw is not None else 0.0, ratio_level=B.RATIO_SEQUENCE)
+    return dict(z=z, V=V, ids=ids, mask=mask, cu=cu, adv=adv, old=old, nllw=nllw, lp=lp, dtype=dtype,
+                want_grad=pick([True, True, False]))
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_sequence_ratio_random_case(seed):
+    """Response-level ratio (App. H) on drawn shapes: empty responses, responses with every token masked, zero
+    advantages, with and without the NLL rows, forward only or with the gradient."""
+    from helpers import GRAD_REL_L2_BF16, GRAD_REL_L2_F32, LOGP_ATOL, LOSS_RTOL, rel_l2
+    c = _draw_sequence_ratio_case(seed)
+    got = run_gpu_policy_loss(c["z"], c["ids"], c["mask"], c["cu"], c["adv"], c["old"], None, c["nllw"], c["lp"],
+                              V=c["V"], want_dlogits=c["want_grad"])
+    ref = O.policy_loss_sequence_ratio(c["z"], c["ids"], c["mask"], c["cu"], c["adv"], c["old"], c["nllw"],
+                                       oracle_lp(c["lp"]))
+    assert got["status"] == 0
+    assert (got["logp"].double() - ref["logp"]).abs().max() <= LOGP_ATOL
+    assert not (ref["seq_margin"] < 1e-4).any(), "a response sits on the clip boundary: change the seed"
+    for k, name, terms in ((0, "loss_pg", "seq_term"), (1, "loss_nll", "nll_term")):
+        # the response-level tolerance: 1e-5 of the total magnitude of the terms (a ratio exponentiates a sum of
+        # float32 log-probs), plus 2e-7 absolute per NLL coefficient for log-probs near zero
+        scale = max(abs(ref[name]), float(ref[terms].abs().sum()))
+        floor = 2e-7 * float(ref["cn"].abs().sum()) if name == "loss_nll" else 0.0
+        assert abs(float(got["loss"][k]) - ref[name]) <= LOSS_RTOL * scale + floor + 1e-12, name
+    assert int(got["stats"][0]) == ref["stats"][0] and int(got["stats"][1]) == ref["stats"][1]
+    if c["want_grad"]:
+        dz = got["dlogits"][:, :c["V"]].double()
+        assert torch.isfinite(dz).all()
+        if float(ref["g"].abs().max()) == 0:
+            assert float(dz.abs().max()) == 0
+        else:
+            assert rel_l2(dz, ref["dlogits"]) <= (GRAD_REL_L2_BF16 if c["dtype"] == torch.bfloat16 else GRAD_REL_L2_F32)
+        zero = ref["g"] == 0
+        if zero.any():
+            assert float(dz[zero].abs().max()) == 0
