@@ -186,3 +186,90 @@ def test_sequence_ratio_random_case(seed):
         zero = ref["g"] == 0
         if zero.any():
             assert float(dz[zero].abs().max()) == 0
+
+
+@pytest.mark.parametrize("seed", range(20))
+def test_group_advantages_and_gate_random_case(seed):
+    """Sec. 3 advantages (own, pooled, batch-whitened) and the SGT gate of Sec. 5.3 on drawn group shapes and reward
+    laws: binary, graded in [0, 1], constant groups, any learner index, every pick rule."""
+    g = torch.Generator().manual_seed(13000 + seed)
+    pick = lambda xs: xs[int(torch.randint(0, len(xs), (1,), generator=g))]
+    P, M, G = pick([1, 2, 7, 64, 300]), pick([1, 2, 3, 4]), pick([1, 2, 4, 8, 16, 33])
+    law = pick(["binary", "graded", "sparse"])
+    if law == "binary":
+        r = (torch.rand(P, M, G, generator=g) < torch.rand(P, M, 1, generator=g)).float()
+    elif law == "graded":
+        r = (torch.rand(P, M, G, generator=g) * 4).round() / 4          # 0, 1/4, ..., 1: many ties
+    else:
+        r = (torch.rand(P, M, G, generator=g) < 0.05).float()           # mostly all-zero groups
+    if P > 1:
+        r[P // 2] = float(pick([0, 1]))                                  # a prompt where every candidate agrees
+    lens = torch.randint(1, 9, (P, M, G), generator=g, dtype=torch.int32)
+    learner = int(torch.randint(0, M, (1,), generator=g))
+    mode = pick([B.ADV_MEAN_ONLY, B.ADV_GROUP_ZNORM, B.ADV_BATCH_ZNORM])
+    ddof = pick([0, 1])
+    rule = pick([B.PICK_NONE, B.PICK_FIRST, B.PICK_SHORTEST, B.PICK_ALL, B.PICK_SEEDED])
+    seed64 = int(torch.randint(0, 2 ** 31 - 1, (1,), generator=g))
+    ap = B.AdvParams(mode, ddof, 1e-6, 0.8, 0.2, rule, seed64)
+    dev = lambda t: t.cuda()
+    own = torch.full((P, M, G), float("nan"), device="cuda")
+    pool = torch.full((P, M, G), float("nan"), device="cuda")
+    rescue = torch.full((P,), 9, dtype=torch.uint8, device="cuda")
+    pk = torch.full((P,), -7, dtype=torch.int32, device="cuda")
+    w = torch.full((P, M, G), float("nan"), device="cuda")
+    n = torch.full((1,), -1, dtype=torch.int32, device="cuda")
+    B.mrl_group_advantages(dev(r), dev(lens), learner, ap, own, pool, rescue, pk, w, n)
+    torch.cuda.synchronize()
+    ref_own, ref_pool = O.group_advantages(r, mode, ddof, 1e-6)
+    for got, ref in ((own, ref_own), (pool, ref_pool)):
+        assert torch.isfinite(got).all()
+        assert (got.cpu().double() - ref).abs().max() <= 2e-6 * max(1.0, float(ref.abs().max()))
+    gate = O.sgt_gate(r, lens, learner, 0.8, 0.2, rule, seed64)
+    assert torch.equal(rescue.cpu(), gate[0]) and torch.equal(pk.cpu(), gate[1])
+    assert torch.equal(w.cpu().double(), gate[2]) and int(n.cpu()) == gate[3]
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_hidden_in_random_options(seed):
+    """The fused LM head with its options drawn together: KL term (any estimator), entropy output, dW accumulated in
+    float32, zero-multiplier rows skipped, pair tiles — logits, gradients and terms against the float64 oracle."""
+    hidden, W, ids, mask, cu, adv, logp_old, u, nllw, lp = _draw_lmhead_case(100 + seed)
+    g = torch.Generator().manual_seed(17000 + seed)
+    pick = lambda xs: xs[int(torch.randint(0, len(xs), (1,), generator=g))]
+    N, V = hidden.shape[0], W.shape[0]
+    zz = hidden.double() @ W.double().T
+    logp64, _, _ = O.token_logprobs(zz, ids, mask)
+    with_kl, with_ent, accum = pick([True, False]), pick([True, False]), pick([True, False])
+    if pick([True, False, False]):
+        lp.flags |= B.FLAG_SKIP_ZERO_ROWS
+    if accum:
+        lp.flags |= B.FLAG_ACCUMULATE_DW
+    ref_trace = (logp64 + 0.3 * torch.randn(N, generator=g, dtype=torch.float64)).float() if with_kl else None
+    kl = KlTerm(lp, ref_trace, 0.02, pick([B.KL_K1, B.KL_K2, B.KL_K3])) if with_kl else None
+    ent = torch.full((N,), float("nan"), device="cuda") if with_ent else None
+    if with_ent:
+        lp.entropy = ent.data_ptr()
+    dW_init = torch.randn(V, hidden.shape[1], generator=g) * 0.01 if accum else None
+    got = run_gpu_lmhead(hidden, W, ids, mask, cu, adv, logp_old, u, nllw, lp, dW_init=dW_init)
+    ref = O.fused_lmhead_loss(hidden, W, ids, mask, cu, adv, logp_old, u, nllw, oracle_lp(lp), logp_ref=ref_trace)
+    if lp.flags & B.FLAG_SKIP_ZERO_ROWS and not with_kl:
+        dead = ref["valid"] & ((ref["cu"] == 0) | (ref["A"] == 0)) & (ref["cn"] == 0)
+        # blocks of 256 rows made of dead or masked rows are not produced: such rows report logp = 0; a dead row in a
+        # live block may report either
+        lg = got["logp"].double()
+        both = dead & (lg == 0)
+        ref = dict(ref, logp=torch.where(both, torch.zeros_like(ref["logp"]), ref["logp"]))
+    tie = bool((ref["valid"] & (ref["margin"] < 2e-5)).any())
+    no_gradient = float(ref["g"].abs().max()) == 0
+    compare_lmhead(got, ref, check_grads=not tie and not no_gradient, dW_base=dW_init)
+    if kl is not None:
+        # k1 is linear in a log-prob that carries the error of a float32-accumulated bf16 dot product (a few 1e-7, and
+        # not zero-mean: the tensor core does not round its accumulator to nearest), so the term is held relative to
+        # the sum of its |terms|, as in tests/test_kl_gpu.py
+        scale = max(abs(ref["loss_kl"]), float(ref["kl_term"].abs().sum()))
+        assert abs(kl.value() - ref["loss_kl"]) <= 1e-5 * scale + 1e-12
+    if with_ent:
+        ref_ent = O.token_entropy(zz, ids, mask)
+        e = ent.cpu().double()
+        read = e != 0 if lp.flags & B.FLAG_SKIP_ZERO_ROWS else torch.ones(N, dtype=torch.bool)
+        assert torch.isfinite(e).all() and (e - ref_ent)[read].abs().max() <= 1e-4
