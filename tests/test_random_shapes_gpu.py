@@ -273,3 +273,43 @@ def test_hidden_in_random_options(seed):
         e = ent.cpu().double()
         read = e != 0 if lp.flags & B.FLAG_SKIP_ZERO_ROWS else torch.ones(N, dtype=torch.bool)
         assert torch.isfinite(e).all() and (e - ref_ent)[read].abs().max() <= 1e-4
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_host_pipeline_random_case(seed):
+    """The host-buffer entry point on drawn batches — empty sequences between others, masks, either aggregation, any
+    micro-batch size from one sequence to everything, token or response level — against one device call on the whole
+    batch: per-row outputs bit for bit, the loss up to the order of its sums."""
+    from test_host_pipeline_gpu import run_host
+    g = torch.Generator().manual_seed(21000 + seed)
+    pick = lambda xs: xs[int(torch.randint(0, len(xs), (1,), generator=g))]
+    dtype = pick([torch.bfloat16, torch.bfloat16, torch.float32])
+    V = pick([1008, 4096, 8192 + 16, 40000])          # the entry point wants rows of whole 32-byte units
+    N = pick([1, 40, 150, 300])
+    S = pick([1, 3, 8, 20])
+    z = (torch.randn(N, V, generator=g) * 2.0).to(dtype)
+    ids = torch.randint(0, V, (N,), generator=g, dtype=torch.int32)
+    cu = _cuts_with_empty_sequences(N, S, g)
+    adv = torch.randn(S, generator=g)
+    adv[torch.rand(S, generator=g) < 0.25] = 0.0
+    mask = (torch.rand(N, generator=g) < 0.8).to(torch.uint8) if pick([True, False]) else None
+    logp, _, _ = O.token_logprobs(z, ids, mask)
+    seq_level = pick([False, False, True])
+    old = (logp + (0.03 if seq_level else 0.15) * torch.randn(N, generator=g, dtype=torch.float64)).float()
+    tw = (torch.rand(N, generator=g) + 0.5) if (not seq_level and pick([True, False])) else None
+    nllw = (torch.rand(N, generator=g) < 0.3).float() if pick([True, False]) else None
+    agg = pick([B.AGG_TOKEN_MEAN, B.AGG_SEQ_MEAN_TOKEN_MEAN])
+    longest = max(1, int((cu[1:] - cu[:-1]).max()))
+    slab_rows = max(longest, pick([1, 7, 64, 100000]))
+    mk = lambda: make_lp(agg=agg, nll_coeff=0.05 if nllw is not None else 0.0,
+                         ratio_level=B.RATIO_SEQUENCE if seq_level else B.RATIO_TOKEN)
+    one = run_gpu_policy_loss(z, ids, mask, cu, adv, old, tw, nllw, mk())
+    got = run_host(z, ids, mask, cu, adv, old, tw, nllw, mk(), slab_rows)
+    assert got["status"] == 0 and one["status"] == 0
+    bits = torch.int16 if dtype == torch.bfloat16 else torch.int32
+    assert torch.equal(got["logp"], one["logp"])
+    assert torch.equal(got["dlogits"].view(bits), one["dlogits"].view(bits))
+    assert torch.equal(got["stats"], one["stats"])
+    for k in range(2):
+        a, b = float(got["loss"][k]), float(one["loss"][k])
+        assert abs(a - b) <= 2e-6 * max(abs(a), abs(b)) + 1e-9          # float32 sums in another order
