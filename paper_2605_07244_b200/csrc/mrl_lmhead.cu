@@ -30,12 +30,19 @@ constexpr uint32_t kABytes = BM * BK * 2;  // a CTA's A tile of one stage
 // requests compete with the operand copies for the SM's path to L2 (the dZ product lost 8 % of its tensor time to
 // them).  Staged through shared memory the same bytes leave as whole 128-byte lines.
 constexpr uint32_t kEpiRowBytes = 144, kEpiWarpBytes = 32 * kEpiRowBytes, kEpiStageBytes = 4 * kEpiWarpBytes;
-// kC CTAs share a tile of kC * 128 rows: each holds its own 128 rows of A and 256 / kC rows of B per stage
-template <int kC>
+// kC CTAs share a tile of kC * 128 rows: each holds its own 128 rows of A and 256 / kC rows of B per stage.
+// kR = 2 (single CTAs only): a CTA works on a tile of 256 rows as two 128-row halves that share the B tile -- two MMAs
+// per K step, one into each half of tensor memory -- so a stage carries 64 KB for twice the flops (a third fewer
+// operand bytes per flop from L2, like a pair, without the pair's traffic between shared memories); the accumulators
+// are then not double-buffered, which suits products whose K is long against their epilogue.
+template <int kC, int kR = 1>
 struct GemmCfg {
+  static_assert(kR == 1 || (kR == 2 && kC == 1), "tall tiles are a single-CTA shape");
   static constexpr int kBRows = BN / kC;
-  static constexpr uint32_t kBBytes = kBRows * BK * 2, kStageBytes = kABytes + kBBytes;
-  static constexpr int kStages = kC == 2 ? 6 : 4;  // 192 KB of stages either way
+  static constexpr uint32_t kACtaBytes = kR * kABytes;
+  static constexpr uint32_t kBBytes = kBRows * BK * 2, kStageBytes = kACtaBytes + kBBytes;
+  static constexpr int kStages = (192 * 1024) / kStageBytes;  // 4 (128-row tiles), 6 (pairs), 3 (tall): 192 KB of stages
+  static constexpr int kAccs = kAccStages / kR;               // accumulators a CTA cycles through
   static constexpr size_t kSmem = (size_t)kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/ +
                                   kEpiStageBytes /*epilogue staging*/;
 };
@@ -307,11 +314,12 @@ __device__ __forceinline__ uint4 lds_v4(uint32_t addr) {
 
 // ------------------------------------------------------------------------------------------ the GEMM kernel
 // kAMn / kBMn: the operand is stored MN-major (its M / N index contiguous, K strided) instead of K-major.
-template <int EPI, int kC, bool kAMn, bool kBMn>
+template <int EPI, int kC, bool kAMn, bool kBMn, int kR = 1>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
                    const GemmParams p) {
-  using Cfg = GemmCfg<kC>;
+  using Cfg = GemmCfg<kC, kR>;
+  constexpr int kAccs = Cfg::kAccs;
   constexpr int kStages = Cfg::kStages;
   constexpr uint32_t kStageBytes = Cfg::kStageBytes;
   constexpr bool kLse = EPI == EPI_LSE || EPI == EPI_LSE_ENT;
@@ -380,7 +388,7 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
         int m, n;
         tile_coords(t, m_tiles, p.n_tiles, p.group_m, m, n);
         if (p.m_list != nullptr) m = p.m_list[m];
-        const int a_row = (m * kC + rank) * BM, b_row = n * BN + rank * Cfg::kBRows;
+        const int a_row = (m * kC + rank) * (BM * kR), b_row = n * BN + rank * Cfg::kBRows;
         // K-block indices come from the list (when there is one) eight at a time and one group ahead, so that their
         // loads never sit between two copies
         auto k_index = [&](int kb) { return (p.k_list != nullptr && kb < k_blocks) ? __ldg(p.k_list + kb) : kb; };
@@ -414,21 +422,21 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
                 load_blocks(a_dst, &tmapA, a_row / 64, kx);
               } else {
 #pragma unroll
-                for (int q = 0; q < BM / 64; ++q) load(a_dst + (uint32_t)q * (BK * 128), &tmapA, a_row + 64 * q, kx);
+                for (int q = 0; q < kR * BM / 64; ++q) load(a_dst + (uint32_t)q * (BK * 128), &tmapA, a_row + 64 * q, kx);
               }
             } else {
               load(a_dst, &tmapA, kx, a_row);
             }
             if (kBMn) {
               if (p.b_blocks) {
-                load_blocks(a_dst + kABytes, &tmapB, b_row / 64, kx);
+                load_blocks(a_dst + Cfg::kACtaBytes, &tmapB, b_row / 64, kx);
               } else {
 #pragma unroll
                 for (int q = 0; q < Cfg::kBRows / 64; ++q)
-                  load(a_dst + kABytes + (uint32_t)q * (BK * 128), &tmapB, b_row + 64 * q, kx);
+                  load(a_dst + Cfg::kACtaBytes + (uint32_t)q * (BK * 128), &tmapB, b_row + 64 * q, kx);
               }
             } else {
-              load(a_dst + kABytes, &tmapB, kx, b_row);
+              load(a_dst + Cfg::kACtaBytes, &tmapB, kx, b_row);
             }
             if (++stage == kStages) { stage = 0; phase ^= 1u; }
           }
@@ -444,13 +452,13 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
       for (int t = unit; t < total_tiles && ok; t += n_units) {
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)acc * BN;
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kR) * BN;
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
           tc_fence_after();
           const uint32_t a_src = tiles + (uint32_t)stage * kStageBytes;
           const uint64_t adesc = kAMn ? smem_desc_mn128(a_src) : smem_desc_k128(a_src);
-          const uint64_t bdesc = kBMn ? smem_desc_mn128(a_src + kABytes) : smem_desc_k128(a_src + kABytes);
+          const uint64_t bdesc = kBMn ? smem_desc_mn128(a_src + Cfg::kACtaBytes) : smem_desc_k128(a_src + Cfg::kACtaBytes);
           // one step of K = 16: 32 bytes along a K-major swizzle row, two 1024-byte atoms of an MN-major tile
           constexpr uint64_t a_step = kAMn ? (2048 >> 4) : 2, b_step = kBMn ? (2048 >> 4) : 2;
 #pragma unroll
@@ -458,7 +466,9 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
             if (kC == 2)
               tc_mma_pair(d_tmem, adesc + a_step * k, bdesc + b_step * k, kIdesc<kC, kAMn, kBMn>, (kb | k) != 0);
             else
-              tc_mma(d_tmem, adesc + a_step * k, bdesc + b_step * k, kIdesc<kC, kAMn, kBMn>, (kb | k) != 0);
+              for (int h = 0; h < kR; ++h)  // the 128-row halves of a tall tile: 16 KB further in A, BN columns further in D
+                tc_mma(d_tmem + (uint32_t)h * BN, adesc + a_step * k + (uint64_t)h * (kABytes >> 4), bdesc + b_step * k,
+                       kIdesc<kC, kAMn, kBMn>, (kb | k) != 0);
           }
           // the stage is free (in both CTAs) once these MMAs have read it
           if (kC == 2) tc_commit_pair(empty_bar(stage), 3); else tc_commit(empty_bar(stage));
@@ -466,7 +476,7 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
         }
         if (!ok) break;
         if (kC == 2) tc_commit_pair(tfull_bar(acc), 3); else tc_commit(tfull_bar(acc));
-        if (++acc == kAccStages) { acc = 0; acc_phase ^= 1u; }
+        if (++acc == kAccs) { acc = 0; acc_phase ^= 1u; }
       }
     }
   } else {
@@ -480,9 +490,12 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
       int m, n;
       tile_coords(t, m_tiles, p.n_tiles, p.group_m, m, n);
       if (p.m_list != nullptr) m = p.m_list[m];
-      const int row = (m * kC + rank) * BM + row_in_tile;
-      const bool row_ok = row < p.M;
       const int ncols_valid = min(BN, p.N - n * BN);
+#pragma unroll 1
+      for (int h = 0; h < kR; ++h) {  // the 128-row halves of a tall tile, one after the other
+      const int half_row0 = ((m * kC + rank) * kR + h) * BM;
+      const int row = half_row0 + row_in_tile;
+      const bool row_ok = row < p.M;
       // per-row inputs before the accumulator is ready
       LseRow st = {-INFINITY, 0.f, 0.f, false, 0.f};
       int rel_id = -1;
@@ -498,16 +511,18 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
         neg_k = -(l2 - log2f(fabsf(g)));  // 2^(z log2e - k) = |g| softmax(z); unused when g = 0
         sgn = g < 0.f ? -1.f : 1.f;
       }
-      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
-      tc_fence_after();
-      const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)acc * BN;
+      if (h == 0) {
+        if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+      }
+      const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * kR + h) * BN;
       // staging area of this warp, and which of its 16-byte pieces this lane moves when a staged block is written out:
       // piece i of the lane is bytes [16 (lane % 8), + 16) of row lane / 8 + 4 i, so a warp instruction covers four
       // whole rows of 128 bytes
       const uint32_t stg = epi_stage0 + (uint32_t)quad * kEpiWarpBytes;
       const uint32_t stg_mine = stg + (uint32_t)lane * kEpiRowBytes;
       const int piece_row = lane >> 3, piece_col = lane & 7;
-      const long long tile_row0 = (long long)(m * kC + rank) * BM + quad * 32;
+      const long long tile_row0 = (long long)half_row0 + quad * 32;
 #pragma unroll 1
       for (int c = 0; c < BN; c += 32) {
         if (c >= ncols_valid) break;  // uniform across the CTA
@@ -623,18 +638,20 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
           }
         }
       }
-      // the accumulator has been read: hand it back to the MMA warp
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) {  // the leader's barrier collects the epilogue warps of both CTAs
-        if (kC == 2 && rank != 0) mbar_arrive_remote(mapa_u32(tempty_bar(acc), 0u)); else mbar_arrive(tempty_bar(acc));
+      if (h == kR - 1) {  // the accumulator has been read: hand it back to the MMA warp
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {  // the leader's barrier collects the epilogue warps of both CTAs
+          if (kC == 2 && rank != 0) mbar_arrive_remote(mapa_u32(tempty_bar(acc), 0u)); else mbar_arrive(tempty_bar(acc));
+        }
       }
       if (kLse && row_ok) {
         p.partial[(long long)n * p.part_ld + row] = make_float2(st.m, st.s);
         if (EPI == EPI_LSE_ENT) p.partial_u[(long long)n * p.part_ld + row] = st.u;
         if (st.has) p.zt[row] = st.zt;
       }
-      if (++acc == kAccStages) { acc = 0; acc_phase ^= 1u; }
+      }  // halves
+      if (++acc == kAccs) { acc = 0; acc_phase ^= 1u; }
     }
   }
 
@@ -894,6 +911,16 @@ struct TileLists {
   int *m256, *m128, *k64, *counts;
 };
 
+// Whether a product with both operands MN-major (dW) takes tall tiles: its K must be long enough that the epilogue, which
+// a tall tile cannot overlap with the next tile's MMAs (about 5,000 cycles against 1,024 per K-block), stays a few per
+// cent, and there must be at least one tall tile per SM.  Measured on the dW product of a 16,384-column chunk at
+// K = 65,536: 7.2 -> 6.3-6.4 ms, at a clock only 3 % lower (pairs of CTAs gain the same activity and lose it to clock).
+// The dHidden product (K = 16,384, float32 read-modify-write epilogue) measured slower with tall tiles and keeps 128 rows.
+bool tall_policy(const GemmParams& p) {
+  const long long tall_tiles = (long long)((p.M + 2 * BM - 1) / (2 * BM)) * ((p.N + BN - 1) / BN);
+  return p.K >= 8192 && tall_tiles >= sm_count();
+}
+
 // `m_rows` / `k_rows`: the M (resp. K) dimension of the product is the batch's rows and only the listed blocks count.
 template <int EPI, bool kAMn, bool kBMn>
 int launch_gemm(const void* A, long long lda, const void* B, long long ldb, GemmParams p, bool pair_tiles,
@@ -906,9 +933,14 @@ int launch_gemm(const void* A, long long lda, const void* B, long long ldb, Gemm
   const int arc = mrl_once_per_device(attr_done, [] {
     const cudaError_t e = cudaFuncSetAttribute(lmhead_gemm_kernel<EPI, 2, kAMn, kBMn>,
                                                cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GemmCfg<2>::kSmem);
-    return e != cudaSuccess ? e
-                            : cudaFuncSetAttribute(lmhead_gemm_kernel<EPI, 1, kAMn, kBMn>,
-                                                   cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GemmCfg<1>::kSmem);
+    if (e != cudaSuccess) return e;
+    if constexpr (EPI == EPI_STORE && kAMn && kBMn) {
+      const cudaError_t e2 = cudaFuncSetAttribute(lmhead_gemm_kernel<EPI, 1, kAMn, kBMn, 2>,
+                                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GemmCfg<1, 2>::kSmem);
+      if (e2 != cudaSuccess) return e2;
+    }
+    return cudaFuncSetAttribute(lmhead_gemm_kernel<EPI, 1, kAMn, kBMn>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)GemmCfg<1>::kSmem);
   });
   if (arc != MRL_OK) return arc;
   cudaLaunchConfig_t cfg = {};
@@ -924,12 +956,16 @@ int launch_gemm(const void* A, long long lda, const void* B, long long ldb, Gemm
   cfg.numAttrs = 1;
   const int pairs = pair_tiles ? resident_pairs<EPI, kAMn, kBMn>(&cfg) : 0;
   const int kC = pairs > 0 ? 2 : 1;
+  // tall tiles (256 rows in one CTA, accumulators not double-buffered)
+  constexpr bool kTallShape = EPI == EPI_STORE && kAMn && kBMn;
+  const bool tall = kTallShape && kC == 1 && tall_policy(p);
+  const int kR = tall ? 2 : 1;
   CUtensorMap ta, tb;
   // K-major: tiles of [box rows x 64 of K]; MN-major: boxes of [64 of K rows x 64 of M / N]
   // (an MN-major operand whose M / N extent is a multiple of 64 gets the three-dimensional map: one copy per stage)
-  p.a_blocks = (kAMn && p.M % 64 == 0) ? BM / 64 : 0;
+  p.a_blocks = (kAMn && p.M % 64 == 0) ? kR * BM / 64 : 0;
   p.b_blocks = (kBMn && p.N % 64 == 0) ? BN / kC / 64 : 0;
-  int rc = !kAMn        ? make_tmap(&ta, A, p.M, p.K, lda, BM)
+  int rc = !kAMn        ? make_tmap(&ta, A, p.M, p.K, lda, kR * BM)
            : p.a_blocks ? make_tmap_mn_blocks(&ta, A, p.K, p.M, lda, p.a_blocks)
                         : make_tmap(&ta, A, p.K, p.M, lda, BK);
   if (rc != MRL_OK) return rc;
@@ -937,10 +973,10 @@ int launch_gemm(const void* A, long long lda, const void* B, long long ldb, Gemm
        : p.b_blocks ? make_tmap_mn_blocks(&tb, B, p.K, p.N, ldb, p.b_blocks)
                     : make_tmap(&tb, B, p.K, p.N, ldb, BK);
   if (rc != MRL_OK) return rc;
-  p.m_tiles = (p.M + BM * kC - 1) / (BM * kC);
+  p.m_tiles = (p.M + BM * kC * kR - 1) / (BM * kC * kR);
   if (m_rows != nullptr) {
-    p.m_list = kC == 2 ? m_rows->m256 : m_rows->m128;
-    p.m_count = m_rows->counts + (kC == 2 ? 0 : 1);
+    p.m_list = kC * kR == 2 ? m_rows->m256 : m_rows->m128;
+    p.m_count = m_rows->counts + (kC * kR == 2 ? 0 : 1);
   }
   if (k_rows != nullptr) {
     p.k_list = k_rows->k64;
@@ -949,7 +985,7 @@ int launch_gemm(const void* A, long long lda, const void* B, long long ldb, Gemm
   // rows of A per raster group: the group's rows of A stay in L2 while B streams past them, so B is fetched from
   // DRAM once per group -- the taller the group the better, as long as its A panel (rows x K) fits L2 beside the
   // stream (measured: 4,096 rows at K = 4,096, 2,048 rows at K >= 16,384; DRAM traffic costs clock under the power cap)
-  p.group_m = (p.K <= 8192 ? 4096 : 2048) / (BM * kC);
+  p.group_m = (p.K <= 8192 ? 4096 : 2048) / (BM * kC * kR);
   const long long tiles = (long long)p.m_tiles * p.n_tiles;
   if (tiles > 0x7fffffffll) return MRL_ERR_UNSUPPORTED_SHAPE;
   if (kC == 2) {
@@ -961,6 +997,15 @@ int launch_gemm(const void* A, long long lda, const void* B, long long ldb, Gemm
     return e == cudaSuccess ? MRL_OK : MRL_ERR_CUDA;
   }
   const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
+  if constexpr (kTallShape) {
+    if (tall) {
+      mrl_profile_before(st, "lmhead_gemm_kernel (tall tiles)");
+      lmhead_gemm_kernel<EPI, 1, kAMn, kBMn, 2><<<grid, kGemmThreads, GemmCfg<1, 2>::kSmem, st>>>(ta, tb, p);
+      mrl_profile_after(st);
+      MRL_CUDA_OK(cudaGetLastError());
+      return MRL_OK;
+    }
+  }
   mrl_profile_before(st, "lmhead_gemm_kernel");
   lmhead_gemm_kernel<EPI, 1, kAMn, kBMn><<<grid, kGemmThreads, GemmCfg<1>::kSmem, st>>>(ta, tb, p);
   mrl_profile_after(st);

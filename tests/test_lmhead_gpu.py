@@ -392,3 +392,49 @@ def test_long_k_twin_every_row_live_dW_and_dHidden_element_by_element():
     rows_err = (got["dH"][keep].double() - ref["dHidden"][keep]).norm(dim=1) / ref["dHidden"][keep].norm(dim=1).clamp_min(1e-30)
     live = ref["g"][keep] != 0
     assert float(rows_err[live].max()) <= 4 * GRAD_REL_L2_BF16
+
+
+def test_tall_tile_dW_matches_oracle_with_dead_row_blocks():
+    """A dW product large enough for the 256-row tiles of a single CTA (K = 8,192 rows, 64 x 3 tall tiles): the step's
+    last launch must be that kernel, and dW / dHidden must match the oracle with whole 256-row blocks of rows dead
+    (zero-advantage sequences), i.e. with the K-block list of the long product in use."""
+    N, H, V, S = 8192, 768, 16384, 32
+    g = torch.Generator().manual_seed(33)
+    hidden = torch.randn(N, H, generator=g).to(torch.bfloat16)
+    W = (torch.randn(V, H, generator=g) * (2.0 / H ** 0.5)).to(torch.bfloat16)
+    ids = torch.randint(0, V, (N,), generator=g, dtype=torch.int32)
+    cu = torch.arange(0, N + 1, N // S, dtype=torch.int32)
+    adv = torch.randn(S, generator=g)
+    adv[::4] = 0.0                                                  # every fourth sequence (256 rows) has no gradient
+    z = hidden.double() @ W.double().T
+    logp, _, _ = O.token_logprobs(z, ids)
+    del z
+    logp_old = (logp + 0.1 * torch.randn(N, generator=g, dtype=torch.float64)).float()
+    # A token whose ratio sits on a clip bound may be clipped on one side only, and its gradient row reaches every row
+    # of dW: such tokens (one or two in 8,192) are masked out, so that the element-wise comparison below is decided
+    rho = torch.exp(logp - logp_old.double())
+    mask = (torch.minimum((rho - 0.8).abs(), (rho - 1.2).abs()) >= 1e-4).to(torch.uint8)
+    assert int((mask == 0).sum()) <= 16
+    lp = make_lp()
+    with B.DominantKernelTimer(8) as timer:
+        got = run_gpu_lmhead(hidden, W, ids, mask, cu, adv, logp_old, None, None, lp)
+    assert "tall" in timer.last_kernel, timer.last_kernel
+    ref = O.fused_lmhead_loss(hidden, W, ids, mask, cu, adv, logp_old, None, None, oracle_lp(lp))
+    assert got["status"] == 0 and not bool((ref["valid"] & (ref["margin"] < TIE_MARGIN)).any())
+    assert (got["logp"].double() - ref["logp"]).abs().max() <= LOGP_ATOL
+    assert loss_close(got["loss"][0], ref["loss_pg"], ref["pg_term"].abs().sum())
+    assert rel_l2(got["dH"].double(), ref["dHidden"]) <= GRAD_REL_L2_BF16
+    assert float(got["dH"][ref["g"] == 0].float().abs().max()) == 0
+    assert rel_l2(got["dW"].double(), ref["dW"]) <= GRAD_REL_L2_BF16
+    # Element by element.  Every entry of dW is a sum over the tokens of terms of both signs; it is held against the same
+    # product taken from the oracle's dZ rounded to bf16 (the tensor-core operand type), where only the float32
+    # accumulation order, the bf16 rounding of the output and one-ulp differences between the two roundings of dZ remain
+    # (the kernel's dZ is good to 1e-5, so a few per mille of its elements round the other way, each by one bf16 ulp, at most 2^-7
+    # of its own term): the bound is 2^-7 of the sum of the magnitudes of an entry's terms, half a typical entry here,
+    # where a tile read from the wrong place would be off by whole entries.
+    dq = ref["dlogits"].bfloat16().double()
+    dW_q = dq.T @ hidden.double()
+    tol = 2.0 ** -7 * (dq.abs().T @ hidden.double().abs()) + 2.0 ** -8 * dW_q.abs()
+    bad = (got["dW"].double() - dW_q).abs() > tol
+    assert not bool(bad.any()), f"{int(bad.sum())} dW entries beyond their bound, rows {bad.any(dim=1).nonzero()[:8, 0].tolist()}"
+    assert float(tol.mean()) < float(dW_q.abs().mean())                 # the bound is tighter than the entries
