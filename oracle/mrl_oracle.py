@@ -318,7 +318,7 @@ def kl_penalty(logp, logp_ref, c, lp: LossParams):
         L_KL = beta * sum_t c_t k(d_t),      dL_KL/dlogp_t = beta c_t k'(d_t),
         k1' = 1,  k2' = d,  k3' = 1 - exp(-d).
 
-    Returns dict: kl_term f64[N] (beta c_t k_t), g_kl f64[N] (the part of g_t: -dL_KL/dlogp_t), d.
+    Returns dict: kl_term f64[N] (beta c_t k_t), g_kl f64[N] (the part of g_t: -dL_KL/dlogp_t), d, w (beta c_t).
     """
     logp = torch.as_tensor(logp).to(F64)
     d = logp - torch.as_tensor(logp_ref).to(F64)
@@ -333,7 +333,7 @@ def kl_penalty(logp, logp_ref, c, lp: LossParams):
     w = lp.kl_coeff * c
     on = w != 0
     zero = torch.zeros_like(d)
-    return dict(kl_term=torch.where(on, w * k, zero), g_kl=torch.where(on, -w * dk, zero), d=d)
+    return dict(kl_term=torch.where(on, w * k, zero), g_kl=torch.where(on, -w * dk, zero), d=d, w=w)
 
 
 def policy_loss(logits, ids, mask, cu_seqlens, adv_seq, logp_old, tok_weight=None, nll_weight=None,
@@ -365,6 +365,7 @@ def policy_loss(logits, ids, mask, cu_seqlens, adv_seq, logp_old, tok_weight=Non
         _, c, _ = row_coefficients(valid, cu_seqlens, adv_seq, None, None, lp)     # c_t alone (u_t = 1)
         kl = kl_penalty(logp, logp_ref, c, lp)
         out["g"] = sur["g"] = sur["g"] + kl["g_kl"]
+        out["g_kl"], out["kl_w"] = kl["g_kl"], kl["w"]     # the penalty's share of g and beta c_t, kept for the tests' error scale
         out["kl_term"] = kl["kl_term"]
         out["loss_kl"] = float(kl["kl_term"].sum())
     out["stats"] = (int(valid.sum()), int((valid & (A != 0) & sur["clipped"]).sum()))
@@ -456,6 +457,7 @@ def policy_loss_sequence_ratio(logits, ids, mask, cu_seqlens, adv_seq, logp_old,
         _, c, _ = row_coefficients(valid, cu_seqlens, adv_seq, None, None, lp)
         kl = kl_penalty(logp, logp_ref, c, lp)
         out["g"] = sur["g"] = sur["g"] + kl["g_kl"]
+        out["g_kl"], out["kl_w"] = kl["g_kl"], kl["w"]     # the penalty's share of g and beta c_t, kept for the tests' error scale
         out["kl_term"] = kl["kl_term"]
         out["loss_kl"] = float(kl["kl_term"].sum())
     cu = torch.as_tensor(cu_seqlens).long()

@@ -115,20 +115,29 @@ def compare_policy_loss(got, ref, V, dtype, check_stats=True, loss_floor=0.0, ca
         assert torch.isfinite(dz).all()
         keep = ~tie
         tol = GRAD_REL_L2_BF16 if dtype == torch.bfloat16 else GRAD_REL_L2_F32
-        e = rel_l2(dz[keep], want[keep])
-        assert e <= tol, f"dlogits rel L2 {e}"
+        # (a row whose softmax is nearly one-hot has dz = g (p - onehot) ~ 0 from 1 - p, which float32 carries to 1e-7
+        # absolute, not relative: such a row counts with |g|, the scale of its entries' parts, in the norm below)
+        row_scale = torch.maximum(want[keep].norm(dim=1), ref["g"][keep].abs())
+        e = float((dz[keep] - want[keep]).norm()) / max(float(row_scale.norm()), 1e-300)
+        assert e <= tol or float((dz[keep] - want[keep]).norm()) == 0, f"dlogits rel L2 {e}"
         # rows that must be exactly zero are exactly zero
         zero_rows = keep & (ref["g"] == 0)
         assert dz[zero_rows].abs().max() == 0 if zero_rows.any() else True
         # per-row check on rows with a gradient: no single row hides behind the global norm
         live = keep & (ref["g"] != 0)
         if live.any():
-            # (g = c u A rho + cn may cancel: the error scales with |c u A rho| + |cn|, not with |g|)
+            # (g = c u A rho + cn - beta c k'(d) may cancel: the error scales with the magnitudes of its parts, not with |g|)
             num = (dz[live] - want[live]).norm(dim=1)
-            cancel = ((ref["g"] - ref["cn"]).abs() + ref["cn"].abs())[live] / ref["g"][live].abs()
+            g_kl = ref["g_kl"] if "g_kl" in ref else torch.zeros_like(ref["g"])
+            cancel = ((ref["g"] - ref["cn"] - g_kl).abs() + ref["cn"].abs() + g_kl.abs())[live] / ref["g"][live].abs()
             # and a row whose softmax is (nearly) one-hot has dz ~ 0: measure against |g|, the scale of g (p - onehot)
             den = torch.maximum(want[live].norm(dim=1), ref["g"][live].abs()) * cancel
-            assert (num / den).max() <= 2 * tol, f"worst row rel L2 {(num / den).max()}"
+            # The slopes k2' = d and k3' = 1 - exp(-d) move one for one with the log-prob, which a float32 carries to
+            # about 1e-6 at |logp| ~ 10: that share of g is off by up to beta c_t 2e-6 however small d makes it.
+            slack = torch.zeros_like(num)
+            if "kl_w" in ref:
+                slack = (ref["kl_w"].abs() * 2e-6 / ref["g"].abs())[live] * want[live].norm(dim=1)
+            assert ((num - slack).clamp_min(0) / den).max() <= 2 * tol, f"worst row rel L2 {(num / den).max()}"
         for r in tie.nonzero()[:, 0].tolist():      # near-tie rows: either side of the clip is valid
             alt = rel_l2(dz[r], want[r])
             assert alt <= tol or dz[r].abs().max() == 0 or want[r].abs().max() == 0

@@ -92,7 +92,10 @@ def test_logits_in_random_case(seed):
     # vocabulary with a dominant logit) cannot be held to 1e-5 of itself: floor at 2e-2 of the sum of its coefficients (2e-7 absolute per log-prob).
     compare_policy_loss(got, ref, c["V"], c["dtype"], cancelling=True, loss_floor=2e-2 * float(ref["cn"].abs().sum()))
     if kl is not None:
-        assert loss_close(kl.value(), ref["loss_kl"], ref["kl_term"].abs().sum())
+        # (every estimator's slope is at most max(1, |d|) and a float32 log-prob is good to about 1e-6: the term is off
+        # by up to that times the coefficients, which sum to beta = 0.01, however small its own value is)
+        scale = max(abs(ref["loss_kl"]), 0.1 * float(ref["kl_term"].abs().sum()))
+        assert abs(kl.value() - ref["loss_kl"]) <= 1e-5 * scale + 1e-6 * 0.01
 
 
 def _draw_lmhead_case(seed):
@@ -266,13 +269,17 @@ def test_hidden_in_random_options(seed):
         # k1 is linear in a log-prob that carries the error of a float32-accumulated bf16 dot product (a few 1e-7, and
         # not zero-mean: the tensor core does not round its accumulator to nearest), so the term is held relative to
         # the sum of its |terms|, as in tests/test_kl_gpu.py
+        # (and every estimator's slope is at most max(1, |d|): a one-token batch whose d is small has a term far below
+        # the 4e-6 this path's log-probs are good to at H <= 320, times the coefficients, which sum to beta = 0.02)
         scale = max(abs(ref["loss_kl"]), float(ref["kl_term"].abs().sum()))
-        assert abs(kl.value() - ref["loss_kl"]) <= 1e-5 * scale + 1e-12
+        assert abs(kl.value() - ref["loss_kl"]) <= 1e-5 * scale + 4e-6 * 0.02
     if with_ent:
         ref_ent = O.token_entropy(zz, ids, mask)
         e = ent.cpu().double()
         read = e != 0 if lp.flags & B.FLAG_SKIP_ZERO_ROWS else torch.ones(N, dtype=torch.bool)
-        assert torch.isfinite(e).all() and (e - ref_ent)[read].abs().max() <= 1e-4
+        assert torch.isfinite(e).all()
+        if read.any():
+            assert (e - ref_ent)[read].abs().max() <= 1e-4
 
 
 @pytest.mark.parametrize("seed", range(12))
@@ -310,6 +317,14 @@ def test_host_pipeline_random_case(seed):
     assert torch.equal(got["logp"], one["logp"])
     assert torch.equal(got["dlogits"].view(bits), one["dlogits"].view(bits))
     assert torch.equal(got["stats"], one["stats"])
+    # the loss: float32 sums in another order (per micro-batch, then accumulated), so the two agree to a few float32
+    # roundings of the total magnitude of the terms, which the oracle provides (the loss itself may cancel to far less)
+    if seq_level:
+        ref = O.policy_loss_sequence_ratio(z, ids, mask, cu, adv, old, nllw, oracle_lp(mk()), want_dlogits=False)
+        mags = (float(ref["seq_term"].abs().sum()), float(ref["nll_term"].abs().sum()))
+    else:
+        ref = O.policy_loss(z, ids, mask, cu, adv, old, tw, nllw, oracle_lp(mk()), want_dlogits=False)
+        mags = (float(ref["pg_term"].abs().sum()), float(ref["nll_term"].abs().sum()))
     for k in range(2):
         a, b = float(got["loss"][k]), float(one["loss"][k])
-        assert abs(a - b) <= 2e-6 * max(abs(a), abs(b)) + 1e-9          # float32 sums in another order
+        assert abs(a - b) <= 2e-6 * max(abs(a), abs(b), mags[k]) + 1e-12
