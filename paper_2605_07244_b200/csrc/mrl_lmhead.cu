@@ -911,14 +911,17 @@ struct TileLists {
   int *m256, *m128, *k64, *counts;
 };
 
-// Whether a product with both operands MN-major (dW) takes tall tiles: its K must be long enough that the epilogue, which
-// a tall tile cannot overlap with the next tile's MMAs (about 5,000 cycles against 1,024 per K-block), stays a few per
-// cent, and there must be at least one tall tile per SM.  Measured on the dW product of a 16,384-column chunk at
-// K = 65,536: 7.2 -> 6.3-6.4 ms, at a clock only 3 % lower (pairs of CTAs gain the same activity and lose it to clock).
-// The dHidden product (K = 16,384, float32 read-modify-write epilogue) measured slower with tall tiles and keeps 128 rows.
+// Whether a product with both operands MN-major (dW) takes tall tiles: its K must be long enough to pay for the
+// epilogue, which a tall tile cannot overlap with the next tile's MMAs, and there must be a tall tile per SM.
+// Measured on B200, one 16,384 x 4,096 product, tall against 128-row tiles (ms): bf16 store K = 2,048 0.199 / 0.199,
+// 4,096 0.359 / 0.379, 8,192 0.689 / 0.768, 65,536 6.08 / 6.77; float32 accumulate (read-modify-write epilogue)
+// 8,192 0.808 / 0.800, 16,384 1.483 / 1.536, 65,536 5.95 / 6.62 -- at a clock only 3 % lower inside the step, where
+// pairs of CTAs gain the same activity and lose it to clock.  The dHidden product (K = 16,384, float32 read-modify-write
+// of a tile as large as its mainloop is short) measured slower with tall tiles and keeps 128 rows.
 bool tall_policy(const GemmParams& p) {
   const long long tall_tiles = (long long)((p.M + 2 * BM - 1) / (2 * BM)) * ((p.N + BN - 1) / BN);
-  return p.K >= 8192 && tall_tiles >= sm_count();
+  const int min_k = p.c_mode == C_BF16 ? 4096 : 16384;
+  return p.K >= min_k && tall_tiles >= sm_count();
 }
 
 // `m_rows` / `k_rows`: the M (resp. K) dimension of the product is the batch's rows and only the listed blocks count.
