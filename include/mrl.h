@@ -105,7 +105,8 @@ extern "C" {
 #define MRL_FLAG_ACCUMULATE_DW 4u     /* fused LM head: dW is float32 [V, H] and is added to, not overwritten */
 #define MRL_FLAG_PAIR_TILES 8u        /* fused LM head: 256-row tiles worked by pairs of CTAs (tcgen05 cta_group::2).
                                          Same results.  Faster for a product timed alone; inside a long
-                                         power-capped step the default 128-row tiles were faster on B200 */
+                                         power-capped step the default tiles (one CTA each: 128 rows, 256 rows for the
+                                         long-K dW product) were faster on B200 */
 
 /* `which` of mrl_workspace_bytes */
 #define MRL_WS_TOKEN_LOGPROBS 0
